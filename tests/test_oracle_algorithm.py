@@ -1,0 +1,97 @@
+"""Pins for the oracle's composition of Algorithm 1."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import QSpec
+
+QS = {
+    "identity": QSpec(oracle.IDENTITY),
+    "sign1": QSpec(oracle.SIGN1, chunk=128),
+    "topk": QSpec(oracle.TOPK, k=37),
+    "qsgd": QSpec(oracle.QSGD, chunk=128, levels=15),
+}
+PAIRS = [("identity", "identity"), ("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"),
+         ("sign1", "topk"), ("topk", "identity"), ("qsgd", "sign1")]
+
+
+def _grads(n, d, T, seed=0):
+    r = np.random.default_rng(seed)
+    mu = r.standard_normal((n, d)).astype(np.float32)
+    return [(mu + 0.5 * r.standard_normal((n, d))).astype(np.float32) for _ in range(T)]
+
+
+def test_identity_reduces_to_parallel_sgd_bitwise():
+    n, d, T, gamma = 4, 1000, 6, 0.1
+    gs = _grads(n, d, T)
+    st = oracle.State.zeros(n, d)
+    x = np.zeros(d, dtype=np.float32)
+    for t, g in enumerate(gs):
+        oracle.step(st, g, QS["identity"], QS["identity"], gamma, 0, t)
+        # parallel SGD: x <- x - gamma * (1/n) sum_i g_i  (Section 1), same fp32 evaluation order
+        acc = np.zeros(d, dtype=np.float32)
+        for i in range(n):
+            acc = acc + g[i]
+        x = x - np.float32(gamma) * (acc * np.float32(1.0 / n))
+        assert np.array_equal(st.x, x)
+        assert not st.delta_w.any() and not st.delta_s.any()
+
+
+@pytest.mark.parametrize("wq,sq", PAIRS)
+def test_residual_reconstructs_compensated_gradient(wq, sq):
+    n, d, gamma = 3, 700, 0.1
+    st = oracle.State.zeros(n, d)
+    for t, g in enumerate(_grads(n, d, 3, seed=5)):
+        old_w, old_s = st.delta_w.copy(), st.delta_s.copy()
+        C_all = oracle.worker_pass(st, g, QS[wq], 1, t)
+        v_w = g + old_w
+        tol = 2.0**-23 * np.maximum(np.abs(v_w), np.abs(C_all))
+        assert np.all(np.abs((C_all.astype(np.float64) + st.delta_w) - v_w) <= tol)
+        if wq in ("identity", "topk"):
+            assert np.array_equal(C_all + st.delta_w, v_w)
+        Cv = oracle.server_pass(st, C_all, QS[sq], 1, t)
+        v_s = oracle.server_mean_add(C_all, old_s)
+        tol = 2.0**-23 * np.maximum(np.abs(v_s), np.abs(Cv))
+        assert np.all(np.abs((Cv.astype(np.float64) + st.delta_s) - v_s) <= tol)
+        st.x = oracle.apply_update(st.x, Cv, gamma)
+
+
+@pytest.mark.parametrize("wq,sq", PAIRS)
+def test_telescoping_identity_of_the_global_update_rule(wq, sq):
+    """Eq. 5-6: y_t = x_t - gamma * Omega_{t-1} follows plain SGD for any Q, so after T steps
+    x_T - gamma * (delta_T + mean_i delta_T^(i)) = x_0 - gamma * sum_t mean_i g_t^(i)."""
+    n, d, T, gamma = 4, 640, 25, 0.1
+    gs = _grads(n, d, T, seed=9)
+    x0 = np.random.default_rng(1).standard_normal(d).astype(np.float32)
+    st = oracle.State.zeros(n, d, x0)
+    for t, g in enumerate(gs):
+        oracle.step(st, g, QS[wq], QS[sq], gamma, 3, t)
+    rhs = x0.astype(np.float64) - gamma * sum(g.astype(np.float64).mean(axis=0) for g in gs)
+    omega = st.delta_s.astype(np.float64) + st.delta_w.astype(np.float64).mean(axis=0)
+    lhs = st.x.astype(np.float64) - gamma * omega
+    scale = max(np.abs(rhs).max(), max(np.abs(g).max() for g in gs))
+    assert np.max(np.abs(lhs - rhs)) <= 40 * T * 2.0**-24 * scale
+
+
+@pytest.mark.parametrize("wq,sq", [("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd")])
+def test_error_stays_bounded_on_stationary_gradients(wq, sq):
+    """Section 4: a contracting Q keeps ||delta_t|| bounded; a broken residual makes it grow."""
+    n, d, T = 2, 512, 120
+    st = oracle.State.zeros(n, d)
+    norms = []
+    for t, g in enumerate(_grads(n, d, T, seed=2)):
+        oracle.step(st, g, QS[wq], QS[sq], 0.1, 8, t)
+        norms.append(np.linalg.norm(st.delta_w) + np.linalg.norm(st.delta_s))
+    assert max(norms[T // 2:]) <= 1.5 * max(norms[:T // 2]) + 1e-6
+
+
+def test_server_uses_its_own_stream_and_workers_differ():
+    n, d = 2, 256
+    g = np.tile(np.random.default_rng(3).standard_normal(d).astype(np.float32), (n, 1))
+    st = oracle.State.zeros(n, d)
+    oracle.worker_pass(st, g, QS["qsgd"], 4, 0)
+    a, b = st.worker_payloads
+    assert not np.array_equal(a["lvl"], b["lvl"])          # same v, different worker stream
+    v = oracle.ef_add(g[0], np.zeros(d, dtype=np.float32))
+    _, as_server = oracle.q_qsgd(v, 128, 15, 4, 0, oracle.SERVER_WID)
+    assert not np.array_equal(a["lvl"], as_server["lvl"])
