@@ -1,0 +1,203 @@
+/*
+ * dsq.h -- C ABI of the DoubleSqueeze step library (CUDA, sm_100a).
+ *
+ * One iteration of DoubleSqueeze (Algorithm 1 of arXiv:1905.05957) with the n
+ * workers held as the rows of one [n, d] fp32 tensor on a single GPU:
+ *
+ *   worker  i :  v_i = g_i + delta_i          (Section 3.1, Eq. 2)
+ *                send Q[v_i]                  (Algorithm 1, "Compress")
+ *                delta_i = v_i - Q[v_i]       (Eq. 3)
+ *   server    :  v = delta + (1/n) sum_i Q[v_i]
+ *                send Q[v];  delta = v - Q[v] (Eq. 4)
+ *   worker    :  x = x - gamma Q[v]           (Algorithm 1, "Update the local model")
+ *
+ * Q is one of the compression options of Section 3.2 / Section 5.1; the worker
+ * pass and the server pass may use different ones.
+ *
+ * General rules
+ *  - Every pointer in ds_buffers, and the gradient g, is DEVICE memory owned by
+ *    the caller.  The library allocates no device memory and keeps no copy of g.
+ *    The handle is host memory only.
+ *  - ds_worker_compress / ds_server_aggregate_compress / ds_apply_update only
+ *    enqueue work on the given CUDA stream (a cudaStream_t passed as void*; NULL
+ *    is the default stream); they never synchronise.  One handle must be used on
+ *    one stream at a time.
+ *  - Every function returns a ds_status.  Nothing throws across the boundary.
+ *    Conditions detected on the device are OR-ed into *dev_status (DS_DEV_*),
+ *    which the caller reads when it chooses; kernels never trap.
+ *  - All multi-byte payload fields are little-endian; all arithmetic is IEEE-754
+ *    binary32 round-to-nearest-even with no fused multiply-add.
+ */
+#ifndef DSQ_H_
+#define DSQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ds_ctx* ds_handle;
+
+typedef enum {
+  DS_OK = 0,
+  DS_NEED_BUFFERS = 1,          /* ds_create in query mode: *_bytes filled, no handle made */
+  DS_ERR_INVALID_ARG = -1,
+  DS_ERR_ALIGN = -2,            /* a buffer is not 16-byte aligned */
+  DS_ERR_BUFFER_TOO_SMALL = -3,
+  DS_ERR_STATE = -4,            /* calls out of order within a step */
+  DS_ERR_CUDA = -5,             /* a launch failed; see ds_last_error() */
+  DS_ERR_UNSUPPORTED = -6
+} ds_status;
+
+/* bits of *dev_status */
+#define DS_DEV_TOPK_INCONSISTENT 0x1u /* top-k selection counted a number of entries other than k */
+
+/* flags of ds_server_aggregate_compress */
+#define DS_FUSE_APPLY 0x1u /* also perform x = x - gamma Q[v]; ds_apply_update is then not called */
+
+/*
+ * Compression operators.
+ *
+ * DS_Q_IDENTITY  Q[v] = v.  The step is then plain parallel SGD (Section 1).
+ *
+ * DS_Q_SIGN1     "1-bit compression" of Section 5.1 (Section 3.2 "1-Bit Quantization"): the sign
+ *                of every entry plus a scaling factor that restores the magnitude.  Here the
+ *                factor is the mean absolute value of each chunk of `chunk` consecutive entries
+ *                of the flat vector (the last chunk may be short; its true length divides).
+ *                bit = (v >= 0);  Q[v]_j = bit ? +s_c : -s_c.
+ *
+ * DS_Q_TOPK      "Top-k compression" of Section 5.1 (Section 3.2 "Top-k sparsification"): the k
+ *                entries of largest absolute value over the whole d-vector keep their value, all
+ *                others become 0.  Equal magnitudes are taken by lower index first.  Always
+ *                exactly k entries.
+ *
+ * DS_Q_QSGD      "Randomized Quantization" of Section 3.2: |v_j| is rounded at random to one of
+ *                its two neighbours on the grid {0, q, ..., levels*q}, q = N_c / levels, with the
+ *                probabilities that make it unbiased; N_c is the l2 norm of the entry's chunk of
+ *                `chunk` consecutive entries; the sign is kept.  Randomness: Philox4x32-10,
+ *                key = (seed low, seed high), counter = (offset_in_chunk/4, chunk index, worker
+ *                index or 0xFFFFFFFF on the server pass, step); entry uses output word
+ *                offset_in_chunk%4, top 24 bits, as a uniform in [0,1).
+ *
+ * Chunk reductions (sum of |v| or of v*v) are pairwise sums in index order over the chunk padded
+ * with zeros to `chunk` entries, so results do not depend on launch geometry.
+ */
+typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3 } ds_op;
+
+typedef struct {
+  int32_t op;        /* ds_op */
+  uint32_t chunk;    /* SIGN1, QSGD: a power of two in [128, 8192]; else ignored */
+  uint64_t k;        /* TOPK: 0 <= k <= d; else ignored */
+  uint32_t levels;   /* QSGD: 1 <= levels <= 255; else ignored */
+  uint32_t reserved; /* must be 0 */
+} ds_qspec;
+
+typedef struct {
+  uint32_t n;        /* workers, 1 <= n <= 65535 */
+  uint32_t reserved; /* must be 0 */
+  uint64_t d;        /* model dimension, 1 <= d < 2^32 */
+  float gamma;       /* learning rate, finite */
+  uint32_t reserved2;
+  ds_qspec worker_q; /* Q of the worker pass */
+  ds_qspec server_q; /* Q of the server pass */
+  uint64_t seed;     /* Philox key for DS_Q_QSGD */
+} ds_config;
+
+/*
+ * Caller-owned device buffers.  Layouts:
+ *   x        float[d]        model; the caller sets x_0
+ *   delta_w  float[n*d]      worker errors, row i = worker i; the caller zero-fills (delta = 0)
+ *   delta_s  float[d]        server error; the caller zero-fills
+ *   worker_payload           n payloads at a fixed stride, see ds_get_layout()
+ *   server_payload           one payload
+ *   workspace                scratch of the top-k path (contents are meaningless between calls);
+ *                            may be NULL when workspace_bytes is 0
+ *   dev_status uint32[1]     the caller zero-fills
+ * Every non-NULL pointer must be 16-byte aligned and at least *_bytes long.
+ */
+typedef struct {
+  float* x;
+  float* delta_w;
+  float* delta_s;
+  void* worker_payload;
+  void* server_payload;
+  void* workspace;
+  uint32_t* dev_status;
+  size_t x_bytes, delta_w_bytes, delta_s_bytes;
+  size_t worker_payload_bytes, server_payload_bytes, workspace_bytes;
+} ds_buffers;
+
+/*
+ * Byte layout of one payload.  `stride` is the distance between consecutive workers' payloads
+ * (for the server payload: its total size).  Sub-array i starts `off[i]` bytes into the payload,
+ * is 16-byte aligned and holds `count[i]` elements:
+ *   IDENTITY  [0] float c[d]
+ *   SIGN1     [0] uint32 bits[ceil(d/32)]  entry j -> bit j%32 of word j/32, pad bits 0
+ *             [1] float  scale[ceil(d/chunk)]
+ *   TOPK      [0] uint32 idx[k] ascending  [1] float val[k] (bit copies of v[idx])
+ *   QSGD      [0] uint8  lvl[d]            [1] uint32 sgn[ceil(d/32)] (bit = v >= 0)
+ *             [2] float  norm[ceil(d/chunk)] (0 for a chunk sent as all zeros)
+ */
+typedef struct {
+  uint64_t stride;
+  uint64_t off[3];
+  uint64_t count[3];
+} ds_payload_layout;
+
+/* Host-only.  which = 0: worker payload, 1: server payload.  DS_ERR_INVALID_ARG on a bad config. */
+int ds_get_layout(const ds_config* cfg, int which, ds_payload_layout* out);
+
+/*
+ * Algorithm 1, "Input": fixes n, d, gamma and the operators.  Host-only; launches nothing.
+ * Query mode: with bufs->x == NULL every *_bytes field of *bufs is filled and DS_NEED_BUFFERS is
+ * returned (handle untouched).  Otherwise pointers and sizes are checked (DS_ERR_INVALID_ARG,
+ * DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL) and a handle is returned in *out.
+ */
+int ds_create(const ds_config* cfg, ds_buffers* bufs, ds_handle* out);
+
+/*
+ * Algorithm 1, "On worker" (Eq. 2, compress, Eq. 3) for all n workers.
+ * g: device float[n*d], row i = gradient of worker i; read once, not retained.
+ * step: iteration number t (enters the random stream only).
+ * Writes worker_payload and delta_w.  DS_ERR_STATE unless the previous step is complete.
+ */
+int ds_worker_compress(ds_handle h, const float* g, uint32_t step, void* cuda_stream);
+
+/*
+ * Algorithm 1, "On parameter server" (Eq. 4): decode the n worker payloads, average in worker
+ * order, add delta_s, compress, keep the residual.  Writes server_payload and delta_s; with
+ * DS_FUSE_APPLY also updates x and completes the step.  DS_ERR_STATE unless ds_worker_compress
+ * was the previous call.
+ */
+int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, void* cuda_stream);
+
+/*
+ * Algorithm 1, "Update the local model": x = x - gamma Q[v], decoded from server_payload.
+ * DS_ERR_STATE unless an unfused ds_server_aggregate_compress was the previous call.
+ */
+int ds_apply_update(ds_handle h, void* cuda_stream);
+
+/* Frees the host handle.  Device buffers stay the caller's. */
+int ds_destroy(ds_handle h);
+
+/*
+ * Convenience for callers that hold data in HOST memory: copies g_host (float[n*d], ideally
+ * pinned) into the caller's device staging buffer g_dev, runs worker + server(+fused apply), and
+ * copies the server payload and/or x back to host if the respective pointer is non-NULL.  All
+ * on `cuda_stream`, asynchronously; the caller synchronises the stream before reading.
+ */
+int ds_step_host(ds_handle h, const float* g_host, float* g_dev, uint32_t step, void* server_payload_host,
+                 float* x_host, void* cuda_stream);
+
+/* Text of the most recent CUDA error seen by this thread's calls ("" if none). */
+const char* ds_last_error(void);
+
+/* Library version, major*100 + minor. */
+int ds_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSQ_H_ */

@@ -1,0 +1,220 @@
+"""ctypes binding of the C ABI in include/dsq.h.  Argument marshalling only.
+
+PyTorch appears here for device memory and streams; every step of the path runs in the
+library's kernels.  There is no CPU fallback: a missing library or device raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from .workloads import Q, Workload
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libdsq.so")
+
+DS_OK, DS_NEED_BUFFERS = 0, 1
+DS_ERR_INVALID_ARG, DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL = -1, -2, -3
+DS_ERR_STATE, DS_ERR_CUDA, DS_ERR_UNSUPPORTED = -4, -5, -6
+DS_FUSE_APPLY = 1
+DS_DEV_TOPK_INCONSISTENT = 1
+OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3}
+EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
+           "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version")
+
+
+class ds_qspec(C.Structure):
+    _fields_ = [("op", C.c_int32), ("chunk", C.c_uint32), ("k", C.c_uint64), ("levels", C.c_uint32),
+                ("reserved", C.c_uint32)]
+
+
+class ds_config(C.Structure):
+    _fields_ = [("n", C.c_uint32), ("reserved", C.c_uint32), ("d", C.c_uint64), ("gamma", C.c_float),
+                ("reserved2", C.c_uint32), ("worker_q", ds_qspec), ("server_q", ds_qspec), ("seed", C.c_uint64)]
+
+
+class ds_buffers(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("delta_w", C.c_void_p), ("delta_s", C.c_void_p),
+                ("worker_payload", C.c_void_p), ("server_payload", C.c_void_p), ("workspace", C.c_void_p),
+                ("dev_status", C.c_void_p),
+                ("x_bytes", C.c_size_t), ("delta_w_bytes", C.c_size_t), ("delta_s_bytes", C.c_size_t),
+                ("worker_payload_bytes", C.c_size_t), ("server_payload_bytes", C.c_size_t),
+                ("workspace_bytes", C.c_size_t)]
+
+
+class ds_payload_layout(C.Structure):
+    _fields_ = [("stride", C.c_uint64), ("off", C.c_uint64 * 3), ("count", C.c_uint64 * 3)]
+
+
+class DsqError(RuntimeError):
+    def __init__(self, code: int, what: str, detail: str = ""):
+        super().__init__(f"{what} failed with ds_status {code}" + (f": {detail}" if detail else ""))
+        self.code = code
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads csrc/libdsq.so (built by build.py).  Raises if it is absent: there is no other path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_1905_05957_b200.build` "
+                           "(or __graft_entry__.build()); this package has no fallback implementation")
+    L = C.CDLL(LIB_PATH)
+    vp, u32 = C.c_void_p, C.c_uint32
+    L.ds_get_layout.argtypes = [C.POINTER(ds_config), C.c_int, C.POINTER(ds_payload_layout)]
+    L.ds_create.argtypes = [C.POINTER(ds_config), C.POINTER(ds_buffers), C.POINTER(vp)]
+    L.ds_worker_compress.argtypes = [vp, vp, u32, vp]
+    L.ds_server_aggregate_compress.argtypes = [vp, u32, u32, vp]
+    L.ds_apply_update.argtypes = [vp, vp]
+    L.ds_destroy.argtypes = [vp]
+    L.ds_step_host.argtypes = [vp, vp, vp, u32, vp, vp, vp]
+    L.ds_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        if getattr(L, name).restype is not C.c_char_p:
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _qspec(q: Q) -> ds_qspec:
+    return ds_qspec(OPS[q.op], q.chunk, q.k, q.levels, 0)
+
+
+def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int) -> ds_config:
+    return ds_config(n, 0, d, gamma, 0, _qspec(worker_q), _qspec(server_q), seed)
+
+
+def get_layout(cfg: ds_config, which: int) -> ds_payload_layout:
+    out = ds_payload_layout()
+    rc = load_library().ds_get_layout(C.byref(cfg), which, C.byref(out))
+    if rc != DS_OK:
+        raise DsqError(rc, "ds_get_layout")
+    return out
+
+
+_VIEW_DTYPES = {
+    "identity": (("c", torch.float32),),
+    "sign1": (("bits", torch.int32), ("scale", torch.float32)),
+    "topk": (("idx", torch.int32), ("val", torch.float32)),
+    "qsgd": (("lvl", torch.uint8), ("sgn", torch.int32), ("norm", torch.float32)),
+}
+
+
+def payload_views(buf: torch.Tensor, layout: ds_payload_layout, op: str, rows: int) -> list[dict]:
+    """Typed views of the sub-arrays of each payload inside the raw byte buffer (no copies).
+    uint32 fields are exposed as int32 tensors with the same bits."""
+    out = []
+    for i in range(rows):
+        base = i * layout.stride
+        views = {}
+        for j, (name, dt) in enumerate(_VIEW_DTYPES[op]):
+            nbytes = layout.count[j] * torch.empty(0, dtype=dt).element_size()
+            views[name] = buf[base + layout.off[j]: base + layout.off[j] + nbytes].view(dt)
+        out.append(views)
+    return out
+
+
+class DoubleSqueeze:
+    """One DoubleSqueeze state (x, delta_w, delta_s) on one GPU, stepped through the C ABI."""
+
+    def __init__(self, n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int = 0,
+                 device: str | torch.device = "cuda", x0: torch.Tensor | None = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_1905_05957_b200 needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.device = torch.device(device)
+        self.n, self.d, self.gamma, self.seed = n, d, gamma, seed
+        self.worker_q, self.server_q = worker_q, server_q
+        self.cfg = make_config(n, d, gamma, worker_q, server_q, seed)
+        bufs = ds_buffers()
+        rc = self.lib.ds_create(C.byref(self.cfg), C.byref(bufs), None)
+        if rc != DS_NEED_BUFFERS:
+            raise DsqError(rc, "ds_create (size query)")
+        dev = self.device
+        self.x = torch.zeros(d, dtype=torch.float32, device=dev) if x0 is None else \
+            x0.to(device=dev, dtype=torch.float32).contiguous().clone()
+        self.delta_w = torch.zeros(n, d, dtype=torch.float32, device=dev)
+        self.delta_s = torch.zeros(d, dtype=torch.float32, device=dev)
+        self.worker_payload = torch.zeros(bufs.worker_payload_bytes, dtype=torch.uint8, device=dev)
+        self.server_payload = torch.zeros(bufs.server_payload_bytes, dtype=torch.uint8, device=dev)
+        self.workspace = torch.zeros(max(bufs.workspace_bytes, 16), dtype=torch.uint8, device=dev)
+        self.dev_status = torch.zeros(4, dtype=torch.int32, device=dev)
+        bufs.x, bufs.delta_w, bufs.delta_s = self.x.data_ptr(), self.delta_w.data_ptr(), self.delta_s.data_ptr()
+        bufs.worker_payload, bufs.server_payload = self.worker_payload.data_ptr(), self.server_payload.data_ptr()
+        bufs.workspace, bufs.dev_status = self.workspace.data_ptr(), self.dev_status.data_ptr()
+        self.bufs = bufs
+        self.workspace_bytes = bufs.workspace_bytes
+        h = C.c_void_p()
+        rc = self.lib.ds_create(C.byref(self.cfg), C.byref(bufs), C.byref(h))
+        if rc != DS_OK:
+            raise DsqError(rc, "ds_create")
+        self.handle = h
+        self.worker_layout = get_layout(self.cfg, 0)
+        self.server_layout = get_layout(self.cfg, 1)
+
+    @classmethod
+    def for_workload(cls, wl: Workload, device="cuda") -> "DoubleSqueeze":
+        return cls(wl.n, wl.d, wl.gamma, wl.worker_q, wl.server_q, wl.seed, device)
+
+    # -- the three calls of one iteration -----------------------------------------------------
+    def _stream(self, stream) -> int:
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        return s.cuda_stream
+
+    def _check(self, rc: int, what: str):
+        if rc != DS_OK:
+            raise DsqError(rc, what, self.lib.ds_last_error().decode())
+
+    def worker_compress(self, g: torch.Tensor, step: int, stream=None):
+        assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous() and g.numel() == self.n * self.d
+        self._check(self.lib.ds_worker_compress(self.handle, g.data_ptr(), step, self._stream(stream)),
+                    "ds_worker_compress")
+
+    def server_aggregate_compress(self, step: int, fuse_apply: bool = False, stream=None):
+        self._check(self.lib.ds_server_aggregate_compress(self.handle, step, DS_FUSE_APPLY if fuse_apply else 0,
+                                                          self._stream(stream)), "ds_server_aggregate_compress")
+
+    def apply_update(self, stream=None):
+        self._check(self.lib.ds_apply_update(self.handle, self._stream(stream)), "ds_apply_update")
+
+    def step(self, g: torch.Tensor, t: int, fuse_apply: bool = True, stream=None):
+        self.worker_compress(g, t, stream)
+        self.server_aggregate_compress(t, fuse_apply, stream)
+        if not fuse_apply:
+            self.apply_update(stream)
+
+    def step_host(self, g_host: torch.Tensor, g_dev: torch.Tensor, t: int, server_payload_host=None, x_host=None,
+                  stream=None):
+        """Host-buffer form: H2D of g, the fused step, D2H of the server payload and/or x; asynchronous."""
+        assert not g_host.is_cuda and g_host.is_contiguous() and g_dev.is_cuda
+        sp = server_payload_host.data_ptr() if server_payload_host is not None else None
+        xp = x_host.data_ptr() if x_host is not None else None
+        self._check(self.lib.ds_step_host(self.handle, g_host.data_ptr(), g_dev.data_ptr(), t, sp, xp,
+                                          self._stream(stream)), "ds_step_host")
+
+    # -- views ----------------------------------------------------------------------------------
+    def worker_views(self) -> list[dict]:
+        return payload_views(self.worker_payload, self.worker_layout, self.worker_q.op, self.n)
+
+    def server_views(self) -> dict:
+        return payload_views(self.server_payload, self.server_layout, self.server_q.op, 1)[0]
+
+    def device_status(self) -> int:
+        return int(self.dev_status[0].item())
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.ds_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

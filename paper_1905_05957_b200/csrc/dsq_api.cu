@@ -1,0 +1,324 @@
+// C ABI of the DoubleSqueeze step library: argument checking, payload layout, and the dispatch of
+// each call of Algorithm 1 onto the kernels.  Host code only; no device memory is allocated here.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "dsq_internal.h"
+
+using namespace dsq;
+
+namespace {
+
+thread_local char g_last_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char* where) {
+  snprintf(g_last_error, sizeof g_last_error, "%s: %s", where, cudaGetErrorString(e));
+  return DS_ERR_CUDA;
+}
+
+inline uint64_t round16(uint64_t b) { return (b + 15u) & ~uint64_t(15); }
+inline bool is_pow2(uint32_t x) { return x && !(x & (x - 1)); }
+inline uint32_t log2u(uint32_t x) { uint32_t l = 0; while ((1u << l) < x) ++l; return l; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool qspec_ok(const ds_qspec& q, uint64_t d) {
+  if (q.reserved != 0) return false;
+  switch (q.op) {
+    case DS_Q_IDENTITY: return true;
+    case DS_Q_SIGN1: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192;
+    case DS_Q_QSGD: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192 && q.levels >= 1 && q.levels <= 255;
+    case DS_Q_TOPK: return q.k <= d;
+    default: return false;
+  }
+}
+
+bool config_ok(const ds_config* c) {
+  if (!c) return false;
+  if (c->n < 1 || c->n > 65535 || c->reserved != 0) return false;
+  if (c->d < 1 || c->d >= (1ull << 32)) return false;
+  if (!std::isfinite(c->gamma)) return false;
+  return qspec_ok(c->worker_q, c->d) && qspec_ok(c->server_q, c->d);
+}
+
+void layout_of(const ds_qspec& q, uint64_t d, ds_payload_layout* L) {
+  memset(L, 0, sizeof *L);
+  const uint64_t nw = (d + 31) / 32;
+  uint64_t pos = 0;
+  auto put = [&](int i, uint64_t count, uint64_t elem) {
+    L->off[i] = pos;
+    L->count[i] = count;
+    pos = round16(pos + count * elem);
+  };
+  switch (q.op) {
+    case DS_Q_IDENTITY: put(0, d, 4); break;
+    case DS_Q_SIGN1: put(0, nw, 4); put(1, (d + q.chunk - 1) / q.chunk, 4); break;
+    case DS_Q_TOPK: put(0, q.k, 4); put(1, q.k, 4); break;
+    case DS_Q_QSGD: put(0, d, 1); put(1, nw, 4); put(2, (d + q.chunk - 1) / q.chunk, 4); break;
+  }
+  L->stride = pos ? pos : 16;
+}
+
+}  // namespace
+
+struct ds_ctx {
+  ds_config cfg;
+  ds_buffers buf;
+  ds_payload_layout wl, sl;
+  TopkPlan wplan, splan;  // workspace carving of the top-k path (worker rows / server row)
+  float* acc;             // dense accumulator for sparse worker payloads (inside workspace), or NULL
+  int phase;              // 0: step complete, 1: worker pass done, 2: unfused server pass done
+};
+
+namespace {
+
+// Workspace = [top-k scratch shared by both passes][dense accumulator for sparse worker payloads]
+uint64_t plan_workspace(ds_ctx* c) {
+  const ds_config& cfg = c->cfg;
+  uint64_t topk_bytes = 0;
+  if (cfg.worker_q.op == DS_Q_TOPK) {
+    topk_plan(cfg.d, cfg.n, cfg.worker_q.k, &c->wplan);
+    topk_bytes = c->wplan.bytes;
+  }
+  if (cfg.server_q.op == DS_Q_TOPK) {
+    topk_plan(cfg.d, 1, cfg.server_q.k, &c->splan);
+    if (c->splan.bytes > topk_bytes) topk_bytes = c->splan.bytes;
+  }
+  uint64_t total = round16(topk_bytes);
+  const uint64_t acc_off = total;
+  if (cfg.worker_q.op == DS_Q_TOPK) total += round16(cfg.d * 4);
+  c->acc = (cfg.worker_q.op == DS_Q_TOPK && c->buf.workspace)
+               ? reinterpret_cast<float*>(static_cast<uint8_t*>(c->buf.workspace) + acc_off)
+               : nullptr;
+  return total;
+}
+
+SrcParams worker_src(const ds_ctx* c, const float* g) {
+  SrcParams s;
+  memset(&s, 0, sizeof s);
+  s.g = g;
+  s.delta = c->buf.delta_w;
+  s.d = c->cfg.d;
+  s.n = c->cfg.n;
+  s.vec = (c->cfg.d % 4 == 0) && aligned16(g);
+  return s;
+}
+
+SrcParams server_src(const ds_ctx* c, int* kind) {
+  SrcParams s;
+  memset(&s, 0, sizeof s);
+  const ds_qspec& wq = c->cfg.worker_q;
+  s.delta = c->buf.delta_s;
+  s.d = c->cfg.d;
+  s.n = c->cfg.n;
+  s.inv_n = 1.0f / (float)c->cfg.n;
+  s.wp = static_cast<const uint8_t*>(c->buf.worker_payload);
+  s.wp_stride = c->wl.stride;
+  for (int i = 0; i < 3; ++i) s.wp_off[i] = c->wl.off[i];
+  s.w_log2_chunk = (wq.op == DS_Q_SIGN1 || wq.op == DS_Q_QSGD) ? log2u(wq.chunk) : 0;
+  s.w_levels = (float)wq.levels;
+  s.acc = c->acc;
+  s.vec = 1;
+  switch (wq.op) {
+    case DS_Q_IDENTITY: *kind = SRC_SRV_IDENTITY; break;
+    case DS_Q_SIGN1: *kind = SRC_SRV_SIGN1; break;
+    case DS_Q_TOPK: *kind = SRC_SRV_TOPK; break;
+    default: *kind = SRC_SRV_QSGD; break;
+  }
+  return s;
+}
+
+// One compression pass over `rows` vectors: rows = n with the worker source, 1 with a server source.
+int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, const ds_payload_layout& L,
+             uint8_t* payload, float* delta, uint32_t rows, bool server, float* x_fused, uint32_t step,
+             cudaStream_t st) {
+  const uint64_t d = c->cfg.d;
+  cudaError_t e = cudaSuccess;
+  switch (q.op) {
+    case DS_Q_IDENTITY:
+      e = launch_identity(src_kind, src, reinterpret_cast<float*>(payload + L.off[0]), L.stride / 4, delta, d, x_fused,
+                          c->cfg.gamma, rows, st);
+      break;
+    case DS_Q_SIGN1:
+    case DS_Q_QSGD: {
+      ChunkParams p;
+      memset(&p, 0, sizeof p);
+      if (q.op == DS_Q_SIGN1) {
+        p.out_bits = reinterpret_cast<uint32_t*>(payload + L.off[0]);
+        p.out_scale = reinterpret_cast<float*>(payload + L.off[1]);
+      } else {
+        p.out_lvl = payload + L.off[0];
+        p.out_bits = reinterpret_cast<uint32_t*>(payload + L.off[1]);
+        p.out_scale = reinterpret_cast<float*>(payload + L.off[2]);
+      }
+      p.bits_stride = L.stride / 4;
+      p.scale_stride = L.stride / 4;
+      p.lvl_stride = L.stride;
+      p.delta_out = delta;
+      p.delta_row_stride = d;
+      p.x = x_fused;
+      p.gamma = c->cfg.gamma;
+      p.levels_f = (float)q.levels;
+      p.levels_u = q.levels;
+      p.key0 = (uint32_t)(c->cfg.seed & 0xFFFFFFFFu);
+      p.key1 = (uint32_t)(c->cfg.seed >> 32);
+      p.step = step;
+      p.server_pass = server ? 1u : 0u;
+      e = launch_chunked(q.op, src_kind, src, p, rows, q.chunk, st);
+      break;
+    }
+    case DS_Q_TOPK: {
+      TopkIO io;
+      io.idx = reinterpret_cast<uint32_t*>(payload + L.off[0]);
+      io.val = reinterpret_cast<float*>(payload + L.off[1]);
+      io.payload_stride = L.stride;
+      io.v_inout = delta;  // v is written over delta, then the kept entries are zeroed: delta = v - Q[v]
+      io.x = x_fused;
+      io.gamma = c->cfg.gamma;
+      io.dev_status = c->buf.dev_status;
+      e = launch_topk(src_kind, src, server ? c->splan : c->wplan, c->buf.workspace, io, rows, q.k, st);
+      break;
+    }
+    default: return DS_ERR_UNSUPPORTED;
+  }
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "kernel launch");
+}
+
+}  // namespace
+
+extern "C" {
+
+int ds_version(void) { return 100; }
+
+const char* ds_last_error(void) { return g_last_error; }
+
+int ds_get_layout(const ds_config* cfg, int which, ds_payload_layout* out) {
+  if (!config_ok(cfg) || !out || (which != 0 && which != 1)) return DS_ERR_INVALID_ARG;
+  layout_of(which == 0 ? cfg->worker_q : cfg->server_q, cfg->d, out);
+  return DS_OK;
+}
+
+int ds_create(const ds_config* cfg, ds_buffers* bufs, ds_handle* out) {
+  if (!config_ok(cfg) || !bufs) return DS_ERR_INVALID_ARG;
+  ds_ctx tmp;
+  memset(&tmp, 0, sizeof tmp);
+  tmp.cfg = *cfg;
+  tmp.buf = *bufs;
+  layout_of(cfg->worker_q, cfg->d, &tmp.wl);
+  layout_of(cfg->server_q, cfg->d, &tmp.sl);
+  const uint64_t need_x = cfg->d * 4, need_dw = (uint64_t)cfg->n * cfg->d * 4, need_ds = cfg->d * 4;
+  const uint64_t need_wp = (uint64_t)cfg->n * tmp.wl.stride, need_sp = tmp.sl.stride;
+  const uint64_t need_ws = plan_workspace(&tmp);
+  if (bufs->x == nullptr) {  // query mode
+    bufs->x_bytes = need_x;
+    bufs->delta_w_bytes = need_dw;
+    bufs->delta_s_bytes = need_ds;
+    bufs->worker_payload_bytes = need_wp;
+    bufs->server_payload_bytes = need_sp;
+    bufs->workspace_bytes = need_ws;
+    return DS_NEED_BUFFERS;
+  }
+  if (!out) return DS_ERR_INVALID_ARG;
+  if (!bufs->delta_w || !bufs->delta_s || !bufs->worker_payload || !bufs->server_payload || !bufs->dev_status)
+    return DS_ERR_INVALID_ARG;
+  if (need_ws && !bufs->workspace) return DS_ERR_INVALID_ARG;
+  const void* ptrs[] = {bufs->x, bufs->delta_w, bufs->delta_s, bufs->worker_payload, bufs->server_payload, bufs->workspace};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return DS_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(bufs->dev_status) & 3u) != 0) return DS_ERR_ALIGN;
+  if (bufs->x_bytes < need_x || bufs->delta_w_bytes < need_dw || bufs->delta_s_bytes < need_ds ||
+      bufs->worker_payload_bytes < need_wp || bufs->server_payload_bytes < need_sp || bufs->workspace_bytes < need_ws)
+    return DS_ERR_BUFFER_TOO_SMALL;
+  ds_ctx* c = new (std::nothrow) ds_ctx(tmp);
+  if (!c) return DS_ERR_INVALID_ARG;
+  plan_workspace(c);
+  c->phase = 0;
+  *out = c;
+  return DS_OK;
+}
+
+int ds_worker_compress(ds_handle h, const float* g, uint32_t step, void* cuda_stream) {
+  if (!h || !g) return DS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(g) & 3u) != 0) return DS_ERR_ALIGN;
+  if (h->phase != 0) return DS_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const SrcParams src = worker_src(h, g);
+  const int rc = run_pass(h, SRC_WORKER, src, h->cfg.worker_q, h->wl, static_cast<uint8_t*>(h->buf.worker_payload),
+                          h->buf.delta_w, h->cfg.n, false, nullptr, step, st);
+  if (rc == DS_OK) h->phase = 1;
+  return rc;
+}
+
+int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, void* cuda_stream) {
+  if (!h || (flags & ~DS_FUSE_APPLY)) return DS_ERR_INVALID_ARG;
+  if (h->phase != 1) return DS_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int kind = 0;
+  const SrcParams src = server_src(h, &kind);
+  if (kind == SRC_SRV_TOPK) {
+    // (1/n) sum_i Q[v_i] for sparse payloads: dense accumulator, workers added in order 0..n-1
+    cudaError_t e = cudaMemsetAsync(h->acc, 0, h->cfg.d * 4, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    const uint8_t* wp = static_cast<const uint8_t*>(h->buf.worker_payload);
+    for (uint32_t i = 0; i < h->cfg.n; ++i) {
+      const uint8_t* pl = wp + (uint64_t)i * h->wl.stride;
+      e = launch_sparse_accumulate(reinterpret_cast<const uint32_t*>(pl + h->wl.off[0]),
+                                   reinterpret_cast<const float*>(pl + h->wl.off[1]), h->cfg.worker_q.k, h->acc, st);
+      if (e != cudaSuccess) return cuda_fail(e, "sparse accumulate");
+    }
+  }
+  const bool fuse = (flags & DS_FUSE_APPLY) != 0;
+  const int rc = run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload),
+                          h->buf.delta_s, 1, true, fuse ? h->buf.x : nullptr, step, st);
+  if (rc == DS_OK) h->phase = fuse ? 0 : 2;
+  return rc;
+}
+
+int ds_apply_update(ds_handle h, void* cuda_stream) {
+  if (!h) return DS_ERR_INVALID_ARG;
+  if (h->phase != 2) return DS_ERR_STATE;
+  const ds_qspec& q = h->cfg.server_q;
+  PayloadView pv;
+  memset(&pv, 0, sizeof pv);
+  pv.op = q.op;
+  pv.base = static_cast<const uint8_t*>(h->buf.server_payload);
+  for (int i = 0; i < 3; ++i) pv.off[i] = h->sl.off[i];
+  pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD) ? log2u(q.chunk) : 0;
+  pv.levels_f = (float)q.levels;
+  pv.k = q.k;
+  const cudaError_t e = launch_apply(pv, h->buf.x, h->cfg.d, h->cfg.gamma, static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return cuda_fail(e, "apply update");
+  h->phase = 0;
+  return DS_OK;
+}
+
+int ds_step_host(ds_handle h, const float* g_host, float* g_dev, uint32_t step, void* server_payload_host, float* x_host,
+                 void* cuda_stream) {
+  if (!h || !g_host || !g_dev) return DS_ERR_INVALID_ARG;
+  if (!aligned16(g_dev)) return DS_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(g_dev, g_host, (uint64_t)h->cfg.n * h->cfg.d * 4, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return cuda_fail(e, "copy of g to the device");
+  int rc = ds_worker_compress(h, g_dev, step, cuda_stream);
+  if (rc != DS_OK) return rc;
+  rc = ds_server_aggregate_compress(h, step, DS_FUSE_APPLY, cuda_stream);
+  if (rc != DS_OK) return rc;
+  if (server_payload_host) {
+    e = cudaMemcpyAsync(server_payload_host, h->buf.server_payload, h->sl.stride, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy of the server payload to the host");
+  }
+  if (x_host) {
+    e = cudaMemcpyAsync(x_host, h->buf.x, h->cfg.d * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy of x to the host");
+  }
+  return DS_OK;
+}
+
+int ds_destroy(ds_handle h) {
+  if (!h) return DS_ERR_INVALID_ARG;
+  delete h;
+  return DS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,118 @@
+// Elementwise kernels: Q = identity (Algorithm 1 then is parallel SGD, Section 1), the stand-alone
+// model update x = x - gamma Q[v] (Algorithm 1, last line of the loop), and the ordered
+// accumulation of sparse worker payloads for the server mean (first line of Eq. 4).
+#include "dsq_common.cuh"
+#include "dsq_internal.h"
+
+namespace dsq {
+
+template <int SRC>
+__global__ void __launch_bounds__(kThreads) k_identity(const SrcParams src, float* out_c, uint64_t c_row_stride,
+                                                       float* delta_out, uint64_t delta_row_stride, float* x,
+                                                       float gamma) {
+  const uint32_t row = blockIdx.y;
+  const uint64_t nq = (src.d + 3) / 4;
+  for (uint64_t qd = (uint64_t)blockIdx.x * kThreads + threadIdx.x; qd < nq; qd += (uint64_t)gridDim.x * kThreads) {
+    const uint64_t e = qd * 4;
+    const uint32_t cnt = (uint32_t)min((uint64_t)4, src.d - e);
+    const float4 v = src_load4<SRC>(src, row, e, cnt);
+    store_row4(out_c + (uint64_t)row * c_row_stride, e, cnt, 1, v);  // Q[v] = v
+    store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, make_float4(0.f, 0.f, 0.f, 0.f));
+    if (x) {
+      float4 xv = load_row4(x, e, cnt, 1);
+      xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, v.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, v.y));
+      xv.z = __fsub_rn(xv.z, __fmul_rn(gamma, v.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(gamma, v.w));
+      store_row4(x, e, cnt, 1, xv);
+    }
+  }
+}
+
+static unsigned grid_for(uint64_t items) {
+  const uint64_t blocks = (items + kThreads - 1) / kThreads;
+  const uint64_t cap = 148ull * 8ull * 4ull;  // a few waves of 8 CTAs on each of the 148 SMs
+  return (unsigned)(blocks < cap ? (blocks ? blocks : 1) : cap);
+}
+
+cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64_t c_row_stride, float* delta_out,
+                            uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st) {
+  dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
+#define DSQ_ID(S) k_identity<S><<<grid, kThreads, 0, st>>>(src, out_c, c_row_stride, delta_out, delta_row_stride, x, gamma)
+  switch (srck) {
+    case SRC_WORKER: DSQ_ID(SRC_WORKER); break;
+    case SRC_SRV_IDENTITY: DSQ_ID(SRC_SRV_IDENTITY); break;
+    case SRC_SRV_SIGN1: DSQ_ID(SRC_SRV_SIGN1); break;
+    case SRC_SRV_TOPK: DSQ_ID(SRC_SRV_TOPK); break;
+    case SRC_SRV_QSGD: DSQ_ID(SRC_SRV_QSGD); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef DSQ_ID
+  return cudaGetLastError();
+}
+
+// Dense decode of a server payload and update of x.
+__global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, float* x, uint64_t d, float gamma) {
+  const uint64_t nq = (d + 3) / 4;
+  for (uint64_t qd = (uint64_t)blockIdx.x * kThreads + threadIdx.x; qd < nq; qd += (uint64_t)gridDim.x * kThreads) {
+    const uint64_t e = qd * 4;
+    const uint32_t cnt = (uint32_t)min((uint64_t)4, d - e);
+    float4 C;
+    if (pv.op == DS_Q_IDENTITY) {
+      C = load_row4(reinterpret_cast<const float*>(pv.base + pv.off[0]), e, cnt, 1);
+    } else if (pv.op == DS_Q_SIGN1) {
+      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]) + (e >> 5)) >> (uint32_t)(e & 31);
+      const float s = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
+      C = make_float4((w & 1u) ? s : -s, (w & 2u) ? s : -s, (w & 4u) ? s : -s, (w & 8u) ? s : -s);
+    } else {  // DS_Q_QSGD
+      const uint32_t lv = __ldcs(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0] + e));
+      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[1]) + (e >> 5)) >> (uint32_t)(e & 31);
+      const float q = __fdiv_rn(__ldg(reinterpret_cast<const float*>(pv.base + pv.off[2]) + (e >> pv.log2_chunk)),
+                                pv.levels_f);
+      const float m0 = __fmul_rn((float)(lv & 255u), q), m1 = __fmul_rn((float)((lv >> 8) & 255u), q);
+      const float m2 = __fmul_rn((float)((lv >> 16) & 255u), q), m3 = __fmul_rn((float)(lv >> 24), q);
+      C = make_float4((w & 1u) ? m0 : -m0, (w & 2u) ? m1 : -m1, (w & 4u) ? m2 : -m2, (w & 8u) ? m3 : -m3);
+    }
+    float4 xv = load_row4(x, e, cnt, 1);
+    xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
+    xv.z = __fsub_rn(xv.z, __fmul_rn(gamma, C.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(gamma, C.w));
+    store_row4(x, e, cnt, 1, xv);
+  }
+}
+
+// Sparse payload: only the k listed entries of x change (the others would subtract gamma * 0).
+__global__ void __launch_bounds__(kThreads) k_apply_sparse(const uint32_t* __restrict__ idx, const float* __restrict__ val,
+                                                           uint64_t k, float* x, float gamma) {
+  for (uint64_t m = (uint64_t)blockIdx.x * kThreads + threadIdx.x; m < k; m += (uint64_t)gridDim.x * kThreads) {
+    const uint32_t j = idx[m];
+    x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val[m]));
+  }
+}
+
+cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st) {
+  if (pv.op == DS_Q_TOPK) {
+    if (pv.k == 0) return cudaSuccess;
+    k_apply_sparse<<<grid_for(pv.k), kThreads, 0, st>>>(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]),
+                                                        reinterpret_cast<const float*>(pv.base + pv.off[1]), pv.k, x, gamma);
+  } else {
+    k_apply_dense<<<grid_for((d + 3) / 4), kThreads, 0, st>>>(pv, x, d, gamma);
+  }
+  return cudaGetLastError();
+}
+
+// acc[idx[m]] = acc[idx[m]] + val[m].  Indices inside one payload are distinct, so there is no
+// conflict; the launches for workers 0..n-1 are issued in that order on one stream, which makes
+// the sum over workers sequential in worker order as Eq. 4 is evaluated.
+__global__ void __launch_bounds__(kThreads) k_sparse_accumulate(const uint32_t* __restrict__ idx,
+                                                                const float* __restrict__ val, uint64_t k, float* acc) {
+  for (uint64_t m = (uint64_t)blockIdx.x * kThreads + threadIdx.x; m < k; m += (uint64_t)gridDim.x * kThreads) {
+    const uint32_t j = idx[m];
+    acc[j] = __fadd_rn(acc[j], val[m]);
+  }
+}
+
+cudaError_t launch_sparse_accumulate(const uint32_t* idx, const float* val, uint64_t k, float* acc, cudaStream_t st) {
+  if (k == 0) return cudaSuccess;
+  k_sparse_accumulate<<<grid_for(k), kThreads, 0, st>>>(idx, val, k, acc);
+  return cudaGetLastError();
+}
+
+}  // namespace dsq

@@ -1,0 +1,84 @@
+// Host-side launch interface shared by the kernel translation units and the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dsq.h"
+#include "dsq_common.cuh"
+
+namespace dsq {
+
+// Destination of a chunk-wise operator (SIGN1 or QSGD).
+struct ChunkParams {
+  uint32_t* out_bits;        // sign words, row stride bits_stride (in words)
+  float* out_scale;          // SIGN1: scale per chunk; QSGD: norm per chunk; row stride scale_stride (floats)
+  uint8_t* out_lvl;          // QSGD: level bytes, row stride lvl_stride (bytes)
+  uint64_t bits_stride, scale_stride, lvl_stride;
+  float* delta_out;          // residual destination, row stride delta_row_stride (floats)
+  uint64_t delta_row_stride;
+  float* x;                  // non-NULL: fused model update (server pass)
+  float gamma;
+  float levels_f;            // QSGD: s
+  uint32_t levels_u;
+  uint32_t key0, key1, step; // Philox key and the step word of the counter
+  uint32_t server_pass;      // 1: counter word 2 is 0xFFFFFFFF, else the row (worker) index
+  uint32_t log2G;            // filled by the launcher
+};
+
+// Destination of a decoded payload for the dense model update.
+struct PayloadView {
+  int op;
+  const uint8_t* base;
+  uint64_t off[3];
+  uint32_t log2_chunk;
+  float levels_f;
+  uint64_t k;
+};
+
+// Per-vector state of the radix select (device memory inside the workspace).
+struct TopkState {
+  uint32_t k_rem;      // entries still to take inside the current threshold bin
+  uint32_t tb1, tb2;   // threshold digits: key bits 30..19 and 18..7
+  uint32_t tau;        // full 31-bit key of the k-th largest entry
+  uint32_t r;          // how many entries with key == tau are kept (lowest indices first)
+  uint32_t total_gt, total_tie, pad;
+};
+
+// Carving of the workspace for `rows` simultaneous selections over d-vectors.
+struct TopkPlan {
+  uint64_t d, k;
+  uint32_t rows;
+  uint64_t nseg;        // 8192-entry segments per vector
+  uint64_t bm_stride;   // bitmap words per vector (whole segments)
+  uint64_t off_hist, off_state, off_bm_gt, off_bm_eq, off_seg;
+  uint64_t bytes;
+};
+
+struct TopkIO {
+  uint32_t* idx;            // payload sub-arrays of row 0; rows are payload_stride bytes apart
+  float* val;
+  uint64_t payload_stride;
+  float* v_inout;           // [rows, d]: receives v, then has the kept entries zeroed (the residual)
+  float* x;                 // non-NULL: fused model update at the kept entries (server pass)
+  float gamma;
+  uint32_t* dev_status;
+};
+
+void topk_plan(uint64_t d, uint32_t rows, uint64_t k, TopkPlan* plan);
+cudaError_t launch_topk(int src_kind, const SrcParams& src, const TopkPlan& plan, void* workspace, const TopkIO& io,
+                        uint32_t rows, uint64_t k, cudaStream_t st);
+
+cudaError_t launch_chunked(int op, int src_kind, const SrcParams& src, const ChunkParams& p, uint32_t rows,
+                           uint32_t chunk, cudaStream_t st);
+
+// Q = identity: payload c = v, residual +0, optional fused update.
+cudaError_t launch_identity(int src_kind, const SrcParams& src, float* out_c, uint64_t c_row_stride, float* delta_out,
+                            uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);
+
+// x = x - gamma * decode(payload)
+cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);
+
+// acc[idx[m]] += val[m] for one worker's sparse payload (indices are unique within a payload)
+cudaError_t launch_sparse_accumulate(const uint32_t* idx, const float* val, uint64_t k, float* acc, cudaStream_t st);
+
+}  // namespace dsq

@@ -1,0 +1,36 @@
+"""The five workloads at full size, in the launch configuration the benchmark times: one step from
+a seeded random state (non-zero errors and model), compared with the oracle element by element."""
+import numpy as np
+import psutil
+import pytest
+import torch
+
+import oracle
+from paper_1905_05957_b200 import DoubleSqueeze, WORKLOADS, make_gradients
+from tests.helpers import compare_state, to_oracle_q
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5])
+def test_full_size_step_matches_oracle(wid):
+    wl = WORKLOADS[wid]
+    need = 4 * wl.n * wl.d * 4 + (2 << 30)
+    if psutil.virtual_memory().available < need:
+        pytest.skip(f"host memory: need {need >> 30} GiB for the oracle's copy of workload {wid}")
+    dev = "cuda"
+    ds = DoubleSqueeze.for_workload(wl, dev)
+    gen = torch.Generator(device=dev).manual_seed(1000 + wid)
+    g = make_gradients(wl, 3, device=dev)
+    scale = float(g[0, :100_000].abs().mean())
+    ds.delta_w.normal_(0.0, 0.5 * scale, generator=gen)
+    ds.delta_s.normal_(0.0, 0.25 * scale, generator=gen)
+    ds.x.normal_(0.0, 1.0, generator=gen)
+    st = oracle.State(ds.x.cpu().numpy().copy(), ds.delta_w.cpu().numpy().copy(), ds.delta_s.cpu().numpy().copy())
+    ds.step(g, 3, fuse_apply=True)
+    torch.cuda.synchronize()
+    g_host = g.cpu().numpy()
+    del g
+    oracle.step(st, g_host, to_oracle_q(wl.worker_q), to_oracle_q(wl.server_q), wl.gamma, wl.seed, 3)
+    compare_state(ds, st, g_host, tag=f"workload {wid}: ")
+    ds.close()

@@ -1,0 +1,147 @@
+"""CUDA library against the oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1905_05957_b200 import DoubleSqueeze, Q, WORKLOADS, make_gradients
+from tests.helpers import compare_state, to_oracle_q
+
+pytestmark = pytest.mark.gpu
+
+SIGN = lambda L=4096: Q("sign1", chunk=L)
+QSGD = lambda L=2048, s=255: Q("qsgd", chunk=L, levels=s)
+TOPK = lambda k: Q("topk", k=k)
+IDENT = Q("identity")
+
+
+def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None):
+    """Free-running: both sides start from the same state and see the same gradients; after every
+    step every output must agree."""
+    ds = DoubleSqueeze(n, d, gamma, wq, sq, seed, x0=x0)
+    st = oracle.State.zeros(n, d, None if x0 is None else x0.cpu().numpy())
+    if state0 is not None:
+        dw, dsv = state0
+        ds.delta_w.copy_(dw)
+        ds.delta_s.copy_(dsv)
+        st.delta_w = dw.cpu().numpy().copy()
+        st.delta_s = dsv.cpu().numpy().copy()
+    for t, g in enumerate(gs):
+        g_dev = g.cuda().contiguous()
+        ds.step(g_dev, t, fuse_apply=fuse)
+        torch.cuda.synchronize()
+        g_host = g.cpu().numpy()
+        oracle.step(st, g_host, to_oracle_q(wq), to_oracle_q(sq), gamma, seed, t)
+        compare_state(ds, st, g_host, tag=f"step {t}: ")
+    ds.close()
+    return ds, st
+
+
+def randn_steps(n, d, T, seed=0, scale=1.0):
+    gen = torch.Generator().manual_seed(seed)
+    return [torch.randn(n, d, generator=gen) * scale for _ in range(T)]
+
+
+# ------------------------------------------------------------------ operators, several tiles + ragged tail
+
+@pytest.mark.parametrize("d", [4096, 10_000, 65_536 + 4 * 37, 33, 1])
+@pytest.mark.parametrize("L", [128, 1024, 4096, 8192])
+def test_sign1_both_passes(d, L):
+    run_lockstep(3, d, SIGN(L), SIGN(L), randn_steps(3, d, 3, seed=d + L))
+
+
+@pytest.mark.parametrize("d", [2048, 10_000, 40_000 + 4, 5])
+@pytest.mark.parametrize("L,s", [(128, 255), (2048, 255), (2048, 1), (512, 15), (8192, 200)])
+def test_qsgd_both_passes(d, L, s):
+    run_lockstep(3, d, QSGD(L, s), QSGD(L, s), randn_steps(3, d, 3, seed=d + L + s, scale=1e-3))
+
+
+@pytest.mark.parametrize("d,k", [(10_000, 100), (70_000, 700), (70_000, 1), (8192, 8192), (300, 0), (33, 7), (1, 1)])
+def test_topk_both_passes(d, k):
+    run_lockstep(3, d, TOPK(k), TOPK(k), randn_steps(3, d, 3, seed=d + k))
+
+
+def test_identity_is_parallel_sgd():
+    run_lockstep(4, 10_001, IDENT, IDENT, randn_steps(4, 10_001, 3))
+
+
+@pytest.mark.parametrize("wq,sq", [
+    (SIGN(4096), TOPK(500)), (TOPK(2000), SIGN(1024)), (QSGD(2048), TOPK(300)), (TOPK(1000), QSGD(256, 7)),
+    (SIGN(256), QSGD(4096, 255)), (QSGD(1024, 3), SIGN(2048)), (IDENT, TOPK(100)), (SIGN(512), IDENT),
+    (TOPK(50), IDENT), (QSGD(128, 9), IDENT), (IDENT, SIGN(128)), (IDENT, QSGD(128, 31)),
+])
+def test_mixed_operators(wq, sq):
+    d = 50_000 + 12
+    run_lockstep(5, d, wq, sq, randn_steps(5, d, 3, seed=11))
+
+
+# ------------------------------------------------------------------ layout and alignment edge cases
+
+@pytest.mark.parametrize("d", [4097, 4098, 4099, 12_345, 31, 127])
+@pytest.mark.parametrize("wq,sq", [(SIGN(1024), SIGN(1024)), (QSGD(1024, 255), QSGD(1024, 255)), ("topk", "topk"),
+                                   (IDENT, IDENT)])
+def test_rows_not_16_byte_aligned(d, wq, sq):
+    if wq == "topk":
+        wq = sq = TOPK(max(1, d // 50))
+    run_lockstep(3, d, wq, sq, randn_steps(3, d, 2, seed=d))
+
+
+@pytest.mark.parametrize("wq,sq", [(SIGN(4096), SIGN(4096)), (QSGD(2048), QSGD(2048)), (TOPK(300), TOPK(300)),
+                                   (SIGN(4096), TOPK(150)), (IDENT, IDENT)])
+def test_unfused_apply_equals_fused(wq, sq):
+    d = 30_000
+    run_lockstep(4, d, wq, sq, randn_steps(4, d, 3, seed=5), fuse=False)
+
+
+# ------------------------------------------------------------------ degenerate data
+
+def test_topk_ties_all_equal_and_integer_valued():
+    n, d = 2, 70_000
+    gen = torch.Generator().manual_seed(3)
+    ties = [torch.randint(-3, 4, (n, d), generator=gen).float() for _ in range(2)]
+    for k in (1, 777, 35_000, d - 1):
+        run_lockstep(n, d, TOPK(k), TOPK(k), ties)
+    same = [torch.full((n, d), -2.5), torch.full((n, d), 2.5)]
+    run_lockstep(n, d, TOPK(1234), TOPK(4321), same)
+    zeros = [torch.zeros(n, d), torch.zeros(n, d)]
+    run_lockstep(n, d, TOPK(10), TOPK(10), zeros)
+
+
+def test_zero_signed_zero_subnormal_and_zero_chunks():
+    n, d = 2, 3 * 4096
+    g = torch.randn(n, d) * 1e-3
+    g[:, :4096] = 0.0            # an all-zero chunk
+    g[:, 4096:4096 + 64] = -0.0
+    g[:, 5000:5100] = 1e-41      # subnormals
+    g[:, 5100:5200] = -1e-41
+    g[0, 8192:] = 1e-30          # squares underflow: a quantisation chunk of norm ~0
+    for wq in (SIGN(4096), QSGD(2048), TOPK(100), SIGN(128), QSGD(128, 5)):
+        run_lockstep(n, d, wq, wq, [g, g.clone(), -g])
+
+
+def test_qsgd_stream_depends_on_seed_and_step():
+    n, d = 2, 8192
+    g = randn_steps(n, d, 1, seed=2)[0]
+    a = DoubleSqueeze(n, d, 0.1, QSGD(), QSGD(), seed=1)
+    b = DoubleSqueeze(n, d, 0.1, QSGD(), QSGD(), seed=(1 << 40) + 1)
+    a.worker_compress(g.cuda(), 0)
+    b.worker_compress(g.cuda(), 0)
+    la, lb = a.worker_views()[0]["lvl"].cpu(), b.worker_views()[0]["lvl"].cpu()
+    assert not torch.equal(la, lb)          # high word of the seed reaches the key
+    assert not torch.equal(la, a.worker_views()[1]["lvl"].cpu())
+
+
+def test_many_workers_and_one_worker():
+    run_lockstep(1, 9000, SIGN(4096), SIGN(4096), randn_steps(1, 9000, 2))
+    run_lockstep(33, 5000, QSGD(2048), SIGN(4096), randn_steps(33, 5000, 2))
+    run_lockstep(7, 20_000, TOPK(200), TOPK(200), randn_steps(7, 20_000, 2))
+
+
+# ------------------------------------------------------------------ the five workloads, scaled down
+
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5])
+def test_workload_recipes_scaled(wid):
+    wl = WORKLOADS[wid]
+    wl = wl if wid == 1 else wl.scaled(d=200_000 + 40, n=min(wl.n, 8), steps=4)
+    gs = [make_gradients(wl, t, device="cpu") for t in range(min(wl.steps, 4))]
+    run_lockstep(wl.n, wl.d, wl.worker_q, wl.server_q, gs, gamma=wl.gamma, seed=wl.seed)
