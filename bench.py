@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the DoubleSqueeze step (worker pass + server pass with fused model update).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl ours|reference]
+
+One "step" is one whole iteration of Algorithm 1 over one batch of synthetic gradients
+(ds_worker_compress + ds_server_aggregate_compress with the fused update).  Prints ONE JSON line.
+For N > 1 (launched by torch.distributed.run) every rank steps an independent replica of the same
+workload on its own GPU -- the path has no exchange between GPUs -- and the value is the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "doublesqueeze_step_gradient_elements_per_s"
+UNIT = "elements/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/; valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {
+    # workload id: (kernel, bytes per launch, digest of csrc/ at capture time)
+}
+
+
+def payload_bytes(q, d: int) -> int:
+    nw = (d + 31) // 32
+    if q.op == "sign1":
+        return 4 * nw + 4 * ((d + q.chunk - 1) // q.chunk)
+    if q.op == "qsgd":
+        return d + 4 * nw + 4 * ((d + q.chunk - 1) // q.chunk)
+    if q.op == "topk":
+        return 8 * q.k
+    return 4 * d
+
+
+def algorithmic_bytes(wl) -> dict:
+    """Bytes the method must move per step: read g and delta_w, write delta_w and the worker
+    payloads; the server reads the payloads, reads and writes delta_s, writes its payload, and
+    reads and writes x (only the k kept entries for top-k)."""
+    n, d = wl.n, wl.d
+    pw, ps = payload_bytes(wl.worker_q, d), payload_bytes(wl.server_q, d)
+    worker = n * d * 12 + n * pw
+    x_bytes = 8 * wl.server_q.k if wl.server_q.op == "topk" else 8 * d
+    server = n * pw + 8 * d + ps + x_bytes
+    return {"worker": worker, "server": server, "total": worker + server}
+
+
+def csrc_digest() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1905_05957_b200", "csrc")
+    for f in sorted(os.listdir(csrc)):
+        if f.endswith((".cu", ".cuh", ".h")):
+            h.update(open(os.path.join(csrc, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak() -> tuple[float, str]:
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm and CPU baseline: the oracle, as it stands, on the host cores
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample_workload(wl):
+    """A bounded sample of the workload for the CPU oracle: same recipe, n workers, d cut so that
+    one step is a few seconds of single-thread work (the oracle runs ~30-80 M entries/s; top-k
+    sorts every vector)."""
+    budget = 120_000_000 if wl.worker_q.op != "topk" else 24_000_000
+    if wl.n * wl.d <= budget:
+        return wl, "full workload"
+    d = max(8192, (budget // wl.n) // 8192 * 8192)
+    return wl.scaled(d=d), f"same recipe with d cut to {d} (n={wl.n})"
+
+
+def time_oracle(wl, steps: int, warmup: int) -> dict:
+    import numpy as np
+
+    import oracle
+    from paper_1905_05957_b200.workloads import make_gradients
+    from tests.helpers import to_oracle_q
+
+    swl, what = oracle_sample_workload(wl)
+    st = oracle.State.zeros(swl.n, swl.d)
+    wq, sq = to_oracle_q(swl.worker_q), to_oracle_q(swl.server_q)
+    gs = [make_gradients(swl, t, device="cpu").numpy() for t in range(2)]
+    for t in range(warmup):
+        oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, t)
+    t0 = time.perf_counter()
+    for t in range(steps):
+        oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, warmup + t)
+    dt = time.perf_counter() - t0
+    assert np.isfinite(st.x).all()
+    return {"value": swl.n * swl.d * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{steps} step(s) of {what}; single thread", "ms_per_step": 1e3 * dt / steps}
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
+    r = time_oracle(wl, steps, warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(wl),
+        "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl) -> dict:
+    def q(s):
+        return {"op": s.op, **({"chunk": s.chunk} if s.chunk else {}), **({"k": s.k} if s.op == "topk" else {}),
+                **({"levels": s.levels} if s.levels else {})}
+    return {"workload": wl.name, "n_workers": wl.n, "d": wl.d, "gradient_dist": wl.dist, "worker_q": q(wl.worker_q),
+            "server_q": q(wl.server_q), "gamma": wl.gamma,
+            "l2": "inputs larger than L2: g and delta_w are streamed once per step and exceed 126 MB"
+                  if wl.n * wl.d * 8 > 2 * 126e6 else "L2 flushed between steps by writing a 256 MB buffer"}
+
+
+# ---------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1905_05957_b200 import DoubleSqueeze, load_library
+    from paper_1905_05957_b200.workloads import make_gradients
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    lib = load_library()          # raises if the CUDA library is missing: there is no other path
+    K, W = args.steps, max(args.warmup, 3)
+
+    ds = DoubleSqueeze.for_workload(wl, dev)
+    ring = [make_gradients(wl, t, device=dev) for t in range(2)]     # distinct g_t, resident in HBM
+    need_flush = wl.n * wl.d * 8 <= 2 * 126e6
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing
+    for t in range(W):
+        ds.step(ring[t % 2], t)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = lib.ds_kernel_launches()
+    t_total = 0.0
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if not need_flush:
+        start.record(stream)
+    for t in range(K):
+        if need_flush:
+            flush.fill_(t & 0xFF)
+        ev[t][0].record(stream)
+        ds.worker_compress(ring[t % 2], W + t)
+        ev[t][1].record(stream)
+        ds.server_aggregate_compress(W + t, fuse_apply=True)
+        ev[t][2].record(stream)
+    if not need_flush:
+        stop.record(stream)
+    barrier()
+    launches = lib.ds_kernel_launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    worker_ms = [ev[t][0].elapsed_time(ev[t][1]) for t in range(K)]
+    server_ms = [ev[t][1].elapsed_time(ev[t][2]) for t in range(K)]
+    step_ms = [ev[t][0].elapsed_time(ev[t][2]) for t in range(K)]
+    t_total = sum(step_ms) if need_flush else start.elapsed_time(stop)   # flush writes are not part of the step
+    status = ds.device_status()
+
+    # ---- end to end: pinned host g -> device, fused step, server payload -> host, every step
+    g_host = [torch.empty(wl.n, wl.d, dtype=torch.float32, pin_memory=True) for _ in range(2)]
+    for a, b in zip(g_host, ring):
+        a.copy_(b)
+    out_host = torch.empty(ds.server_payload.numel(), dtype=torch.uint8, pin_memory=True)
+    Ke = max(1, min(K, 10))
+    for t in range(2):
+        ds.step_host(g_host[t % 2], ring[0], 10_000 + t, server_payload_host=out_host)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(Ke):
+        ds.step_host(g_host[t % 2], ring[0], 20_000 + t, server_payload_host=out_host)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([t_total, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    t_total, e2e_ms = float(times[0]), float(times[1])
+
+    if rank == 0:
+        ab = algorithmic_bytes(wl)
+        peak, peak_kind = measured_peak()
+        wk_ms = statistics.mean(worker_ms)
+        achieved = ab["worker"] / (wk_ms * 1e-3) / 1e9
+        digest = csrc_digest()
+        traffic = None
+        if wl.wid in NCU_TRAFFIC and NCU_TRAFFIC[wl.wid][2] == digest:
+            traffic = NCU_TRAFFIC[wl.wid][1]
+        dominant = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
+                    "topk": "top-k worker pass (pass1, mark, refine, finalize, emit)",
+                    "identity": "k_identity<WORKER>"}[wl.worker_q.op]
+        elems = world * wl.n * wl.d
+        line = {
+            "metric": METRIC, "value": elems * K / (t_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": t_total / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl),
+            "clocks": clocks,
+            "e2e": {"value": elems * Ke / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": wl.n * wl.d * 4,
+                    "d2h_bytes_per_step": int(ds.server_payload.numel()), "steps": Ke},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": traffic,
+                         "algorithmic_bytes_per_launch": ab["worker"], "ms_per_launch": wk_ms},
+            "step_breakdown": {
+                "worker_ms": wk_ms, "server_ms": statistics.mean(server_ms),
+                "step_ms_median": statistics.median(step_ms), "step_ms_p10": sorted(step_ms)[int(0.1 * (K - 1))],
+                "step_ms_p90": sorted(step_ms)[int(0.9 * (K - 1))],
+                "algorithmic_gb_per_step": ab["total"] / 1e9,
+                "step_gbs": ab["total"] / (statistics.median(step_ms) * 1e-3) / 1e9,
+                "step_frac_of_peak": ab["total"] / (statistics.median(step_ms) * 1e-3) / 1e9 / peak,
+                "step_frac_of_nominal_8000": ab["total"] / (statistics.median(step_ms) * 1e-3) / 1e9 / 8000.0,
+                "server_gbs": ab["server"] / (statistics.mean(server_ms) * 1e-3) / 1e9,
+            },
+            "device_status": status,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = {k: v for k, v in time_oracle(wl, args.cpu_steps, 0).items() if k != "ms_per_step"}
+        print(json.dumps(line), flush=True)
+    ds.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", type=int, default=2, help="1..5; 2 = ResNet-18-sized 1-bit (the default)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-steps", type=int, default=3)
+    args = ap.parse_args()
+    from paper_1905_05957_b200.workloads import WORKLOADS
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

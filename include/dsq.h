@@ -194,6 +194,9 @@ int ds_step_host(ds_handle h, const float* g_host, float* g_dev, uint32_t step, 
 /* Text of the most recent CUDA error seen by this thread's calls ("" if none). */
 const char* ds_last_error(void);
 
+/* Number of kernels this library has launched since it was loaded (all handles, all streams). */
+uint64_t ds_kernel_launches(void);
+
 /* Library version, major*100 + minor. */
 int ds_version(void);
 

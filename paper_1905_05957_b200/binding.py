@@ -22,7 +22,8 @@ DS_FUSE_APPLY = 1
 DS_DEV_TOPK_INCONSISTENT = 1
 OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3}
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
-           "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version")
+           "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
+           "ds_kernel_launches")
 
 
 class ds_qspec(C.Structure):
@@ -74,10 +75,10 @@ def load_library() -> C.CDLL:
     L.ds_apply_update.argtypes = [vp, vp]
     L.ds_destroy.argtypes = [vp]
     L.ds_step_host.argtypes = [vp, vp, vp, u32, vp, vp, vp]
-    L.ds_last_error.restype = C.c_char_p
     for name in EXPORTS:
-        if getattr(L, name).restype is not C.c_char_p:
-            getattr(L, name).restype = C.c_int
+        getattr(L, name).restype = C.c_int
+    L.ds_last_error.restype = C.c_char_p
+    L.ds_kernel_launches.restype = C.c_uint64
     _lib = L
     return L
 

@@ -9,6 +9,10 @@
 
 using namespace dsq;
 
+namespace dsq {
+uint64_t g_kernel_launches = 0;
+}
+
 namespace {
 
 thread_local char g_last_error[256] = "";
@@ -190,6 +194,8 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
 extern "C" {
 
 int ds_version(void) { return 100; }
+
+uint64_t ds_kernel_launches(void) { return g_kernel_launches; }
 
 const char* ds_last_error(void) { return g_last_error; }
 

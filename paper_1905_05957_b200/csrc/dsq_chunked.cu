@@ -177,6 +177,7 @@ static cudaError_t launch_v(const SrcParams& src, ChunkParams p, uint32_t rows, 
     case 8: k_chunked<OP, SRC, 8><<<grid, kThreads, 0, st>>>(src, p); break;
     default: return cudaErrorInvalidValue;
   }
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -46,6 +46,7 @@ cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64
     default: return cudaErrorInvalidValue;
   }
 #undef DSQ_ID
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -95,6 +96,7 @@ cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamm
   } else {
     k_apply_dense<<<grid_for((d + 3) / 4), kThreads, 0, st>>>(pv, x, d, gamma);
   }
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -112,6 +114,7 @@ __global__ void __launch_bounds__(kThreads) k_sparse_accumulate(const uint32_t* 
 cudaError_t launch_sparse_accumulate(const uint32_t* idx, const float* val, uint64_t k, float* acc, cudaStream_t st) {
   if (k == 0) return cudaSuccess;
   k_sparse_accumulate<<<grid_for(k), kThreads, 0, st>>>(idx, val, k, acc);
+  count_launches(1);
   return cudaGetLastError();
 }
 

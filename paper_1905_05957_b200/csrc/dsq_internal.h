@@ -8,6 +8,10 @@
 
 namespace dsq {
 
+// Kernels launched by this library since it was loaded (reported by ds_kernel_launches()).
+extern uint64_t g_kernel_launches;
+inline void count_launches(uint64_t n) { g_kernel_launches += n; }
+
 // Destination of a chunk-wise operator (SIGN1 or QSGD).
 struct ChunkParams {
   uint32_t* out_bits;        // sign words, row stride bits_stride (in words)

@@ -399,6 +399,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     default: return cudaErrorInvalidValue;
   }
 #undef DSQ_P1
+  count_launches(1);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   if (k == 0) return cudaSuccess;  // nothing kept: Q[v] = 0, delta = v, x unchanged
 
@@ -416,6 +417,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
                                        reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0,
                                        (uint64_t)(reinterpret_cast<uint8_t*>(io.val) - reinterpret_cast<uint8_t*>(io.idx)),
                                        k32, io.x, io.gamma);
+  count_launches(10);
   return cudaGetLastError();
 }
 

@@ -21,7 +21,7 @@ def lib():
 
 def test_exports_every_declared_symbol(lib):
     header = open(os.path.join(ROOT, "include", "dsq.h")).read()
-    declared = set(re.findall(r"^\s*(?:int|const char\*)\s+(ds_\w+)\s*\(", header, flags=re.M))
+    declared = set(re.findall(r"^\s*(?:int|const char\*|uint64_t)\s+(ds_\w+)\s*\(", header, flags=re.M))
     assert declared == set(b.EXPORTS)
     for name in declared:
         assert getattr(lib, name) is not None
