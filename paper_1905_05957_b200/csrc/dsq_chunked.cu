@@ -6,42 +6,117 @@
 // server pass, the model update.  v, Q[v] and delta never make a second trip through HBM.
 //
 // Geometry.  A chunk of L = 4*V*G entries is owned by G threads (G = 32..256, a power of two)
-// that hold V float4 each; float4 number j of thread t covers entries (j*G + t)*4 .. +3 of the
-// chunk, so a warp always touches 512 contiguous bytes.  A 256-thread CTA owns 256/G chunks.
+// that hold V float4 each; float4 number j ("row" j) of thread t covers entries (j*G + t)*4 .. +3
+// of the chunk, so a warp always touches 512 contiguous bytes.  A 256-thread CTA owns 256/G chunks.
 //
 // Reduction order.  The chunk sum is the pairwise sum in index order over the zero-padded chunk:
 // two levels inside a float4, five xor-butterfly levels inside a warp (one 128-entry group), then
 // a butterfly over the L/128 group sums through shared memory.  Float addition commutes bitwise,
-// so every lane of a butterfly ends with the same value, independent of the launch shape.
+// so the value does not depend on which lane performs an addition.  The V butterflies of a warp
+// are folded into one: at level s a lane keeps the rows whose bit s equals its own lane bit s and
+// hands the others to its partner, so that V rows cost log2(V) halving steps plus 5 - log2(V)
+// ordinary ones instead of 5 V shuffles, with the same additions in the same tree.
 #include "dsq_common.cuh"
 #include "dsq_internal.h"
 
 namespace dsq {
 
-template <int OP, int SRC, int V>
-__global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const ChunkParams p) {
-  __shared__ float s_red[64];
+namespace {
+
+// Sum over the warp of row (lane % V) of a[.]; the butterfly order is lane bit 0, 1, ..., 4.
+template <int V>
+__device__ __forceinline__ float warp_rows_sum(float (&a)[V], uint32_t lane) {
+  int s = 0;
+#pragma unroll
+  for (int n = V; n > 1; n >>= 1, ++s) {
+    const bool up = (lane >> s) & 1u;
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) {
+      const float keep = up ? a[2 * i + 1] : a[2 * i];
+      const float send = up ? a[2 * i] : a[2 * i + 1];
+      a[i] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, 1 << s));
+    }
+  }
+  float x = a[0];
+#pragma unroll
+  for (int o = V; o < 32; o <<= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+
+// Each lane holds one 4-bit field per row (signs of its float4).  Returns the 32-entry sign word
+// of row (lane % V) for the eight lanes lane&~7 .. lane|7 (valid in every lane of the octet whose
+// lane % V names that row).  Same halving idea: log2(V) exchange steps, then OR-combining steps.
+template <int V>
+__device__ __forceinline__ uint32_t octet_sign_words(const uint32_t (&nib)[V], uint32_t lane) {
+  uint32_t f[V];
+#pragma unroll
+  for (int r = 0; r < V; ++r) f[r] = nib[r];
+  int s = 0;
+  int w = 4;  // field width in bits
+#pragma unroll
+  for (int n = V; n > 1; n >>= 1, ++s, w <<= 1) {
+    const bool up = (lane >> s) & 1u;
+    uint32_t send = 0;
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) send |= (up ? f[2 * i] : f[2 * i + 1]) << (i * w);
+    const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1 << s);
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) {
+      const uint32_t keep = up ? f[2 * i + 1] : f[2 * i];
+      const uint32_t got = (recv >> (i * w)) & ((1u << w) - 1u);  // w <= 16 inside this loop
+      f[i] = up ? (got | (keep << w)) : (keep | (got << w));      // the lower lane's entries come first
+    }
+  }
+  uint32_t x = f[0];
+#pragma unroll
+  for (int o = V; o < 8; o <<= 1, w <<= 1) {
+    const bool up = (lane & o) != 0;
+    const uint32_t got = __shfl_xor_sync(0xffffffffu, x, o);
+    x = up ? (got | (x << w)) : (x | (got << w));
+  }
+  return x;
+}
+
+template <int OP, int SRC, int V, int LOG2G, bool FULL>
+__device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkParams& p, float* s_red) {
+  constexpr uint32_t G = 1u << LOG2G;
+  constexpr uint32_t L = (uint32_t)V * G * 4u;
+  constexpr uint32_t NG = (V * G) >> 5;   // 128-entry groups per chunk
+  constexpr uint32_t CPC = kThreads / G;  // chunks per CTA
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
-  const uint32_t G = 1u << p.log2G;
-  const uint32_t sub = tid >> p.log2G, t = tid & (G - 1u);
+  const uint32_t sub = tid >> LOG2G, t = tid & (G - 1u);
   const uint32_t row = blockIdx.y;
-  const uint64_t c = (uint64_t)blockIdx.x * (kThreads >> p.log2G) + sub;  // chunk index in the row
-  const uint32_t L = (uint32_t)V * G * 4u;
+  const uint64_t c = (uint64_t)blockIdx.x * CPC + sub;  // chunk index in the row
   const uint64_t d = src.d;
   const uint64_t base = c * L;
-  const bool chunk_live = base < d;
+  const bool chunk_live = FULL || base < d;
 
   float4 v[V];
   uint32_t cnt[V];
+  if constexpr (FULL && SRC == SRC_WORKER) {
+    const float4* gp = reinterpret_cast<const float4*>(src.g + (uint64_t)row * d + base) + t;
+    const float4* dp = reinterpret_cast<const float4*>(src.delta + (uint64_t)row * d + base) + t;
+    float4 a[V], b[V];
 #pragma unroll
-  for (int j = 0; j < V; ++j) {
-    const uint64_t e = base + (uint64_t)(j * G + t) * 4u;
-    cnt[j] = e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u;
-    v[j] = cnt[j] ? src_load4<SRC>(src, row, e, cnt[j]) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < V; ++j) a[j] = __ldcs(gp + j * G);
+#pragma unroll
+    for (int j = 0; j < V; ++j) b[j] = __ldcs(dp + j * G);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      cnt[j] = 4;
+      v[j] = make_float4(__fadd_rn(a[j].x, b[j].x), __fadd_rn(a[j].y, b[j].y), __fadd_rn(a[j].z, b[j].z),
+                         __fadd_rn(a[j].w, b[j].w));
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const uint64_t e = base + (uint64_t)(j * G + t) * 4u;
+      cnt[j] = FULL ? 4u : (e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u);
+      v[j] = cnt[j] ? src_load4<SRC>(src, row, e, cnt[j]) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   }
 
   // ---- chunk reduction: sum |v| (SIGN1) or sum v*v (QSGD), pairwise in index order
-  const uint32_t NG = (V * G) >> 5;  // 128-entry groups per chunk
   float part[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) {
@@ -52,23 +127,17 @@ __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const
       m0 = __fmul_rn(v[j].x, v[j].x); m1 = __fmul_rn(v[j].y, v[j].y);
       m2 = __fmul_rn(v[j].z, v[j].z); m3 = __fmul_rn(v[j].w, v[j].w);
     }
-    float s = __fadd_rn(__fadd_rn(m0, m1), __fadd_rn(m2, m3));
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
-    part[j] = s;
+    part[j] = __fadd_rn(__fadd_rn(m0, m1), __fadd_rn(m2, m3));
   }
-  float total;
-  if (NG == 1) {
-    total = part[0];
-  } else {
-    if (lane == 0) {
-#pragma unroll
-      for (int j = 0; j < V; ++j) s_red[sub * NG + j * (G >> 5) + (t >> 5)] = part[j];
-    }
+  float total = warp_rows_sum<V>(part, lane);  // lane holds the 128-entry group sum of row lane % V
+  if constexpr (NG > 1) {
+    // group index inside the chunk: row j = lane, warp (t >> 5) of the row
+    if (lane < (uint32_t)V) s_red[sub * NG + lane * (G >> 5) + (t >> 5)] = total;
     __syncthreads();
     float x;
-    if (NG <= 32) {
+    if constexpr (NG <= 32) {
       x = lane < NG ? s_red[sub * NG + lane] : 0.f;
+#pragma unroll
       for (uint32_t o = 1; o < NG; o <<= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
     } else {  // NG == 64
       x = __fadd_rn(s_red[sub * 64 + 2 * lane], s_red[sub * 64 + 2 * lane + 1]);
@@ -79,7 +148,7 @@ __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const
   }
 
   // ---- per-chunk quantities
-  const uint32_t len = chunk_live ? (uint32_t)min((uint64_t)L, d - base) : 1u;
+  const uint32_t len = FULL ? L : (chunk_live ? (uint32_t)min((uint64_t)L, d - base) : 1u);
   float s_or_q, inv_q = 0.f;
   if constexpr (OP == DS_Q_SIGN1) {
     s_or_q = __fdiv_rn(total, (float)len);  // mean |v| over the true chunk length
@@ -99,18 +168,19 @@ __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const
   }
 
   // ---- encode, residual, optional model update
-  float* delta_row = p.delta_out + (uint64_t)row * p.delta_row_stride;
+  float* delta_chunk = p.delta_out + (uint64_t)row * p.delta_row_stride + base;
+  uint32_t nib[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) {
     const uint32_t tq = (uint32_t)(j * G + t);  // float4 index inside the chunk
     const uint64_t e = base + (uint64_t)tq * 4u;
     float4 C;
-    uint32_t nib = 0;
+    nib[j] = 0;
     if constexpr (OP == DS_Q_SIGN1) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const bool nonneg = compc(v[j], k) >= 0.f;
-        nib |= (nonneg ? 1u : 0u) << k;
+        nib[j] |= (nonneg ? 1u : 0u) << k;
         comp(C, k) = nonneg ? s_or_q : -s_or_q;
       }
     } else {
@@ -130,25 +200,23 @@ __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const
         level = min(level, p.levels_u);
         const float mag = __fmul_rn((float)level, s_or_q);
         const bool nonneg = val >= 0.f;
-        nib |= (nonneg ? 1u : 0u) << k;
+        nib[j] |= (nonneg ? 1u : 0u) << k;
         comp(C, k) = nonneg ? mag : -mag;
         packed |= level << (8 * k);
       }
       if (cnt[j]) *reinterpret_cast<uint32_t*>(p.out_lvl + (uint64_t)row * p.lvl_stride + e) = packed;
     }
-    // sign words: eight neighbouring lanes hold one 32-entry word
-    nib &= (1u << cnt[j]) - 1u;
-    uint32_t word = nib << ((lane & 7u) * 4u);
-    word |= __shfl_xor_sync(0xffffffffu, word, 1);
-    word |= __shfl_xor_sync(0xffffffffu, word, 2);
-    word |= __shfl_xor_sync(0xffffffffu, word, 4);
-    if ((lane & 7u) == 0 && cnt[j]) p.out_bits[(uint64_t)row * p.bits_stride + (e >> 5)] = word;
+    if constexpr (!FULL) nib[j] &= (1u << cnt[j]) - 1u;  // pad bits are 0
 
     if (cnt[j]) {
       float4 dl;
       dl.x = __fsub_rn(v[j].x, C.x); dl.y = __fsub_rn(v[j].y, C.y);
       dl.z = __fsub_rn(v[j].z, C.z); dl.w = __fsub_rn(v[j].w, C.w);
-      store_row4(delta_row, e, cnt[j], src.vec, dl);
+      if constexpr (FULL) {
+        st_stream4(delta_chunk + tq * 4u, dl);
+      } else {
+        store_row4(delta_chunk, (uint64_t)tq * 4u, cnt[j], src.vec, dl);
+      }
       if (p.x) {  // fused model update (server pass only): x = x - gamma * Q[v]
         float4 xv = load_row4(p.x, e, cnt[j], 1);
         xv.x = __fsub_rn(xv.x, __fmul_rn(p.gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(p.gamma, C.y));
@@ -157,24 +225,41 @@ __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const
       }
     }
   }
+  // sign words: eight neighbouring lanes hold one 32-entry word per row; lane (octet base + r)
+  // stores the word of row r
+  const uint32_t word = octet_sign_words<V>(nib, lane);
+  const uint32_t r = lane & 7u;
+  if (r < (uint32_t)V) {
+    const uint64_t e0 = base + (uint64_t)(r * G + (t & ~7u)) * 4u;  // first entry of that word
+    if (FULL || e0 < d) p.out_bits[(uint64_t)row * p.bits_stride + (e0 >> 5)] = word;
+  }
+}
+
+template <int OP, int SRC, int V, int LOG2G>
+__global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const ChunkParams p) {
+  __shared__ float s_red[64];
+  constexpr uint64_t span = (uint64_t)V * 4u * kThreads;  // entries per CTA
+  // interior CTA of an aligned row: no bounds logic anywhere
+  if (src.vec && ((uint64_t)blockIdx.x + 1) * span <= src.d) {
+    chunk_body<OP, SRC, V, LOG2G, true>(src, p, s_red);
+  } else {
+    chunk_body<OP, SRC, V, LOG2G, false>(src, p, s_red);
+  }
 }
 
 template <int OP, int SRC>
-static cudaError_t launch_v(const SrcParams& src, ChunkParams p, uint32_t rows, uint32_t chunk, cudaStream_t st) {
+cudaError_t launch_v(const SrcParams& src, const ChunkParams& p, uint32_t rows, uint32_t chunk, cudaStream_t st) {
   // chunk = 4*V*G with G <= 256: V = 1 for chunk <= 1024, else chunk/1024
-  const uint32_t V = chunk <= 1024 ? 1u : chunk / 1024u;
-  const uint32_t G = chunk / (4u * V);
-  uint32_t log2G = 0;
-  while ((1u << log2G) < G) ++log2G;
-  p.log2G = log2G;
-  const uint64_t nc = (src.d + chunk - 1) / chunk;
-  const uint32_t cpc = kThreads / G;
-  dim3 grid((unsigned)((nc + cpc - 1) / cpc), rows, 1);
-  switch (V) {
-    case 1: k_chunked<OP, SRC, 1><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 2: k_chunked<OP, SRC, 2><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 4: k_chunked<OP, SRC, 4><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 8: k_chunked<OP, SRC, 8><<<grid, kThreads, 0, st>>>(src, p); break;
+  const uint64_t span_entries = chunk <= 1024 ? 1024 : chunk;  // entries per CTA
+  dim3 grid((unsigned)((src.d + span_entries - 1) / span_entries), rows, 1);
+  switch (chunk) {
+    case 128: k_chunked<OP, SRC, 1, 5><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 256: k_chunked<OP, SRC, 1, 6><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 512: k_chunked<OP, SRC, 1, 7><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 1024: k_chunked<OP, SRC, 1, 8><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 2048: k_chunked<OP, SRC, 2, 8><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 4096: k_chunked<OP, SRC, 4, 8><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 8192: k_chunked<OP, SRC, 8, 8><<<grid, kThreads, 0, st>>>(src, p); break;
     default: return cudaErrorInvalidValue;
   }
   count_launches(1);
@@ -182,8 +267,8 @@ static cudaError_t launch_v(const SrcParams& src, ChunkParams p, uint32_t rows, 
 }
 
 template <int OP>
-static cudaError_t launch_src(int srck, const SrcParams& src, const ChunkParams& p, uint32_t rows, uint32_t chunk,
-                              cudaStream_t st) {
+cudaError_t launch_src(int srck, const SrcParams& src, const ChunkParams& p, uint32_t rows, uint32_t chunk,
+                       cudaStream_t st) {
   switch (srck) {
     case SRC_WORKER: return launch_v<OP, SRC_WORKER>(src, p, rows, chunk, st);
     case SRC_SRV_IDENTITY: return launch_v<OP, SRC_SRV_IDENTITY>(src, p, rows, chunk, st);
@@ -193,6 +278,8 @@ static cudaError_t launch_src(int srck, const SrcParams& src, const ChunkParams&
   }
   return cudaErrorInvalidValue;
 }
+
+}  // namespace
 
 cudaError_t launch_chunked(int op, int srck, const SrcParams& src, const ChunkParams& p, uint32_t rows, uint32_t chunk,
                            cudaStream_t st) {
