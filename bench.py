@@ -330,9 +330,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this d (profiling captures)")
     args = ap.parse_args()
     from paper_1905_05957_b200.workloads import WORKLOADS
     wl = WORKLOADS[args.workload]
+    if args.scale_d:
+        wl = wl.scaled(d=args.scale_d)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -138,7 +138,8 @@ typedef struct {
  *             [1] float  scale[ceil(d/chunk)]
  *   TOPK      [0] uint32 idx[k] ascending  [1] float val[k] (bit copies of v[idx])
  *   QSGD      [0] uint8  lvl[d]            [1] uint32 sgn[ceil(d/32)] (bit = v >= 0)
- *             [2] float  norm[ceil(d/chunk)] (0 for a chunk sent as all zeros)
+ *             [2] float  step[ceil(d/chunk)] (the grid step q = N_c / levels that multiplies the
+ *                 levels; 0 for a chunk sent as all zeros)
  */
 typedef struct {
   uint64_t stride;

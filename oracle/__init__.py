@@ -43,8 +43,8 @@ def lib():
         L.orc_decode_sign1.argtypes = [u32p, f32p, u64, u32, f32p]
         L.orc_q_topk.argtypes = [f32p, u64, u64, u32p, f32p, f32p]
         L.orc_decode_topk.argtypes = [u32p, f32p, u64, u64, f32p]
-        L.orc_q_qsgd.argtypes = [f32p, u64, u32, u32, u64, u32, u32, u8p, u32p, f32p, f32p]
-        L.orc_decode_qsgd.argtypes = [u8p, u32p, f32p, u64, u32, u32, f32p]
+        L.orc_q_qsgd.argtypes = [f32p, u64, u32, u32, u64, u32, u32, u8p, u32p, f32p, f32p, f32p]
+        L.orc_decode_qsgd.argtypes = [u8p, u32p, f32p, u64, u32, f32p]
         _lib = L
     return _lib
 
@@ -174,18 +174,20 @@ def q_qsgd(v, L, s, seed, step, wid):
     lvl = np.zeros(d, dtype=np.uint8)
     sgn = np.zeros((d + 31) // 32, dtype=np.uint32)
     norm = np.zeros((d + L - 1) // L, dtype=np.float32)
+    qstep = np.zeros_like(norm)
     Cv = np.empty_like(v)
     _check(lib().orc_q_qsgd(_p(v, C.c_float), d, L, s, C.c_uint64(seed), step, wid, _p(lvl, C.c_uint8),
-                            _p(sgn, C.c_uint32), _p(norm, C.c_float), _p(Cv, C.c_float)), "qsgd")
-    return Cv, {"lvl": lvl, "sgn": sgn, "norm": norm}
+                            _p(sgn, C.c_uint32), _p(norm, C.c_float), _p(qstep, C.c_float), _p(Cv, C.c_float)), "qsgd")
+    # the payload is (lvl, sgn, step); the chunk norm N is returned as well for the tests that pin it
+    return Cv, {"lvl": lvl, "sgn": sgn, "step": qstep, "norm": norm}
 
 
-def decode_qsgd(lvl, sgn, norm, d, L, s):
+def decode_qsgd(lvl, sgn, qstep, d, L):
     lvl = np.ascontiguousarray(lvl, dtype=np.uint8)
     sgn = np.ascontiguousarray(sgn, dtype=np.uint32)
-    norm = _f32(norm)
+    qstep = _f32(qstep)
     Cv = np.empty(d, dtype=np.float32)
-    _check(lib().orc_decode_qsgd(_p(lvl, C.c_uint8), _p(sgn, C.c_uint32), _p(norm, C.c_float), d, L, s,
+    _check(lib().orc_decode_qsgd(_p(lvl, C.c_uint8), _p(sgn, C.c_uint32), _p(qstep, C.c_float), d, L,
                                  _p(Cv, C.c_float)), "decode_qsgd")
     return Cv
 

@@ -270,7 +270,7 @@ int orc_decode_topk(const uint32_t* idx, const float* val, uint64_t k, uint64_t 
 /* ------------------------------------------------------------------------ */
 
 int orc_q_qsgd(const float* v, uint64_t d, uint32_t L, uint32_t s, uint64_t seed, uint32_t step,
-               uint32_t wid, uint8_t* lvl, uint32_t* sgn, float* norm, float* C) {
+               uint32_t wid, uint8_t* lvl, uint32_t* sgn, float* norm, float* qstep, float* C) {
   if (!is_pow2_u32(L) || L < 4 || s < 1 || s > 255) return ORC_ERR_ARG;
   uint64_t nw = (d + 31) / 32, nc = (d + L - 1) / L;
   float* sq = (float*)malloc(sizeof(float) * L);
@@ -298,6 +298,7 @@ int orc_q_qsgd(const float* v, uint64_t d, uint32_t L, uint32_t s, uint64_t seed
     }
     if (!live) { N = 0.0f; q = 0.0f; inv_q = 0.0f; }
     norm[c] = N;
+    qstep[c] = q;
     for (uint32_t t = 0; t < len; ++t) {
       uint64_t j = lo + t;
       uint32_t ctr[4] = {t / 4, (uint32_t)c, wid, step};
@@ -325,12 +326,11 @@ int orc_q_qsgd(const float* v, uint64_t d, uint32_t L, uint32_t s, uint64_t seed
   return ORC_OK;
 }
 
-int orc_decode_qsgd(const uint8_t* lvl, const uint32_t* sgn, const float* norm, uint64_t d, uint32_t L,
-                    uint32_t s, float* C) {
-  if (L == 0 || s == 0) return ORC_ERR_ARG;
-  const float sf = (float)s;
+int orc_decode_qsgd(const uint8_t* lvl, const uint32_t* sgn, const float* qstep, uint64_t d, uint32_t L,
+                    float* C) {
+  if (L == 0) return ORC_ERR_ARG;
   for (uint64_t j = 0; j < d; ++j) {
-    float q = norm[j / L] / sf;
+    float q = qstep[j / L];
     float mag = (float)lvl[j] * q;
     int nonneg = (sgn[j / 32] >> (j % 32)) & 1u;
     C[j] = nonneg ? mag : -mag;

@@ -103,7 +103,7 @@ _VIEW_DTYPES = {
     "identity": (("c", torch.float32),),
     "sign1": (("bits", torch.int32), ("scale", torch.float32)),
     "topk": (("idx", torch.int32), ("val", torch.float32)),
-    "qsgd": (("lvl", torch.uint8), ("sgn", torch.int32), ("norm", torch.float32)),
+    "qsgd": (("lvl", torch.uint8), ("sgn", torch.int32), ("step", torch.float32)),
 }
 
 

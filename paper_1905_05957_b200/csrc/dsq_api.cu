@@ -165,8 +165,7 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       p.gamma = c->cfg.gamma;
       p.levels_f = (float)q.levels;
       p.levels_u = q.levels;
-      p.key0 = (uint32_t)(c->cfg.seed & 0xFFFFFFFFu);
-      p.key1 = (uint32_t)(c->cfg.seed >> 32);
+      p.keys = philox_key_schedule((uint32_t)(c->cfg.seed & 0xFFFFFFFFu), (uint32_t)(c->cfg.seed >> 32));
       p.step = step;
       p.server_pass = server ? 1u : 0u;
       e = launch_chunked(q.op, src_kind, src, p, rows, q.chunk, st);

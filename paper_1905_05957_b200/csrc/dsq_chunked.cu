@@ -108,12 +108,22 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
                          __fadd_rn(a[j].w, b[j].w));
     }
   } else {
+    uint64_t e[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) {
-      const uint64_t e = base + (uint64_t)(j * G + t) * 4u;
-      cnt[j] = FULL ? 4u : (e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u);
-      v[j] = cnt[j] ? src_load4<SRC>(src, row, e, cnt[j]) : make_float4(0.f, 0.f, 0.f, 0.f);
+      e[j] = base + (uint64_t)(j * G + t) * 4u;
+      cnt[j] = FULL ? 4u : (e[j] < d ? (uint32_t)min((uint64_t)4, d - e[j]) : 0u);
     }
+    src_load_tile<SRC, V>(src, row, e, cnt, v);
+  }
+
+  // fused model update (server pass): fetch x now so that its latency hides behind the reduction
+  constexpr bool kServer = SRC != SRC_WORKER;  // only a server pass can carry the update
+  float4 xv[kServer ? V : 1];
+  if (kServer && p.x) {
+#pragma unroll
+    for (int j = 0; j < V; ++j)
+      xv[kServer ? j : 0] = cnt[j] ? load_row4(p.x, base + (uint64_t)(j * G + t) * 4u, cnt[j], 1) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
 
   // ---- chunk reduction: sum |v| (SIGN1) or sum v*v (QSGD), pairwise in index order
@@ -164,7 +174,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
     }
     if (!live) { N = 0.f; q = 0.f; inv_q = 0.f; }
     s_or_q = q;
-    if (chunk_live && t == 0) p.out_scale[(uint64_t)row * p.scale_stride + c] = N;
+    if (chunk_live && t == 0) p.out_scale[(uint64_t)row * p.scale_stride + c] = q;  // the grid step is what is sent
   }
 
   // ---- encode, residual, optional model update
@@ -184,26 +194,30 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
         comp(C, k) = nonneg ? s_or_q : -s_or_q;
       }
     } else {
-      const uint4 rnd = philox4x32_10(make_uint4(tq, (uint32_t)c, p.server_pass ? 0xFFFFFFFFu : row, p.step),
-                                      p.key0, p.key1);
+      const uint4 rnd = philox4x32_10(make_uint4(tq, (uint32_t)c, p.server_pass ? 0xFFFFFFFFu : row, p.step), p.keys);
       const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-      uint32_t packed = 0;
+      uint32_t lb[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const float val = compc(v[j], k);
         const float u = __fmul_rn(__uint2float_rn(w[k] >> 8), 5.9604644775390625e-08f);  // 2^-24, exact
         float r = __fmul_rn(fabsf(val), inv_q);
         r = fminf(r, p.levels_f);
-        const float f = floorf(r);
-        const float pr = __fsub_rn(r, f);
-        uint32_t level = (uint32_t)f + (u < pr ? 1u : 0u);
-        level = min(level, p.levels_u);
-        const float mag = __fmul_rn((float)level, s_or_q);
+        // floor(r) for 0 <= r <= 255 without a conversion: adding 2^23 with rounding toward zero
+        // leaves 2^23 + floor(r), whose low mantissa byte is the integer and whose difference
+        // from 2^23 is the float
+        const float tz = __fadd_rz(r, 8388608.0f);
+        const float f = __fadd_rn(tz, -8388608.0f);
+        const float pr = __fsub_rn(r, f);  // exact
+        const bool up = u < pr;
+        lb[k] = __float_as_uint(tz) + (up ? 1u : 0u);      // low byte = level (no carry: r = 255 has pr = 0)
+        const float lf = up ? __fadd_rn(f, 1.0f) : f;      // the level as a float, exact
+        const float mag = __fmul_rn(lf, s_or_q);
         const bool nonneg = val >= 0.f;
         nib[j] |= (nonneg ? 1u : 0u) << k;
         comp(C, k) = nonneg ? mag : -mag;
-        packed |= level << (8 * k);
       }
+      const uint32_t packed = __byte_perm(__byte_perm(lb[0], lb[1], 0x0040), __byte_perm(lb[2], lb[3], 0x0040), 0x5410);
       if (cnt[j]) *reinterpret_cast<uint32_t*>(p.out_lvl + (uint64_t)row * p.lvl_stride + e) = packed;
     }
     if constexpr (!FULL) nib[j] &= (1u << cnt[j]) - 1u;  // pad bits are 0
@@ -217,11 +231,12 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
       } else {
         store_row4(delta_chunk, (uint64_t)tq * 4u, cnt[j], src.vec, dl);
       }
-      if (p.x) {  // fused model update (server pass only): x = x - gamma * Q[v]
-        float4 xv = load_row4(p.x, e, cnt[j], 1);
-        xv.x = __fsub_rn(xv.x, __fmul_rn(p.gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(p.gamma, C.y));
-        xv.z = __fsub_rn(xv.z, __fmul_rn(p.gamma, C.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(p.gamma, C.w));
-        store_row4(p.x, e, cnt[j], 1, xv);
+      if (kServer && p.x) {  // fused model update (server pass only): x = x - gamma * Q[v]
+        const float4 xo = xv[kServer ? j : 0];
+        float4 xn;
+        xn.x = __fsub_rn(xo.x, __fmul_rn(p.gamma, C.x)); xn.y = __fsub_rn(xo.y, __fmul_rn(p.gamma, C.y));
+        xn.z = __fsub_rn(xo.z, __fmul_rn(p.gamma, C.z)); xn.w = __fsub_rn(xo.w, __fmul_rn(p.gamma, C.w));
+        store_row4(p.x, e, cnt[j], 1, xn);
       }
     }
   }

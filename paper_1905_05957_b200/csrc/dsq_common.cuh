@@ -44,7 +44,7 @@ __device__ __forceinline__ float4 load_row4(const float* base, uint64_t e, uint3
   float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
   if (vec && cnt == 4) {
     r = ld_stream4(base + e);
-  } else {
+  } else if (cnt) {
 #pragma unroll
     for (int k = 0; k < 4; ++k)
       if ((uint32_t)k < cnt) comp(r, k) = __ldcs(base + e + k);
@@ -62,78 +62,155 @@ __device__ __forceinline__ void store_row4(float* base, uint64_t e, uint32_t cnt
   }
 }
 
-// The vector to compress, four consecutive entries at offset e of row `row`.  cnt in [1, 4] is the
-// number of entries that exist (e + cnt <= d); the others are returned as +0.
-template <int SRC>
-__device__ __forceinline__ float4 src_load4(const SrcParams& p, uint32_t row, uint64_t e, uint32_t cnt) {
+// +m or -m according to bit `k` of the sign word `w` (1 = non-negative), without a branch.
+__device__ __forceinline__ float signed_by_bit(float m, uint32_t w, int k) {
+  return __uint_as_float(__float_as_uint(m) ^ ((~w << (31 - k)) & 0x80000000u));
+}
+
+// Exact float value of byte `k` of `x`: place the byte in the mantissa of 2^23 and subtract 2^23.
+__device__ __forceinline__ float byte_to_float(uint32_t x, int k) {
+  return __fadd_rn(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7440u + k)), -8388608.0f);
+}
+
+// The vector to compress, for a tile of V rows: row j of the calling thread is the float4 at entry
+// e[j] of vector `row`; cnt[j] in [0, 4] says how many of its entries exist (the others, and whole
+// rows with cnt 0, are returned as +0).  Must be called by all 32 lanes of a warp together, the
+// lanes holding consecutive float4 of each row (e[j] = 128-aligned warp base + 4 * lane): server
+// sources load the sign words and scales of eight workers with one instruction per row (lane l
+// fetches word l%4 of worker l/4) and hand them round with shuffles.  Workers are accumulated in
+// order 0..n-1, the order in which Eq. 4 is summed.
+template <int SRC, int V>
+__device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, const uint64_t (&e)[V],
+                                              const uint32_t (&cnt)[V], float4 (&v)[V]) {
   if constexpr (SRC == SRC_WORKER) {
     const uint64_t off = (uint64_t)row * p.d;
-    float4 a = load_row4(p.g + off, e, cnt, p.vec);
-    float4 b = load_row4(p.delta + off, e, cnt, p.vec);
-    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+    float4 a[V], b[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) a[j] = load_row4(p.g + off, e[j], cnt[j], p.vec);
+#pragma unroll
+    for (int j = 0; j < V; ++j) b[j] = load_row4(p.delta + off, e[j], cnt[j], p.vec);
+#pragma unroll
+    for (int j = 0; j < V; ++j)
+      v[j] = make_float4(__fadd_rn(a[j].x, b[j].x), __fadd_rn(a[j].y, b[j].y), __fadd_rn(a[j].z, b[j].z),
+                         __fadd_rn(a[j].w, b[j].w));
   } else {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint32_t lane = threadIdx.x & 31u;
+    float4 acc[V], ds[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      ds[j] = load_row4(p.delta, e[j], cnt[j], p.vec);
+    }
     if constexpr (SRC == SRC_SRV_IDENTITY) {
       for (uint32_t i = 0; i < p.n; ++i) {
         const float* c = reinterpret_cast<const float*>(p.wp + i * p.wp_stride + p.wp_off[0]);
-        float4 ci = load_row4(c, e, cnt, 1);
-        acc.x = __fadd_rn(acc.x, ci.x); acc.y = __fadd_rn(acc.y, ci.y);
-        acc.z = __fadd_rn(acc.z, ci.z); acc.w = __fadd_rn(acc.w, ci.w);
-      }
-    } else if constexpr (SRC == SRC_SRV_SIGN1) {
-      const uint64_t word = e >> 5;
-      const uint32_t sh = (uint32_t)(e & 31);
-      const uint64_t ch = e >> p.w_log2_chunk;
-      for (uint32_t i = 0; i < p.n; ++i) {
-        const uint8_t* pl = p.wp + i * p.wp_stride;
-        const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pl + p.wp_off[0]) + word) >> sh;
-        const float s = __ldg(reinterpret_cast<const float*>(pl + p.wp_off[1]) + ch);
-        acc.x = __fadd_rn(acc.x, (w & 1u) ? s : -s); acc.y = __fadd_rn(acc.y, (w & 2u) ? s : -s);
-        acc.z = __fadd_rn(acc.z, (w & 4u) ? s : -s); acc.w = __fadd_rn(acc.w, (w & 8u) ? s : -s);
-      }
-    } else if constexpr (SRC == SRC_SRV_QSGD) {
-      const uint64_t word = e >> 5;
-      const uint32_t sh = (uint32_t)(e & 31);
-      const uint64_t ch = e >> p.w_log2_chunk;
-      for (uint32_t i = 0; i < p.n; ++i) {
-        const uint8_t* pl = p.wp + i * p.wp_stride;
-        const uint32_t lv = __ldcs(reinterpret_cast<const uint32_t*>(pl + p.wp_off[0] + e));
-        const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pl + p.wp_off[1]) + word) >> sh;
-        const float nrm = __ldg(reinterpret_cast<const float*>(pl + p.wp_off[2]) + ch);
-        const float q = __fdiv_rn(nrm, p.w_levels);
-        const float m0 = __fmul_rn((float)(lv & 255u), q), m1 = __fmul_rn((float)((lv >> 8) & 255u), q);
-        const float m2 = __fmul_rn((float)((lv >> 16) & 255u), q), m3 = __fmul_rn((float)(lv >> 24), q);
-        acc.x = __fadd_rn(acc.x, (w & 1u) ? m0 : -m0); acc.y = __fadd_rn(acc.y, (w & 2u) ? m1 : -m1);
-        acc.z = __fadd_rn(acc.z, (w & 4u) ? m2 : -m2); acc.w = __fadd_rn(acc.w, (w & 8u) ? m3 : -m3);
-      }
-    } else {  // SRC_SRV_TOPK
-      acc = load_row4(p.acc, e, cnt, p.vec);
-      store_row4(p.acc, e, cnt, p.vec, make_float4(0.f, 0.f, 0.f, 0.f));
-    }
-    float4 ds = load_row4(p.delta, e, cnt, p.vec);
-    float4 v;
-    v.x = __fadd_rn(__fmul_rn(acc.x, p.inv_n), ds.x); v.y = __fadd_rn(__fmul_rn(acc.y, p.inv_n), ds.y);
-    v.z = __fadd_rn(__fmul_rn(acc.z, p.inv_n), ds.z); v.w = __fadd_rn(__fmul_rn(acc.w, p.inv_n), ds.w);
-    // entries past the end must read as +0 whatever the payload padding holds
-    if (cnt < 4) {
+        float4 ci[V];
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if ((uint32_t)k >= cnt) comp(v, k) = 0.f;
+        for (int j = 0; j < V; ++j) ci[j] = load_row4(c, e[j], cnt[j], 1);
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          acc[j].x = __fadd_rn(acc[j].x, ci[j].x); acc[j].y = __fadd_rn(acc[j].y, ci[j].y);
+          acc[j].z = __fadd_rn(acc[j].z, ci[j].z); acc[j].w = __fadd_rn(acc[j].w, ci[j].w);
+        }
+      }
+    } else if constexpr (SRC == SRC_SRV_SIGN1 || SRC == SRC_SRV_QSGD) {
+      constexpr int kSgn = SRC == SRC_SRV_SIGN1 ? 0 : 1;    // payload sub-array of the sign words
+      constexpr int kScl = SRC == SRC_SRV_SIGN1 ? 1 : 2;    // ... of the per-chunk scale / grid step
+      const uint64_t nw = (p.d + 31) >> 5;
+      const uint32_t sh = (lane & 7u) * 4u;                 // this lane's nibble inside its word
+      for (uint32_t i0 = 0; i0 < p.n; i0 += 8) {
+        uint32_t wreg[V];
+        float sreg[V];
+        uint32_t lv[SRC == SRC_SRV_QSGD ? V : 1][SRC == SRC_SRV_QSGD ? 8 : 1];
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          // warp base of this row: entry of lane 0 (valid arithmetic even where the row is past the end)
+          const uint64_t e0 = e[j] - 4u * lane;
+          const uint64_t word = (e0 >> 5) + (lane & 3u);
+          const uint32_t wi = i0 + (lane >> 2);
+          wreg[j] = 0;
+          sreg[j] = 0.f;
+          if (wi < p.n && word < nw)
+            wreg[j] = __ldg(reinterpret_cast<const uint32_t*>(p.wp + wi * p.wp_stride + p.wp_off[kSgn]) + word);
+          if (lane < 8 && i0 + lane < p.n && e0 < p.d)
+            sreg[j] = __ldg(reinterpret_cast<const float*>(p.wp + (i0 + lane) * p.wp_stride + p.wp_off[kScl]) +
+                            (e0 >> p.w_log2_chunk));
+          if constexpr (SRC == SRC_SRV_QSGD) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              lv[j][u] = 0;
+              if (i0 + u < p.n && cnt[j])
+                lv[j][u] = __ldcs(reinterpret_cast<const uint32_t*>(p.wp + (i0 + u) * p.wp_stride + p.wp_off[0] + e[j]));
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const uint32_t ww = __shfl_sync(0xffffffffu, wreg[j], u * 4 + (lane >> 3)) >> sh;
+            const float sc = __shfl_sync(0xffffffffu, sreg[j], u);
+            if (i0 + u < p.n) {
+              if constexpr (SRC == SRC_SRV_SIGN1) {
+                acc[j].x = __fadd_rn(acc[j].x, signed_by_bit(sc, ww, 0));
+                acc[j].y = __fadd_rn(acc[j].y, signed_by_bit(sc, ww, 1));
+                acc[j].z = __fadd_rn(acc[j].z, signed_by_bit(sc, ww, 2));
+                acc[j].w = __fadd_rn(acc[j].w, signed_by_bit(sc, ww, 3));
+              } else {
+                const uint32_t l4 = lv[j][u];
+                acc[j].x = __fadd_rn(acc[j].x, signed_by_bit(__fmul_rn(byte_to_float(l4, 0), sc), ww, 0));
+                acc[j].y = __fadd_rn(acc[j].y, signed_by_bit(__fmul_rn(byte_to_float(l4, 1), sc), ww, 1));
+                acc[j].z = __fadd_rn(acc[j].z, signed_by_bit(__fmul_rn(byte_to_float(l4, 2), sc), ww, 2));
+                acc[j].w = __fadd_rn(acc[j].w, signed_by_bit(__fmul_rn(byte_to_float(l4, 3), sc), ww, 3));
+              }
+            }
+          }
+        }
+      }
+    } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc; consume and clear it
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        acc[j] = load_row4(p.acc, e[j], cnt[j], p.vec);
+        store_row4(p.acc, e[j], cnt[j], p.vec, make_float4(0.f, 0.f, 0.f, 0.f));
+      }
     }
-    return v;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      v[j].x = __fadd_rn(__fmul_rn(acc[j].x, p.inv_n), ds[j].x); v[j].y = __fadd_rn(__fmul_rn(acc[j].y, p.inv_n), ds[j].y);
+      v[j].z = __fadd_rn(__fmul_rn(acc[j].z, p.inv_n), ds[j].z); v[j].w = __fadd_rn(__fmul_rn(acc[j].w, p.inv_n), ds[j].w);
+      // entries past the end must read as +0 whatever the payload padding holds
+      if (cnt[j] < 4) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)k >= cnt[j]) comp(v[j], k) = 0.f;
+      }
+    }
   }
 }
 
-// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and xors, the key
-// advanced by the two Weyl constants between rounds.
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and xors.  The key
+// of round r is key + r * (0x9E3779B9, 0xBB67AE85); the twenty round-key words are computed once
+// on the host (philox_key_schedule) and read from the kernel parameters.
+struct PhiloxKeys {
+  uint32_t k[10][2];
+};
+
+__host__ __device__ inline PhiloxKeys philox_key_schedule(uint32_t k0, uint32_t k1) {
+  PhiloxKeys ks;
+  for (int r = 0; r < 10; ++r) {
+    ks.k[r][0] = k0 + (uint32_t)r * 0x9E3779B9u;
+    ks.k[r][1] = k1 + (uint32_t)r * 0xBB67AE85u;
+  }
+  return ks;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const PhiloxKeys& ks) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
-    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c.x;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c.z;
+    c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ ks.k[r][0], (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ ks.k[r][1],
+                   (uint32_t)p0);
   }
   return c;
 }

@@ -12,10 +12,16 @@ __global__ void __launch_bounds__(kThreads) k_identity(const SrcParams src, floa
                                                        float gamma) {
   const uint32_t row = blockIdx.y;
   const uint64_t nq = (src.d + 3) / 4;
-  for (uint64_t qd = (uint64_t)blockIdx.x * kThreads + threadIdx.x; qd < nq; qd += (uint64_t)gridDim.x * kThreads) {
-    const uint64_t e = qd * 4;
-    const uint32_t cnt = (uint32_t)min((uint64_t)4, src.d - e);
-    const float4 v = src_load4<SRC>(src, row, e, cnt);
+  // the loop bound is the same for all threads of the CTA: the source is read warp-cooperatively
+  for (uint64_t q0 = (uint64_t)blockIdx.x * kThreads; q0 < nq; q0 += (uint64_t)gridDim.x * kThreads) {
+    const uint64_t ee[1] = {(q0 + threadIdx.x) * 4};
+    const uint64_t e = ee[0];
+    const uint32_t cc[1] = {e < src.d ? (uint32_t)min((uint64_t)4, src.d - e) : 0u};
+    const uint32_t cnt = cc[0];
+    float4 vv[1];
+    src_load_tile<SRC, 1>(src, row, ee, cc, vv);
+    const float4 v = vv[0];
+    if (!cnt) continue;
     store_row4(out_c + (uint64_t)row * c_row_stride, e, cnt, 1, v);  // Q[v] = v
     store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, make_float4(0.f, 0.f, 0.f, 0.f));
     if (x) {
@@ -62,15 +68,15 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, 
     } else if (pv.op == DS_Q_SIGN1) {
       const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]) + (e >> 5)) >> (uint32_t)(e & 31);
       const float s = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
-      C = make_float4((w & 1u) ? s : -s, (w & 2u) ? s : -s, (w & 4u) ? s : -s, (w & 8u) ? s : -s);
+      C = make_float4(signed_by_bit(s, w, 0), signed_by_bit(s, w, 1), signed_by_bit(s, w, 2), signed_by_bit(s, w, 3));
     } else {  // DS_Q_QSGD
       const uint32_t lv = __ldcs(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0] + e));
       const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[1]) + (e >> 5)) >> (uint32_t)(e & 31);
-      const float q = __fdiv_rn(__ldg(reinterpret_cast<const float*>(pv.base + pv.off[2]) + (e >> pv.log2_chunk)),
-                                pv.levels_f);
-      const float m0 = __fmul_rn((float)(lv & 255u), q), m1 = __fmul_rn((float)((lv >> 8) & 255u), q);
-      const float m2 = __fmul_rn((float)((lv >> 16) & 255u), q), m3 = __fmul_rn((float)(lv >> 24), q);
-      C = make_float4((w & 1u) ? m0 : -m0, (w & 2u) ? m1 : -m1, (w & 4u) ? m2 : -m2, (w & 8u) ? m3 : -m3);
+      const float q = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[2]) + (e >> pv.log2_chunk));
+      C = make_float4(signed_by_bit(__fmul_rn(byte_to_float(lv, 0), q), w, 0),
+                      signed_by_bit(__fmul_rn(byte_to_float(lv, 1), q), w, 1),
+                      signed_by_bit(__fmul_rn(byte_to_float(lv, 2), q), w, 2),
+                      signed_by_bit(__fmul_rn(byte_to_float(lv, 3), q), w, 3));
     }
     float4 xv = load_row4(x, e, cnt, 1);
     xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));

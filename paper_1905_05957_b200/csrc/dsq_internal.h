@@ -15,7 +15,7 @@ inline void count_launches(uint64_t n) { g_kernel_launches += n; }
 // Destination of a chunk-wise operator (SIGN1 or QSGD).
 struct ChunkParams {
   uint32_t* out_bits;        // sign words, row stride bits_stride (in words)
-  float* out_scale;          // SIGN1: scale per chunk; QSGD: norm per chunk; row stride scale_stride (floats)
+  float* out_scale;          // SIGN1: scale per chunk; QSGD: grid step q per chunk; row stride scale_stride (floats)
   uint8_t* out_lvl;          // QSGD: level bytes, row stride lvl_stride (bytes)
   uint64_t bits_stride, scale_stride, lvl_stride;
   float* delta_out;          // residual destination, row stride delta_row_stride (floats)
@@ -24,7 +24,8 @@ struct ChunkParams {
   float gamma;
   float levels_f;            // QSGD: s
   uint32_t levels_u;
-  uint32_t key0, key1, step; // Philox key and the step word of the counter
+  PhiloxKeys keys;           // Philox round keys
+  uint32_t step;             // the step word of the counter
   uint32_t server_pass;      // 1: counter word 2 is 0xFFFFFFFF, else the row (worker) index
   uint32_t log2G;            // filled by the launcher
 };

@@ -28,7 +28,7 @@ namespace {
 constexpr uint32_t kBins1 = 4096;        // key bits 30..19
 constexpr uint32_t kSegWords = 256;      // bitmap words per segment (one per thread)
 constexpr uint32_t kSegElems = kSegWords * 32;
-constexpr uint64_t kPass1Span = 65536;   // entries per CTA of pass1 (amortises the histogram flush)
+constexpr uint64_t kPass1Step = 4096;    // entries one CTA of pass1 handles per loop trip
 
 __device__ __forceinline__ uint32_t key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
@@ -36,24 +36,25 @@ inline uint64_t round16(uint64_t b) { return (b + 15u) & ~uint64_t(15); }
 
 // ---------------------------------------------------------------- pass1
 template <int SRC>
-__global__ void __launch_bounds__(kThreads) k_topk_pass1(const SrcParams src, float* v_out, uint32_t* hist) {
+__global__ void __launch_bounds__(kThreads) k_topk_pass1(const SrcParams src, float* v_out, uint32_t* hist, uint64_t span) {
   __shared__ uint32_t s_hist[kBins1];
   const uint32_t tid = threadIdx.x, row = blockIdx.y;
   for (uint32_t b = tid; b < kBins1; b += kThreads) s_hist[b] = 0;
   __syncthreads();
   const uint64_t d = src.d;
-  const uint64_t begin = (uint64_t)blockIdx.x * kPass1Span;
-  const uint64_t end = min(begin + kPass1Span, d);
+  const uint64_t begin = (uint64_t)blockIdx.x * span;  // span: a multiple of kPass1Step
+  const uint64_t end = min(begin + span, d);
   float* out_row = v_out + (uint64_t)row * d;
-  for (uint64_t base = begin; base < end; base += 4u * kThreads * 4u) {
+  for (uint64_t base = begin; base < end; base += kPass1Step) {
     float4 v[4];
     uint32_t cnt[4];
+    uint64_t ee[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const uint64_t e = base + (uint64_t)(j * kThreads + tid) * 4u;
-      cnt[j] = e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u;
-      v[j] = cnt[j] ? src_load4<SRC>(src, row, e, cnt[j]) : make_float4(0.f, 0.f, 0.f, 0.f);
+      ee[j] = base + (uint64_t)(j * kThreads + tid) * 4u;
+      cnt[j] = ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u;
     }
+    src_load_tile<SRC, 4>(src, row, ee, cnt, v);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (!cnt[j]) continue;
@@ -388,8 +389,11 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   cudaError_t e = cudaMemsetAsync(hist, 0, (uint64_t)rows * kBins1 * 4, st);
   if (e != cudaSuccess) return e;
 
-  dim3 g1((unsigned)((d + kPass1Span - 1) / kPass1Span), rows, 1);
-#define DSQ_P1(S) k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, hist)
+  // entries per CTA: long spans amortise the histogram flush, but the grid must still fill the GPU
+  uint64_t span = 16 * kPass1Step;
+  while (span > kPass1Step && ((d + span - 1) / span) * rows < 148ull * 16ull) span /= 2;
+  dim3 g1((unsigned)((d + span - 1) / span), rows, 1);
+#define DSQ_P1(S) k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, hist, span)
   switch (srck) {
     case SRC_WORKER: DSQ_P1(SRC_WORKER); break;
     case SRC_SRV_IDENTITY: DSQ_P1(SRC_SRV_IDENTITY); break;

@@ -53,7 +53,7 @@ def compare_payload(name: str, op: str, gpu_views: dict, ora: dict):
     elif op == "qsgd":
         assert_bits_match(f"{name}.lvl", u32(gpu_views["lvl"]), ora["lvl"])
         assert_bits_match(f"{name}.sgn", u32(gpu_views["sgn"]), ora["sgn"])
-        assert_float_match(f"{name}.norm", gpu_views["norm"].cpu().numpy(), ora["norm"])
+        assert_float_match(f"{name}.step", gpu_views["step"].cpu().numpy(), ora["step"])
     else:
         raise ValueError(op)
 

@@ -179,7 +179,8 @@ def test_qsgd_levels_bracket_the_value_and_decode_roundtrip():
     lv = p["lvl"].astype(np.float64)
     assert np.all(lv >= np.floor(rr) - 1e-3) and np.all(lv <= np.floor(rr) + 1 + 1e-3)
     assert np.all(np.abs(C.astype(np.float64) - v) <= q * (1 + 1e-5))
-    assert np.array_equal(oracle.decode_qsgd(p["lvl"], p["sgn"], p["norm"], d, L, s), C)
+    assert np.array_equal(oracle.decode_qsgd(p["lvl"], p["sgn"], p["step"], d, L), C)
+    assert np.array_equal(p["step"], p["norm"] / np.float32(s))     # what is sent is q = N / s
     # the random stream depends on step, worker and seed, and on nothing else
     C2, p2 = oracle.q_qsgd(v, L, s, 5, 9, 1)
     assert np.array_equal(p["lvl"], p2["lvl"])
