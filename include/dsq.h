@@ -192,6 +192,34 @@ int ds_destroy(ds_handle h);
 int ds_step_host(ds_handle h, const float* g_host, float* g_dev, uint32_t step, void* server_payload_host,
                  float* x_host, void* cuda_stream);
 
+/*
+ * (No counterpart in the paper: a packaging variant of the top-k worker step for one vector.)
+ *
+ * For callers that must not allocate device memory where they compress -- inside a stream
+ * capture, as a plug-in of a framework that owns the memory pool, or in a loop where allocation is
+ * forbidden after start-up -- and therefore cannot provide the top-k workspace that ds_create asks
+ * for.  Computes, for ONE vector,  v = g + delta,  (idx, val) = top-k of v (same rules as
+ * DS_Q_TOPK),  delta = v - Q[v],  using scratch memory that is a fixed array inside the library.
+ *
+ *   g, delta   device float[d]; delta is read and overwritten in place
+ *   idx, val   device uint32[k], float[k]: ascending indices and the values kept
+ *   dev_status device uint32[1], zero-filled by the caller; DS_DEV_* bits are OR-ed in
+ *
+ * Limits and rules:
+ *  - d <= DS_STATIC_TOPK_MAX_D, else DS_ERR_UNSUPPORTED and nothing is launched.  The array costs
+ *    about 2 MiB of device memory on every GPU that loads the library, until the process exits.
+ *  - Calls no cudaMalloc/cudaFree and no allocating library routine.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - All calls share the one array: two calls whose kernels may overlap on the GPU (different
+ *    streams, no dependency between them) race.  Issue them on one stream or order them.
+ *  - Asynchronous on cuda_stream like the other calls; pointers must be 4-byte aligned (16-byte
+ *    aligned g and delta with d % 4 == 0 take the vector path).
+ */
+#define DS_STATIC_TOPK_MAX_D (1u << 23)
+int ds_topk_worker_static(const float* g, float* delta, uint64_t d, uint64_t k, uint32_t* idx, float* val,
+                          uint32_t* dev_status, void* cuda_stream);
+
 /* Text of the most recent CUDA error seen by this thread's calls ("" if none). */
 const char* ds_last_error(void);
 

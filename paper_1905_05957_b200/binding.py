@@ -23,7 +23,7 @@ DS_DEV_TOPK_INCONSISTENT = 1
 OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3}
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
            "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
-           "ds_kernel_launches")
+           "ds_kernel_launches", "ds_topk_worker_static")
 
 
 class ds_qspec(C.Structure):
@@ -75,6 +75,7 @@ def load_library() -> C.CDLL:
     L.ds_apply_update.argtypes = [vp, vp]
     L.ds_destroy.argtypes = [vp]
     L.ds_step_host.argtypes = [vp, vp, vp, u32, vp, vp, vp]
+    L.ds_topk_worker_static.argtypes = [vp, vp, C.c_uint64, C.c_uint64, vp, vp, vp, vp]
     for name in EXPORTS:
         getattr(L, name).restype = C.c_int
     L.ds_last_error.restype = C.c_char_p
@@ -119,6 +120,22 @@ def payload_views(buf: torch.Tensor, layout: ds_payload_layout, op: str, rows: i
             views[name] = buf[base + layout.off[j]: base + layout.off[j] + nbytes].view(dt)
         out.append(views)
     return out
+
+
+DS_STATIC_TOPK_MAX_D = 1 << 23
+
+
+def topk_worker_static(g: torch.Tensor, delta: torch.Tensor, k: int, idx: torch.Tensor, val: torch.Tensor,
+                       dev_status: torch.Tensor, stream=None) -> None:
+    """ds_topk_worker_static: top-k with error feedback for one vector, using the library's built-in
+    scratch array, for callers that cannot allocate device memory where they compress (inside a
+    stream capture, or as a guest of a framework that owns the memory pool).  All tensors are the
+    caller's; delta is updated in place.  Calls on different streams must not overlap."""
+    s = stream if stream is not None else torch.cuda.current_stream(g.device)
+    rc = load_library().ds_topk_worker_static(g.data_ptr(), delta.data_ptr(), g.numel(), k, idx.data_ptr(),
+                                              val.data_ptr(), dev_status.data_ptr(), s.cuda_stream)
+    if rc != DS_OK:
+        raise DsqError(rc, "ds_topk_worker_static")
 
 
 class DoubleSqueeze:

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libdsq.so")
-SOURCES = ["dsq_api.cu", "dsq_chunked.cu", "dsq_elementwise.cu", "dsq_topk.cu"]
+SOURCES = ["dsq_api.cu", "dsq_chunked.cu", "dsq_elementwise.cu", "dsq_topk.cu", "dsq_static.cu"]
 HEADERS = ["dsq_common.cuh", "dsq_internal.h", os.path.join("..", "..", "include", "dsq.h")]
 
 NVCC_FLAGS = [
