@@ -112,8 +112,9 @@ typedef struct {
  *   delta_s  float[d]        server error; the caller zero-fills
  *   worker_payload           n payloads at a fixed stride, see ds_get_layout()
  *   server_payload           one payload
- *   workspace                scratch of the top-k path (contents are meaningless between calls);
- *                            may be NULL when workspace_bytes is 0
+ *   workspace                scratch of the top-k path; may be NULL when workspace_bytes is 0.
+ *                            Zero-fill it once.  Between calls it holds only hints (the previous
+ *                            steps' threshold bins); whatever it holds, results are the same
  *   dev_status uint32[1]     the caller zero-fills
  * Every non-NULL pointer must be 16-byte aligned and at least *_bytes long.
  */

@@ -78,15 +78,17 @@ struct ds_ctx {
 namespace {
 
 // Workspace = [top-k scratch shared by both passes][dense accumulator for sparse worker payloads]
+//             [threshold history of the n worker vectors][threshold history of the server vector]
+// Only the histories carry meaning from one call to the next, and only as a hint.
 uint64_t plan_workspace(ds_ctx* c) {
   const ds_config& cfg = c->cfg;
   uint64_t topk_bytes = 0;
   if (cfg.worker_q.op == DS_Q_TOPK) {
-    topk_plan(cfg.d, cfg.n, cfg.worker_q.k, &c->wplan);
+    topk_plan(cfg.d, cfg.n, cfg.worker_q.k, true, &c->wplan);
     topk_bytes = c->wplan.bytes;
   }
   if (cfg.server_q.op == DS_Q_TOPK) {
-    topk_plan(cfg.d, 1, cfg.server_q.k, &c->splan);
+    topk_plan(cfg.d, 1, cfg.server_q.k, true, &c->splan);
     if (c->splan.bytes > topk_bytes) topk_bytes = c->splan.bytes;
   }
   uint64_t total = round16(topk_bytes);
@@ -95,6 +97,15 @@ uint64_t plan_workspace(ds_ctx* c) {
   c->acc = (cfg.worker_q.op == DS_Q_TOPK && c->buf.workspace)
                ? reinterpret_cast<float*>(static_cast<uint8_t*>(c->buf.workspace) + acc_off)
                : nullptr;
+  uint8_t* ws = static_cast<uint8_t*>(c->buf.workspace);
+  if (cfg.worker_q.op == DS_Q_TOPK) {
+    c->wplan.pred = ws ? reinterpret_cast<TopkPred*>(ws + total) : nullptr;
+    total += round16((uint64_t)cfg.n * sizeof(TopkPred));
+  }
+  if (cfg.server_q.op == DS_Q_TOPK) {
+    c->splan.pred = ws ? reinterpret_cast<TopkPred*>(ws + total) : nullptr;
+    total += round16(sizeof(TopkPred));
+  }
   return total;
 }
 

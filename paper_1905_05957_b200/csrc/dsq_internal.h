@@ -46,17 +46,25 @@ struct TopkState {
   uint32_t tb1, tb2;   // threshold digits: key bits 30..19 and 18..7
   uint32_t tau;        // full 31-bit key of the k-th largest entry
   uint32_t r;          // how many entries with key == tau are kept (lowest indices first)
-  uint32_t total_gt, total_tie, pad;
+  uint32_t total_gt, total_tie;
+  uint32_t need_mark;  // 1: the bitmaps pass1 wrote (if any) do not bracket the threshold bin
+};
+
+// Threshold-bin history of one vector, kept across steps so that pass1 can mark candidates itself.
+struct TopkPred {
+  uint32_t magic, tb_last, tb_prev, pad;
 };
 
 // Carving of the workspace for `rows` simultaneous selections over d-vectors.
 struct TopkPlan {
   uint64_t d, k;
   uint32_t rows;
-  uint64_t nseg;        // 8192-entry segments per vector
+  uint64_t nseg;        // 32768-entry segments per vector
   uint64_t bm_stride;   // bitmap words per vector (whole segments)
-  uint64_t off_hist, off_state, off_bm_gt, off_bm_eq, off_seg;
+  uint64_t list_cap;    // capacity of the candidate-key list per vector (0: no list, gather instead)
+  uint64_t off_hist, off_list_count, off_state, off_bm_gt, off_bm_eq, off_seg, off_list;
   uint64_t bytes;
+  TopkPred* pred;       // [rows] history outside the scratch (device memory), or NULL: no prediction
 };
 
 struct TopkIO {
@@ -69,7 +77,7 @@ struct TopkIO {
   uint32_t* dev_status;
 };
 
-void topk_plan(uint64_t d, uint32_t rows, uint64_t k, TopkPlan* plan);
+void topk_plan(uint64_t d, uint32_t rows, uint64_t k, bool with_list, TopkPlan* plan);
 cudaError_t launch_topk(int src_kind, const SrcParams& src, const TopkPlan& plan, void* workspace, const TopkIO& io,
                         uint32_t rows, uint64_t k, cudaStream_t st);
 

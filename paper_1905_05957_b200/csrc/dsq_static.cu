@@ -13,8 +13,8 @@ using namespace dsq;
 
 namespace {
 
-// Scratch for one selection over at most DS_STATIC_TOPK_MAX_D entries: 16 KiB histogram, 32 B state,
-// two bitmaps of MAX_D/8 bytes each, MAX_D/8192 segment counts of 8 bytes -- about 2.03 MiB.
+// Scratch for one selection over at most DS_STATIC_TOPK_MAX_D entries: 16 KiB histogram, a few words of
+// select state, two bitmaps of MAX_D/8 bytes each and the segment counts -- about 2.03 MiB.
 // Every GPU that loads the library holds this array until the process exits.
 constexpr size_t kScratchBytes = 16384 + 32 + 2 * (DS_STATIC_TOPK_MAX_D / 8) + (DS_STATIC_TOPK_MAX_D / 8192) * 8 + 256;
 static __device__ __align__(256) unsigned char g_topk_scratch[kScratchBytes];
@@ -52,7 +52,7 @@ extern "C" int ds_topk_worker_static(const float* g, float* delta, uint64_t d, u
                         reinterpret_cast<uintptr_t>(dev_status);
   if (all & 3u) return DS_ERR_ALIGN;
   TopkPlan plan;
-  topk_plan(d, 1, k, &plan);
+  topk_plan(d, 1, k, false, &plan);  // no candidate list: the scratch stays small
   if (plan.bytes > kScratchBytes) return DS_ERR_UNSUPPORTED;
   void* scratch = nullptr;
   if (scratch_for_current_device(&scratch) != cudaSuccess) return DS_ERR_CUDA;

@@ -15,7 +15,7 @@ TOPK = lambda k: Q("topk", k=k)
 IDENT = Q("identity")
 
 
-def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None):
+def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None, scribble=False):
     """Free-running: both sides start from the same state and see the same gradients; after every
     step every output must agree."""
     ds = DoubleSqueeze(n, d, gamma, wq, sq, seed, x0=x0)
@@ -27,6 +27,8 @@ def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None
         st.delta_w = dw.cpu().numpy().copy()
         st.delta_s = dsv.cpu().numpy().copy()
     for t, g in enumerate(gs):
+        if scribble:   # the workspace only ever holds hints: any contents must give the same results
+            ds.workspace.random_(0, 256)
         g_dev = g.cuda().contiguous()
         ds.step(g_dev, t, fuse_apply=fuse)
         torch.cuda.synchronize()
@@ -117,6 +119,19 @@ def test_zero_signed_zero_subnormal_and_zero_chunks():
     g[0, 8192:] = 1e-30          # squares underflow: a quantisation chunk of norm ~0
     for wq in (SIGN(4096), QSGD(2048), TOPK(100), SIGN(128), QSGD(128, 5)):
         run_lockstep(n, d, wq, wq, [g, g.clone(), -g])
+
+
+def test_topk_threshold_prediction_hits_misses_and_garbage():
+    """Top-k marks candidates during its first pass from the previous steps' threshold bins.  Steady
+    magnitudes make the prediction hit, jumps make it miss (the slow path runs), and a workspace
+    full of random bytes must change nothing."""
+    n, d, k = 3, 120_000, 1200
+    gen = torch.Generator().manual_seed(8)
+    scales = [1, 1, 1, 1, 1.02, 1.05, 8.0, 8.0, 0.01, 0.01, 0.01, 1, 1]
+    gs = [torch.randn(n, d, generator=gen) * s for s in scales]
+    run_lockstep(n, d, TOPK(k), TOPK(k), gs)
+    run_lockstep(n, d, SIGN(4096), TOPK(k // 2), gs[:6])
+    run_lockstep(n, d, TOPK(k), TOPK(k), gs[:5], scribble=True)
 
 
 def test_qsgd_stream_depends_on_seed_and_step():
