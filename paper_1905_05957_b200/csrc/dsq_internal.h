@@ -47,7 +47,9 @@ struct TopkState {
   uint32_t tau;        // full 31-bit key of the k-th largest entry
   uint32_t r;          // how many entries with key == tau are kept (lowest indices first)
   uint32_t total_gt, total_tie;
-  uint32_t need_mark;  // 1: the bitmaps pass1 wrote (if any) do not bracket the threshold bin
+  uint32_t need_mark;  // 1: the bitmap and list pass1 wrote (if any) do not bracket the threshold bin
+  uint32_t need_full;  // 1: the partial histogram of pass1 (if any) did not reach the k-th entry
+  uint32_t pad;
 };
 
 // Threshold-bin history of one vector, kept across steps so that pass1 can mark candidates itself.
