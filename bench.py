@@ -313,6 +313,8 @@ def run_ours(args, wl):
             },
             "device_status": status,
         }
+        if args.dump_steps:
+            line["step_ms_all"] = [round(x, 4) for x in step_ms]
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = {k: v for k, v in time_oracle(wl, args.cpu_steps, 0).items() if k != "ms_per_step"}
         print(json.dumps(line), flush=True)
@@ -330,6 +332,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--dump-steps", action="store_true", help="add the per-step times to the JSON line")
     ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this d (profiling captures)")
     args = ap.parse_args()
     from paper_1905_05957_b200.workloads import WORKLOADS

@@ -52,9 +52,10 @@ struct TopkState {
   uint32_t pad;
 };
 
-// Threshold-bin history of one vector, kept across steps so that pass1 can mark candidates itself.
+// Threshold history of one vector (the keys tau of the two previous steps), kept across steps so
+// that pass1 can mark candidates itself.
 struct TopkPred {
-  uint32_t magic, tb_last, tb_prev, pad;
+  uint32_t magic, tau_last, tau_prev, pad;
 };
 
 // Carving of the workspace for `rows` simultaneous selections over d-vectors.
@@ -63,8 +64,9 @@ struct TopkPlan {
   uint32_t rows;
   uint64_t nseg;        // 32768-entry segments per vector
   uint64_t bm_stride;   // bitmap words per vector (whole segments)
-  uint64_t list_cap;    // capacity of the candidate-key list per vector (0: no list, gather instead)
-  uint64_t off_hist, off_list_count, off_state, off_bm_gt, off_bm_eq, off_seg, off_list;
+  uint64_t ntile;       // 4096-entry tiles per vector
+  uint64_t list_cap;    // slots of the candidate list per vector (0: no list, gather instead)
+  uint64_t off_hist, off_list_count, off_state, off_bm_gt, off_bm_eq, off_seg, off_list, off_tile_info, off_dense;
   uint64_t bytes;
   TopkPred* pred;       // [rows] history outside the scratch (device memory), or NULL: no prediction
 };

@@ -7,17 +7,18 @@
 // number r of entries equal to tau that still fit.  The top 12 key bits are the "bin".
 //
 // Pipeline with a candidate list (the library's normal path):
-//   pass1      v = source (Eq. 2 / Eq. 4), written over delta.  With a usable history of threshold
-//              bins it predicts a band [lo, hi] of bins for this step's threshold and, while v is
-//              still in registers, (a) sets a bit in the "kept" bitmap for every entry above the
-//              band, (b) appends (key, index) of every entry inside the band to a candidate list,
-//              (c) counts a 256-bin histogram of the entries from 16 bins below the band upwards.
-//   pick       threshold bin tb and the number of entries still to take inside it, from that
-//              partial histogram; accepts it only if the k-th entry lies inside the counted range
-//              and tb inside the band.
-//   hist, pick only after a miss (or without history): full 4096-bin histogram of v, exact tb
-//   mark       only after a miss: re-read v, rebuild bitmap and candidate list for the exact tb
-//   resolve    the next 12 and the last 7 key bits from the candidate list: tau and r
+//   pass1      v = source (Eq. 2 / Eq. 4), written over delta.  With the thresholds of the two
+//              previous steps it predicts a band of keys [lo, hi] around this step's threshold and,
+//              while v is still in registers, (a) sets a bit in the "kept" bitmap for every entry
+//              above the band and counts them, (b) writes (key, index) of every entry inside the
+//              band to the candidate list.  The list has one fixed region per 4096-entry tile
+//              (as many slots as the tile has entries), so no reservation between CTAs is needed.
+//   lhist 1    copies the tile regions into one dense list and counts the top 12 key bits on the
+//              way; accepts the prediction only if the k-th entry falls inside the list
+//              (kept < k <= kept + candidates)
+//   hist, pick only after a miss (or without history): full 4096-bin histogram of v, exact bin tb
+//   mark, compact  only after a miss: re-read v, rebuild bitmap and candidate list for the exact tb
+//   lhist 2,3  the next 12, then the last 7 key bits from the candidate list: tau and r
 //   classify   candidates with key > tau join the kept bitmap, key == tau go to the tie bitmap
 //   count, scan  per-segment population counts and their exclusive prefix
 //   emit       every set bit knows its output slot: write (index, value), zero the entry in delta
@@ -39,35 +40,36 @@ namespace dsq {
 namespace {
 
 constexpr uint32_t kBins1 = 4096;                  // key bits 30..19
-constexpr uint32_t kPartBins = 256;                // bins counted by a predicting pass1
-constexpr uint32_t kFloorMargin = 16;              // ... starting this many bins (one octave) below the band
 constexpr uint32_t kWordsPerThread = 4;            // count / emit / refine: bitmap words per thread
 constexpr uint32_t kSegWords = kThreads * kWordsPerThread;  // 1024 bitmap words per segment
 constexpr uint32_t kSegElems = kSegWords * 32;     // 32768 entries
 constexpr uint64_t kTile = 4096;                   // entries a CTA handles per loop trip
-constexpr uint32_t kWarpBuf = 256;                 // candidate staging entries per warp
 constexpr uint32_t kPredMagic = 0x70D1C7EDu;
+constexpr uint32_t kBandHalf = 1u << 16;           // half-width of the band in key units (0.5 % of magnitude)
+constexpr int kMaxTrend = 1 << 20;                 // largest step-to-step drift that is extrapolated (9 %)
 
 __device__ __forceinline__ uint32_t key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
 inline uint64_t round16(uint64_t b) { return (b + 15u) & ~uint64_t(15); }
 
-// Band of bins expected to contain this step's threshold bin: the last bin, moved by the last
-// change (thresholds drift while the error builds up), widened by one bin on each side.
-// Returns false when there is no usable history.
+// Keys are monotone in log-magnitude (2^23 units per octave), so a threshold that drifts by a
+// steady factor moves by a steady key difference.  The band is the last threshold, extrapolated by
+// the last change (the drift itself changes slowly), widened on both sides by the larger of a
+// quarter of that change and 0.5 % of magnitude.
+// Candidates are the entries with lo <= key <= hi; returns false when there is no usable history.
 __device__ __forceinline__ bool predicted_band(const TopkPred* pred, uint32_t row, uint32_t* lo, uint32_t* hi) {
   if (!pred) return false;
   const TopkPred p = pred[row];
-  if (p.magic != kPredMagic || p.tb_last >= kBins1 || p.tb_prev >= kBins1) return false;
-  int trend = (int)p.tb_last - (int)p.tb_prev;
-  trend = max(-2, min(3, trend));
-  const int c = (int)p.tb_last + trend;
-  *lo = (uint32_t)max(0, min((int)p.tb_last, c) - 1);
-  *hi = (uint32_t)min((int)kBins1 - 1, max((int)p.tb_last, c) + 1);
+  if (p.magic != kPredMagic || (p.tau_last | p.tau_prev) >> 31) return false;
+  long long trend = (long long)p.tau_last - (long long)p.tau_prev;
+  trend = max((long long)-kMaxTrend, min((long long)kMaxTrend, trend));
+  const long long c = (long long)p.tau_last + trend;
+  const long long half = max((long long)kBandHalf, (trend < 0 ? -trend : trend) / 4);
+  const long long l = min((long long)p.tau_last, c) - half, h = max((long long)p.tau_last, c) + half;
+  *lo = (uint32_t)max(0ll, l);
+  *hi = (uint32_t)min(0x7fffffffll, h);
   return true;
 }
-
-__device__ __forceinline__ uint32_t band_floor(uint32_t lo) { return lo > kFloorMargin ? lo - kFloorMargin : 0u; }
 
 // Eight neighbouring lanes each hold a 4-bit field for each of four rows; returns to lane
 // (octet base + r), r < 4, the 32-bit word of row r (fields in lane order).
@@ -88,149 +90,147 @@ __device__ __forceinline__ uint32_t octet_words4(const uint32_t (&nib)[4], uint3
   return u2 ? (recv2 | q << 16) : (q | recv2 << 16);
 }
 
-// Per-warp staging of candidate (key, index) pairs in shared memory.  Candidates are rare, so a
-// warp collects them over many tiles and reserves room in the vector's global list with one
-// atomic per flush; the order of the list is irrelevant (it is histogrammed and scattered).
-struct WarpStage {
-  uint2* buf;          // kWarpBuf entries of this warp (shared memory)
-  uint32_t count;      // warp-uniform
-  uint2* list;         // this vector's list
-  uint32_t* list_count;
-  uint64_t cap;
-
-  __device__ __forceinline__ void flush(uint32_t lane) {
-    if (!count) return;
-    uint32_t base = 0;
-    if (lane == 0) base = atomicAdd(list_count, count);
-    base = __shfl_sync(0xffffffffu, base, 0);
-    __syncwarp();
-    for (uint32_t i = lane; i < count; i += 32)
-      if ((uint64_t)base + i < cap) list[(uint64_t)base + i] = buf[i];
-    __syncwarp();
-    count = 0;
+// Writes the candidates of one tile -- sel[j] bit k flags entry k of row j, whose key is
+// keys[4 j + k] and whose index is idx0[j] + k -- into the tile's own region of the list (kTile slots, enough for every entry of
+// the tile).  Slots are handed out by a shared-memory counter, one atomic per warp; the order
+// inside the region is irrelevant.  Called by all 32 lanes of every warp of the CTA.
+__device__ __forceinline__ void tile_append(uint2* region, uint32_t* s_count, const uint32_t (&keys)[16],
+                                            const uint32_t (&idx0)[4], const uint32_t (&sel)[4], uint32_t lane) {
+  const uint32_t c = __popc(sel[0]) + __popc(sel[1]) + __popc(sel[2]) + __popc(sel[3]);
+  if (__ballot_sync(0xffffffffu, c != 0) == 0) return;
+  uint32_t incl = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= (uint32_t)o) incl += y;
   }
-
-  // sel[j] bit k flags entry k of row j, whose index is e[j] + k.  Called by all 32 lanes.
-  __device__ __forceinline__ void add(const float4 (&v)[4], const uint64_t (&e)[4], const uint32_t (&sel)[4],
-                                      uint32_t lane) {
-    const uint32_t c = __popc(sel[0]) + __popc(sel[1]) + __popc(sel[2]) + __popc(sel[3]);
-    if (__ballot_sync(0xffffffffu, c != 0) == 0) return;
-    uint32_t incl = c;
+  const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+  uint32_t base = 0;
+  if (lane == 0) base = atomicAdd(s_count, total);
+  base = __shfl_sync(0xffffffffu, base, 0);
+  uint32_t pos = base + incl - c;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= (uint32_t)o) incl += y;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);  // <= 512
-    if (count + total > kWarpBuf) flush(lane);
-    if (total > kWarpBuf) {
-      // a tile this dense goes straight to the list
-      uint32_t base = 0;
-      if (lane == 0) base = atomicAdd(list_count, total);
-      base = __shfl_sync(0xffffffffu, base, 0);
-      uint64_t pos = (uint64_t)base + incl - c;
+  for (int j = 0; j < 4; ++j)
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if ((sel[j] >> k) & 1u) {
-            if (pos < cap) list[pos] = make_uint2(key_of(compc(v[j], k)), (uint32_t)(e[j] + k));
-            ++pos;
-          }
-      return;
-    }
-    uint32_t pos = count + incl - c;
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if ((sel[j] >> k) & 1u) buf[pos++] = make_uint2(key_of(compc(v[j], k)), (uint32_t)(e[j] + k));
-    count += total;
-  }
-};
+    for (int k = 0; k < 4; ++k)
+      if ((sel[j] >> k) & 1u) {
+        if (pos < kTile) region[pos] = make_uint2(keys[4 * j + k], idx0[j] + k);
+        ++pos;
+      }
+}
 
 // ================================================================ list pipeline
 
 // ---------------------------------------------------------------- pass1
-// span: entries per CTA, a multiple of kTile.  `padded` = bitmap extent in entries (whole segments).
-template <int SRC>
-__global__ void __launch_bounds__(kThreads) k_topk_pass1(const SrcParams src, float* v_out, uint32_t* hist, uint64_t span,
-                                                         uint64_t padded, const TopkPred* pred, uint32_t* bm_gt,
-                                                         uint64_t bm_stride, uint2* list, uint32_t* list_count,
-                                                         uint64_t cap) {
-  __shared__ uint32_t s_hist[kPartBins];
-  __shared__ uint2 s_stage[(kThreads / 32) * kWarpBuf];
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
-  uint32_t lo = 1, hi = 0;
-  const bool marking = predicted_band(pred, row, &lo, &hi);
-  const uint32_t floor_bin = band_floor(lo);
-  // keys at the edges of the counted range and of the band; hi + 1 = 4096 gives 2^31, above every key
-  const uint32_t key_floor = floor_bin << 19, key_lo = lo << 19, key_above = (hi + 1u) << 19;
-  if (marking) {
-    for (uint32_t b = tid; b < kPartBins; b += kThreads) s_hist[b] = 0;
-    __syncthreads();
-  }
-  WarpStage stage;
-  stage.buf = s_stage + (tid >> 5) * kWarpBuf;
-  stage.count = 0;
-  stage.list = list + (uint64_t)row * cap;
-  stage.list_count = list_count + row;
-  stage.cap = cap;
+// One CTA per 4096-entry tile; the grid covers the padded bitmap extent.  tile_info[tile] receives
+// (candidates written, entries above the band).
+template <int SRC, bool FULL>
+__device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, uint64_t base, float* out_row, bool marking,
+                                           uint32_t key_lo, uint32_t key_hi, uint32_t* bm_row, uint2* region,
+                                           uint32_t* s_count, uint32_t* s_kept) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint64_t d = src.d;
-  const uint64_t begin = (uint64_t)blockIdx.x * span;
-  // when marking, the bitmap is written for whole segments, hence the padded end
-  const uint64_t end = min(begin + span, marking ? padded : d);
-  float* out_row = v_out + (uint64_t)row * d;
-  for (uint64_t base = begin; base < end; base += kTile) {
-    float4 v[4];
-    uint32_t cnt[4];
+  float4 v[4];
+  uint32_t cnt[4];
+  if constexpr (FULL && SRC == SRC_WORKER) {
+    const float4* gp = reinterpret_cast<const float4*>(src.g + (uint64_t)row * d + base) + tid;
+    const float4* dp = reinterpret_cast<const float4*>(src.delta + (uint64_t)row * d + base) + tid;
+    float4 a[4], b[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) a[j] = __ldcs(gp + j * kThreads);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) b[j] = __ldcs(dp + j * kThreads);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      cnt[j] = 4;
+      v[j] = make_float4(__fadd_rn(a[j].x, b[j].x), __fadd_rn(a[j].y, b[j].y), __fadd_rn(a[j].z, b[j].z),
+                         __fadd_rn(a[j].w, b[j].w));
+    }
+  } else {
     uint64_t ee[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       ee[j] = base + (uint64_t)(j * kThreads + tid) * 4u;
-      cnt[j] = ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u;
+      cnt[j] = FULL ? 4u : (ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u);
     }
     src_load_tile<SRC, 4>(src, row, ee, cnt, v);
+  }
+  if constexpr (FULL) {
+    float4* op = reinterpret_cast<float4*>(out_row + base) + tid;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) op[j * kThreads] = v[j];
+  } else {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
+      const uint64_t e = base + (uint64_t)(j * kThreads + tid) * 4u;
       if (cnt[j]) {
         if (src.vec && cnt[j] == 4) {
-          *reinterpret_cast<float4*>(out_row + ee[j]) = v[j];
+          *reinterpret_cast<float4*>(out_row + e) = v[j];
         } else {
-          for (uint32_t k = 0; k < cnt[j]; ++k) out_row[ee[j] + k] = compc(v[j], k);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if ((uint32_t)k < cnt[j]) out_row[e + k] = compc(v[j], k);
         }
       }
-    }
-    if (marking) {
-      uint32_t ngt[4], ncand[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        ngt[j] = 0;
-        ncand[j] = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint32_t key = key_of(compc(v[j], k));
-          if ((uint32_t)k < cnt[j] && key >= key_floor) {  // a few percent of the entries get here
-            atomicAdd(&s_hist[min((key >> 19) - floor_bin, kPartBins - 1u)], 1u);
-            if (key >= key_above) ngt[j] |= 1u << k;
-            else if (key >= key_lo) ncand[j] |= 1u << k;
-          }
-        }
-      }
-      const uint32_t wg = octet_words4(ngt, lane);
-      const uint32_t r = lane & 7u;
-      if (r < 4) bm_gt[(uint64_t)row * bm_stride + (base >> 5) + r * 32u + (tid >> 3)] = wg;
-      stage.add(v, ee, ncand, lane);
     }
   }
-  if (marking) {
-    stage.flush(lane);
-    __syncthreads();
-    uint32_t* h = hist + (uint64_t)row * kBins1 + floor_bin;
-    for (uint32_t b = tid; b < kPartBins; b += kThreads) {
-      const uint32_t c = s_hist[b];
-      if (c && floor_bin + b < kBins1) atomicAdd(&h[b], c);
+  if (!marking) return;
+  uint32_t ngt[4], ncand[4], idx0[4], keys[16];
+  uint32_t kept = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    ngt[j] = 0;
+    ncand[j] = 0;
+    idx0[j] = (uint32_t)base + (uint32_t)(j * kThreads + tid) * 4u;  // indices fit 32 bits: d < 2^32
+    keys[4 * j] = key_of(v[j].x); keys[4 * j + 1] = key_of(v[j].y);
+    keys[4 * j + 2] = key_of(v[j].z); keys[4 * j + 3] = key_of(v[j].w);
+    if (max(max(keys[4 * j], keys[4 * j + 1]), max(keys[4 * j + 2], keys[4 * j + 3])) >= key_lo) {
+      // only the kept entries and the candidates get in here
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (FULL || (uint32_t)k < cnt[j]) {  // entries past the end were loaded as +0 and are no entries
+          if (keys[4 * j + k] > key_hi) ngt[j] |= 1u << k;
+          else if (keys[4 * j + k] >= key_lo) ncand[j] |= 1u << k;
+        }
+      }
     }
+    kept += __popc(ngt[j]);
+  }
+  const uint32_t wg = octet_words4(ngt, lane);
+  const uint32_t r = lane & 7u;
+  if (r < 4) bm_row[(base >> 5) + r * 32u + (tid >> 3)] = wg;
+  tile_append(region, s_count, keys, idx0, ncand, lane);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
+  if (lane == 0 && kept) atomicAdd(s_kept, kept);
+}
+
+template <int SRC>
+__global__ void __launch_bounds__(kThreads) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred,
+                                                         uint32_t* bm_gt, uint64_t bm_stride, uint2* list, uint64_t cap,
+                                                         uint2* tile_info, uint64_t ntile) {
+  __shared__ uint32_t s_count, s_kept;
+  const uint32_t tid = threadIdx.x, row = blockIdx.y;
+  const uint64_t tile = blockIdx.x, base = tile * kTile;
+  const uint64_t d = src.d;
+  uint32_t key_lo = 1, key_hi = 0;
+  const bool marking = predicted_band(pred, row, &key_lo, &key_hi);
+  if (!marking && base >= d) return;  // padding tile and no bitmap to clear
+  if (marking) {
+    if (tid == 0) { s_count = 0; s_kept = 0; }
+    __syncthreads();
+  }
+  float* out_row = v_out + (uint64_t)row * d;
+  uint32_t* bm_row = bm_gt + (uint64_t)row * bm_stride;
+  uint2* region = list + (uint64_t)row * cap + base;
+  if (src.vec && base + kTile <= d) {
+    pass1_tile<SRC, true>(src, row, base, out_row, marking, key_lo, key_hi, bm_row, region, &s_count, &s_kept);
+  } else {
+    pass1_tile<SRC, false>(src, row, base, out_row, marking, key_lo, key_hi, bm_row, region, &s_count, &s_kept);
+  }
+  if (marking && base < d) {
+    __syncthreads();
+    if (tid == 0) tile_info[(uint64_t)row * ntile + tile] = make_uint2(min(s_count, (uint32_t)kTile), s_kept);
   }
 }
 
@@ -280,59 +280,21 @@ __device__ __forceinline__ void cta_pick(const uint32_t* h, uint32_t want, uint3
   __syncthreads();
 }
 
-__device__ __forceinline__ void remember_bin(TopkPred* pred, uint32_t row, uint32_t tb, bool had) {
-  if (!pred) return;
-  TopkPred np;
-  np.magic = kPredMagic;
-  np.tb_prev = had ? pred[row].tb_last : tb;
-  np.tb_last = tb;
-  np.pad = 0;
-  pred[row] = np;
-}
-
-// Level-1 pick, one CTA per vector.  full = 0: judge the partial histogram of a predicting pass1.
-// full = 1: runs after k_topk_hist; does something only for vectors that missed.
-__global__ void __launch_bounds__(1024) k_topk_pick1(uint32_t* hist, TopkState* state, uint32_t k, TopkPred* pred,
-                                                     uint32_t* list_count, int full) {
+// Level-1 pick after a miss, one CTA per vector, on the full histogram written by k_topk_hist.
+__global__ void __launch_bounds__(1024) k_topk_pick1(uint32_t* hist, TopkState* state, uint32_t k) {
   __shared__ uint32_t s_warp[32], s_out[3];
   const uint32_t tid = threadIdx.x, row = blockIdx.x;
   uint32_t* h = hist + (uint64_t)row * kBins1;
   TopkState* st = state + row;
-  if (full && !st->need_full) return;
-  uint32_t lo = 1, hi = 0;
-  const bool had = predicted_band(pred, row, &lo, &hi);
-  if (!full && !had) {  // nothing was counted
-    if (tid == 0) { st->need_full = 1; st->need_mark = 1; if (list_count) list_count[row] = 0; }
-    return;
-  }
+  if (!st->need_full) return;
   if (tid == 0) { s_out[0] = 0; s_out[1] = 0; s_out[2] = 0; }
   __syncthreads();
   cta_pick(h, k, s_warp, s_out);
   for (uint32_t b = tid; b < kBins1; b += 1024) h[b] = 0;
   if (tid != 0) return;
-  const uint32_t tb = s_out[0], rem = s_out[1], total = s_out[2];
-  if (full) {
-    st->tb1 = tb;
-    st->k_rem = rem;
-    st->need_mark = 1;
-    remember_bin(pred, row, tb, had);
-    return;
-  }
-  // the partial histogram is trustworthy if the k-th entry lies inside the counted range, below
-  // its clamped top bin, and the bitmap and list were built for a band that contains its bin
-  const uint32_t floor_bin = band_floor(lo);
-  const bool hit = total >= k && tb < floor_bin + kPartBins - 1u && tb >= lo && tb <= hi;
-  if (hit) {
-    st->tb1 = tb;
-    st->k_rem = rem;
-    st->need_full = 0;
-    st->need_mark = 0;
-    remember_bin(pred, row, tb, true);
-  } else {
-    st->need_full = 1;
-    st->need_mark = 1;
-    if (list_count) list_count[row] = 0;  // mark will list the candidates afresh
-  }
+  st->tb1 = s_out[0];
+  st->k_rem = s_out[1];
+  st->need_mark = 1;
 }
 
 // ---------------------------------------------------------------- full histogram (after a miss)
@@ -355,7 +317,9 @@ __global__ void __launch_bounds__(kThreads) k_topk_hist(const float* v_in, uint6
       if (vec && cnt == 4) {
         v = *reinterpret_cast<const float4*>(vrow + e);
       } else {
-        for (uint32_t k = 0; k < cnt; ++k) comp(v, k) = vrow[e + k];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)k < cnt) comp(v, k) = vrow[e + k];
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k)
@@ -371,48 +335,49 @@ __global__ void __launch_bounds__(kThreads) k_topk_hist(const float* v_in, uint6
 }
 
 // ---------------------------------------------------------------- mark (after a miss)
-// Bitmap of the entries above the exact threshold bin and the list of those inside it.  One tile
-// per loop trip over a small grid; every bitmap word up to the padded end is written.
+// Bitmap of the entries above the exact threshold bin and the list of those inside it.  A small
+// grid strides over the tiles; every bitmap word up to the padded end is written.
 __global__ void __launch_bounds__(kThreads) k_topk_mark(const float* v_in, uint64_t d, int vec, const TopkState* state,
                                                         uint32_t* bm_gt, uint64_t bm_stride, uint64_t padded, uint2* list,
-                                                        uint32_t* list_count, uint64_t cap) {
-  __shared__ uint2 s_stage[(kThreads / 32) * kWarpBuf];
+                                                        uint64_t cap, uint2* tile_info, uint64_t ntile) {
+  __shared__ uint32_t s_count;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   if (!state[row].need_mark) return;
   const uint32_t tb = state[row].tb1;
   const float* vrow = v_in + (uint64_t)row * d;
-  WarpStage stage;
-  stage.buf = s_stage + (tid >> 5) * kWarpBuf;
-  stage.count = 0;
-  stage.list = list + (uint64_t)row * cap;
-  stage.list_count = list_count + row;
-  stage.cap = cap;
-  const uint64_t ntile = padded / kTile;
-  for (uint64_t tile = blockIdx.x; tile < ntile; tile += gridDim.x) {
+  const uint64_t tiles = padded / kTile;
+  for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const uint64_t base = tile * kTile;
+    if (tid == 0) s_count = 0;
+    __syncthreads();
     float4 v[4];
-    uint32_t cnt[4];
-    uint64_t ee[4];
+    uint32_t cnt[4], idx0[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      ee[j] = tile * kTile + (uint64_t)(j * kThreads + tid) * 4u;
-      cnt[j] = ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u;
+      const uint64_t e = base + (uint64_t)(j * kThreads + tid) * 4u;
+      idx0[j] = (uint32_t)e;
+      cnt[j] = e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u;
       v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (cnt[j]) {
         if (vec && cnt[j] == 4) {
-          v[j] = *reinterpret_cast<const float4*>(vrow + ee[j]);
+          v[j] = *reinterpret_cast<const float4*>(vrow + e);
         } else {
-          for (uint32_t k = 0; k < cnt[j]; ++k) comp(v[j], k) = vrow[ee[j] + k];
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if ((uint32_t)k < cnt[j]) comp(v[j], k) = vrow[e + k];
         }
       }
     }
-    uint32_t ngt[4], ncand[4];
+    uint32_t ngt[4], ncand[4], keys[16];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       ngt[j] = 0;
       ncand[j] = 0;
+      keys[4 * j] = key_of(v[j].x); keys[4 * j + 1] = key_of(v[j].y);
+      keys[4 * j + 2] = key_of(v[j].z); keys[4 * j + 3] = key_of(v[j].w);
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const uint32_t bin = key_of(compc(v[j], k)) >> 19;
+        const uint32_t bin = keys[4 * j + k] >> 19;
         const bool in = (uint32_t)k < cnt[j];
         ngt[j] |= (in && bin > tb ? 1u : 0u) << k;
         ncand[j] |= (in && bin == tb ? 1u : 0u) << k;
@@ -421,62 +386,178 @@ __global__ void __launch_bounds__(kThreads) k_topk_mark(const float* v_in, uint6
     const uint32_t wg = octet_words4(ngt, lane);
     const uint32_t r = lane & 7u;
     if (r < 4) bm_gt[(uint64_t)row * bm_stride + tile * (kTile / 32) + r * 32u + (tid >> 3)] = wg;
-    stage.add(v, ee, ncand, lane);
+    if (base < d) tile_append(list + (uint64_t)row * cap + base, &s_count, keys, idx0, ncand, lane);
+    __syncthreads();
+    if (tid == 0 && base < d) tile_info[(uint64_t)row * ntile + tile] = make_uint2(min(s_count, (uint32_t)kTile), 0u);
   }
-  stage.flush(lane);
 }
 
-// ---------------------------------------------------------------- resolve
-// One CTA per vector: the second and third radix digits from the candidate list.
-__global__ void __launch_bounds__(1024) k_topk_resolve(const uint2* list, const uint32_t* list_count, uint64_t cap,
-                                                       TopkState* state) {
+// ---------------------------------------------------------------- tile regions -> dense list
+// Copies the candidates out of the per-tile regions into one dense list per vector (order
+// irrelevant).  A warp takes eight tiles at a time: one read of their counts, one reservation in
+// the dense list for all eight, then the regions.  With HIST the top-12-bit histogram of the keys
+// is counted on the way (into s_hist) and the return value is this thread's share of the
+// "entries above the band" counts.  Called by whole CTAs.
+template <bool HIST>
+__device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint2* info, uint64_t ntile, uint2* drow,
+                                                 uint32_t* dense_count, uint32_t* s_hist) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  const uint32_t warps = blockDim.x >> 5;
+  uint32_t kept = 0;
+  const uint64_t wstep = (uint64_t)gridDim.x * warps * 8;
+  for (uint64_t t0 = ((uint64_t)blockIdx.x * warps + (tid >> 5)) * 8; t0 < ntile; t0 += wstep) {
+    uint2 mine = make_uint2(0, 0);
+    if (lane < 8 && t0 + lane < ntile) mine = info[t0 + lane];
+    mine.x = min(mine.x, (uint32_t)kTile);
+    kept += mine.y;
+    uint32_t incl = mine.x;
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= (uint32_t)o) incl += y;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 7);
+    if (total == 0) continue;
+    uint32_t base = 0;
+    if (lane == 0) base = atomicAdd(dense_count, total);
+    base = __shfl_sync(0xffffffffu, base, 0);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint32_t n = __shfl_sync(0xffffffffu, mine.x, u);
+      const uint32_t off = __shfl_sync(0xffffffffu, incl - mine.x, u);
+      const uint2* reg = lrow + (t0 + u) * kTile;
+      for (uint32_t i = lane; i < n; i += 32) {
+        const uint2 e = reg[i];
+        drow[(uint64_t)base + off + i] = e;
+        if (HIST) atomicAdd(&s_hist[(e.x >> 19) & 0xFFFu], 1u);
+      }
+    }
+  }
+  return kept;
+}
+
+// After a miss: the list that mark rebuilt, made dense.
+__global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, uint64_t cap, const uint2* tile_info,
+                                                           uint64_t ntile, uint2* dense, uint32_t* dense_count,
+                                                           const TopkState* state) {
+  const uint32_t row = blockIdx.y;
+  if (!state[row].need_mark) return;
+  gather_tiles<false>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile, dense + (uint64_t)row * cap,
+                      &dense_count[row], nullptr);
+}
+
+// ---------------------------------------------------------------- list histogram + pick
+// One radix digit from the candidate list: LEVEL 1 = key bits 30..19 (and the verdict on the
+// prediction), LEVEL 2 = bits 18..7, LEVEL 3 = bits 6..0 (tau and r complete; tau is remembered
+// for the next step's prediction).  Several CTAs per vector histogram slices of the list into the
+// vector's global histogram; the CTA that finishes last (a ticket counter, no waiting) picks the
+// digit and clears histogram and ticket.
+template <int LEVEL>
+__global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t cap, const uint2* tile_info, uint64_t ntile,
+                                                     uint2* dense, uint32_t* dense_count, uint32_t* kept_count,
+                                                     TopkState* state, uint32_t* hist, uint32_t* done, uint32_t k,
+                                                     TopkPred* pred) {
   __shared__ uint32_t s_hist[kBins1];
   __shared__ uint32_t s_warp[32], s_out[3];
-  const uint32_t tid = threadIdx.x, row = blockIdx.x;
+  __shared__ uint32_t s_last;
+  constexpr uint32_t NB = LEVEL == 3 ? 128u : 4096u;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   const uint2* lrow = list + (uint64_t)row * cap;
-  const uint64_t n = min((uint64_t)list_count[row], cap);
+  const uint2* info = tile_info + (uint64_t)row * ntile;
   TopkState* st = state + row;
-  const uint32_t tb1 = st->tb1, want = st->k_rem;
-  for (uint32_t b = tid; b < kBins1; b += 1024) s_hist[b] = 0;
-  if (tid == 0) { s_out[0] = 0; s_out[1] = 0; }
+  uint32_t band_lo = 1, band_hi = 0;
+  // LEVEL 1 reads what pass1 wrote, which exists only if pass1 had a band to work with
+  const bool readable = LEVEL != 1 || predicted_band(pred, row, &band_lo, &band_hi);
+  const uint32_t tb1 = st->tb1, top24 = (st->tb1 << 12) | st->tb2;
+  for (uint32_t b = tid; b < NB; b += 1024) s_hist[b] = 0;
   __syncthreads();
-  for (uint64_t i0 = 0; i0 < n; i0 += 8 * 1024) {
-    uint32_t key[8];
+  uint32_t kept = 0;
+  if (LEVEL == 1) {
+    if (readable) kept = gather_tiles<true>(lrow, info, ntile, dense + (uint64_t)row * cap, &dense_count[row], s_hist);
+  } else {
+    const uint2* drow = dense + (uint64_t)row * cap;
+    const uint64_t n = min((uint64_t)dense_count[row], cap);
+    const uint64_t step = (uint64_t)gridDim.x * 8 * 1024;
+    for (uint64_t i0 = (uint64_t)blockIdx.x * 8 * 1024; i0 < n; i0 += step) {
+      uint32_t key[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const uint64_t i = i0 + (uint64_t)u * 1024 + tid;
-      key[u] = i < n ? lrow[i].x : 0xFFFFFFFFu;  // bin 8191: never equal to tb1
+      for (int u = 0; u < 8; ++u) {
+        const uint64_t i = i0 + (uint64_t)u * 1024 + tid;
+        key[u] = i < n ? drow[i].x : 0xFFFFFFFFu;  // bit 31 set: matches no bin and no prefix
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (LEVEL == 2) {
+          if ((key[u] >> 19) == tb1) atomicAdd(&s_hist[(key[u] >> 7) & 0xFFFu], 1u);
+        } else {
+          if ((key[u] >> 7) == top24) atomicAdd(&s_hist[key[u] & 0x7Fu], 1u);
+        }
+      }
     }
-#pragma unroll
-    for (int u = 0; u < 8; ++u)
-      if ((key[u] >> 19) == tb1) atomicAdd(&s_hist[(key[u] >> 7) & 0xFFFu], 1u);
   }
+  if (LEVEL == 1) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
+    if (lane == 0 && kept) atomicAdd(&kept_count[row], kept);
+  }
+  __syncthreads();
+  uint32_t* h = hist + (uint64_t)row * kBins1;
+  for (uint32_t b = tid; b < NB; b += 1024) {
+    const uint32_t c = s_hist[b];
+    if (c) atomicAdd(&h[b], c);
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&done[row], 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // every CTA of this vector has flushed: read the complete histogram past L1, pick, clear
+  for (uint32_t b = tid; b < kBins1; b += 1024) {
+    s_hist[b] = b < NB ? __ldcg(&h[b]) : 0u;
+    if (b < NB) h[b] = 0;
+  }
+  uint32_t want = st->k_rem;
+  if (LEVEL == 1) {
+    const uint32_t kept = __ldcg(&kept_count[row]);
+    want = kept < k ? k - kept : 0u;  // 0: the threshold lies above the band
+  }
+  if (tid == 0) { s_out[0] = 0; s_out[1] = 0; s_out[2] = 0; done[row] = 0; }
   __syncthreads();
   cta_pick(s_hist, want, s_warp, s_out);
-  const uint32_t tb2 = s_out[0], rem2 = s_out[1];
-  __syncthreads();
-  for (uint32_t b = tid; b < kBins1; b += 1024) s_hist[b] = 0;
-  if (tid == 0) { s_out[0] = 0; s_out[1] = 0; }
-  __syncthreads();
-  const uint32_t top24 = (tb1 << 12) | tb2;
-  for (uint64_t i0 = 0; i0 < n; i0 += 8 * 1024) {
-    uint32_t key[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const uint64_t i = i0 + (uint64_t)u * 1024 + tid;
-      key[u] = i < n ? lrow[i].x : 0xFFFFFFFFu;
+  if (tid != 0) return;
+  if (LEVEL == 1) {
+    // the prediction holds iff the k-th largest entry is one of the listed candidates
+    uint32_t lo = 1, hi = 0;
+    const bool hit = predicted_band(pred, row, &lo, &hi) && want >= 1 && want <= s_out[2];
+    if (hit) {
+      st->tb1 = s_out[0];
+      st->k_rem = s_out[1];
+      st->need_full = 0;
+      st->need_mark = 0;
+    } else {
+      st->need_full = 1;  // hist, pick, mark and compact rebuild bitmap and list for the exact bin
+      st->need_mark = 1;
+      dense_count[row] = 0;
     }
-#pragma unroll
-    for (int u = 0; u < 8; ++u)
-      if ((key[u] >> 7) == top24) atomicAdd(&s_hist[key[u] & 0x7Fu], 1u);
-  }
-  __syncthreads();
-  cta_pick(s_hist, rem2, s_warp, s_out);
-  if (tid == 0) {
-    st->tb2 = tb2;
-    st->tau = (top24 << 7) | s_out[0];
+  } else if (LEVEL == 2) {
+    st->tb2 = s_out[0];
+    st->k_rem = s_out[1];
+  } else {
+    const uint32_t tau = (top24 << 7) | s_out[0];
+    st->tau = tau;
     st->r = s_out[1];
     st->k_rem = s_out[1];
+    if (pred) {
+      uint32_t lo = 1, hi = 0;
+      const bool had = predicted_band(pred, row, &lo, &hi);
+      TopkPred np;
+      np.magic = kPredMagic;
+      np.tau_prev = had ? pred[row].tau_last : tau;
+      np.tau_last = tau;
+      np.pad = 0;
+      pred[row] = np;
+    }
   }
 }
 
@@ -484,19 +565,29 @@ __global__ void __launch_bounds__(1024) k_topk_resolve(const uint2* list, const 
 // Candidates above tau join the kept bitmap; candidates equal to tau are set in the tie bitmap
 // (which the launcher cleared).  Candidate bits are never set in bm_gt beforehand, so the ORs
 // commute with nothing else.
-__global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* list, const uint32_t* list_count, uint64_t cap,
+__global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* dense, const uint32_t* dense_count, uint64_t cap,
                                                             const TopkState* state, uint32_t* bm_gt, uint32_t* bm_tie,
                                                             uint64_t bm_stride) {
   const uint32_t row = blockIdx.y;
-  const uint2* lrow = list + (uint64_t)row * cap;
-  const uint64_t n = min((uint64_t)list_count[row], cap);
+  const uint2* drow = dense + (uint64_t)row * cap;
+  const uint64_t n = min((uint64_t)dense_count[row], cap);
   const uint32_t tau = state[row].tau;
   uint32_t* g = bm_gt + (uint64_t)row * bm_stride;
   uint32_t* t = bm_tie + (uint64_t)row * bm_stride;
-  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (uint64_t)gridDim.x * kThreads) {
-    const uint2 e = lrow[i];
-    if (e.x > tau) atomicOr(&g[e.y >> 5], 1u << (e.y & 31u));
-    else if (e.x == tau) atomicOr(&t[e.y >> 5], 1u << (e.y & 31u));
+  const uint64_t step = (uint64_t)gridDim.x * kThreads * 4;
+  for (uint64_t i0 = (uint64_t)blockIdx.x * kThreads * 4 + threadIdx.x; i0 < n; i0 += step) {
+    uint2 e[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = i0 + (uint64_t)u * kThreads;
+      e[u] = i < n ? drow[i] : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (i0 + (uint64_t)u * kThreads >= n) continue;
+      if (e[u].x > tau) atomicOr(&g[e[u].y >> 5], 1u << (e[u].y & 31u));
+      else if (e[u].x == tau) atomicOr(&t[e[u].y >> 5], 1u << (e[u].y & 31u));
+    }
   }
 }
 
@@ -555,7 +646,9 @@ __global__ void __launch_bounds__(kThreads) k_topk_pass1_basic(const SrcParams s
       if (src.vec && cnt[j] == 4) {
         *reinterpret_cast<float4*>(out_row + ee[j]) = v[j];
       } else {
-        for (uint32_t k = 0; k < cnt[j]; ++k) out_row[ee[j] + k] = compc(v[j], k);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)k < cnt[j]) out_row[ee[j] + k] = compc(v[j], k);
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k)
@@ -616,7 +709,9 @@ __global__ void __launch_bounds__(kThreads) k_topk_mark_basic(const float* v_in,
         if (vec && cnt == 4) {
           v = *reinterpret_cast<const float4*>(vrow + e);
         } else {
-          for (uint32_t k = 0; k < cnt; ++k) comp(v, k) = vrow[e + k];
+  #pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)k < cnt) comp(v, k) = vrow[e + k];
         }
       }
       ngt[j] = 0;
@@ -815,30 +910,59 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(payload + (uint64_t)row * payload_stride + off_idx);
   float* out_val = reinterpret_cast<float*>(payload + (uint64_t)row * payload_stride + off_val);
   float* vrow = v_io + (uint64_t)row * d;
+  // which bits of each word are emitted, and the output slot of the first of them
+  uint32_t selw[4], posw[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    if (cw[i]) {
-      const uint32_t ties_before = pre.y + (excl >> 16);
-      uint32_t keep = tie[i];
-      const uint32_t room = r > ties_before ? r - ties_before : 0u;
-      while ((uint32_t)__popc(keep) > room) keep &= ~(0x80000000u >> __clz(keep));  // drop the highest tie
-      uint32_t sel = gt[i] | keep;
-      uint32_t pos = pre.x + (excl & 0xFFFFu) + min(ties_before, r);
-      while (sel) {
-        const uint32_t b = __ffs(sel) - 1u;
-        sel &= sel - 1u;
-        const uint64_t j = (widx + i) * 32u + b;
-        const float val = vrow[j];
-        if (pos < k) {  // always true when the counts are consistent; keeps a bad count inside the payload
-          out_idx[pos] = (uint32_t)j;
-          out_val[pos] = val;
-        }
-        vrow[j] = 0.f;  // delta = v - Q[v] at a kept entry
-        if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
-        ++pos;
-      }
-    }
+    const uint32_t ties_before = pre.y + (excl >> 16);
+    uint32_t keep = tie[i];
+    const uint32_t room = r > ties_before ? r - ties_before : 0u;
+    while ((uint32_t)__popc(keep) > room) keep &= ~(0x80000000u >> __clz(keep));  // drop the highest tie
+    selw[i] = gt[i] | keep;
+    posw[i] = pre.x + (excl & 0xFFFFu) + min(ties_before, r);
     excl += cw[i];
+  }
+  // the first two kept entries of every word are fetched before anything is stored, so that a
+  // thread has up to eight gathers in flight; words with more (rare) finish in the loop below
+  uint32_t b0[4], b1[4];
+  float v0[4], v1[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t s0 = selw[i], s1 = s0 & (s0 - 1u);
+    b0[i] = s0 ? __ffs(s0) - 1u : 32u;
+    b1[i] = s1 ? __ffs(s1) - 1u : 32u;
+    v0[i] = b0[i] < 32u ? vrow[(widx + i) * 32u + b0[i]] : 0.f;
+    v1[i] = b1[i] < 32u ? vrow[(widx + i) * 32u + b1[i]] : 0.f;
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t pos = posw[i];
+    if (b0[i] < 32u) {
+      const uint64_t j = (widx + i) * 32u + b0[i];
+      if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v0[i]; }  // pos < k whenever the counts are consistent
+      vrow[j] = 0.f;                                                      // delta = v - Q[v] at a kept entry
+      if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v0[i]));
+      ++pos;
+    }
+    if (b1[i] < 32u) {
+      const uint64_t j = (widx + i) * 32u + b1[i];
+      if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v1[i]; }
+      vrow[j] = 0.f;
+      if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v1[i]));
+      ++pos;
+    }
+    uint32_t sel = selw[i] & (selw[i] - 1u);
+    sel &= sel - 1u;  // the entries after the first two
+    while (sel) {
+      const uint32_t b = __ffs(sel) - 1u;
+      sel &= sel - 1u;
+      const uint64_t j = (widx + i) * 32u + b;
+      const float val = vrow[j];
+      if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = val; }
+      vrow[j] = 0.f;
+      if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
+      ++pos;
+    }
   }
 }
 
@@ -851,15 +975,18 @@ void topk_plan(uint64_t d, uint32_t rows, uint64_t k, bool with_list, TopkPlan* 
   const uint64_t nw = (d + 31) / 32;
   p->nseg = (nw + kSegWords - 1) / kSegWords;
   p->bm_stride = p->nseg * kSegWords;
-  p->list_cap = with_list ? d : 0;
+  p->ntile = (d + kTile - 1) / kTile;
+  p->list_cap = with_list ? p->ntile * kTile : 0;  // one kTile-slot region per tile
   uint64_t pos = 0;
   p->off_hist = pos;       pos += (uint64_t)rows * kBins1 * 4;      // histogram and list counters are
-  p->off_list_count = pos; pos = round16(pos + (uint64_t)rows * 4);  // cleared by one memset
+  p->off_list_count = pos; pos = round16(pos + (uint64_t)rows * 12);  // tickets, kept counts: cleared by one memset
   p->off_state = pos;      pos = round16(pos + (uint64_t)rows * sizeof(TopkState));
   p->off_bm_gt = pos;      pos = round16(pos + (uint64_t)rows * p->bm_stride * 4);
   p->off_bm_eq = pos;      pos = round16(pos + (uint64_t)rows * p->bm_stride * 4);
   p->off_seg = pos;        pos = round16(pos + (uint64_t)rows * p->nseg * sizeof(uint2));
   p->off_list = pos;       pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint2));
+  p->off_tile_info = pos;  pos = round16(pos + (with_list ? (uint64_t)rows * p->ntile * sizeof(uint2) : 0));
+  p->off_dense = pos;      pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint2));
   p->bytes = pos;
   p->pred = nullptr;
 }
@@ -874,15 +1001,22 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   uint32_t* bm_eq = reinterpret_cast<uint32_t*>(ws + pl.off_bm_eq);  // candidates (no list) / ties
   uint2* seg = reinterpret_cast<uint2*>(ws + pl.off_seg);
   uint2* list = pl.list_cap ? reinterpret_cast<uint2*>(ws + pl.off_list) : nullptr;
+  uint2* tile_info = reinterpret_cast<uint2*>(ws + pl.off_tile_info);
+  uint2* dense = reinterpret_cast<uint2*>(ws + pl.off_dense);
   const uint64_t d = src.d, cap = pl.list_cap;
   const uint64_t padded = pl.nseg * (uint64_t)kSegElems;
-  cudaError_t e = cudaMemsetAsync(hist, 0, (uint64_t)rows * kBins1 * 4 + (uint64_t)rows * 4, st);
+  uint32_t* done = list_count + rows;        // ticket counters of the list histograms
+  uint32_t* kept_count = list_count + 2 * rows;  // entries above the predicted band
+  cudaError_t e = cudaMemsetAsync(hist, 0, (uint64_t)rows * kBins1 * 4 + (uint64_t)rows * 12, st);
   if (e != cudaSuccess) return e;
 
-  // entries per CTA of pass1: enough CTAs to fill the GPU several times over
+  // pass1: one CTA per tile of the padded extent
+  const uint64_t ntile_padded = padded / kTile;
+  dim3 g1((unsigned)ntile_padded, rows, 1);
+  // pass1 without a list keeps its span form
   uint64_t span = 16 * kTile;
   while (span > kTile && ((padded + span - 1) / span) * rows < 148ull * 16ull) span /= 2;
-  dim3 g1((unsigned)((padded + span - 1) / span), rows, 1);
+  dim3 g1b((unsigned)((padded + span - 1) / span), rows, 1);
   const uint32_t k32 = (uint32_t)k;
   dim3 gs((unsigned)pl.nseg, rows, 1);
   // kernels that re-read a whole vector after a miss: a grid that fills the GPU and strides over tiles
@@ -894,8 +1028,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   if (list && k) {
     TopkPred* pred = pl.pred;
 #define DSQ_P1(S)                                                                                                 \
-  k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, hist, span, padded, pred, bm_gt, pl.bm_stride, list, \
-                                           list_count, cap)
+  k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, pred, bm_gt, pl.bm_stride, list, cap, tile_info, pl.ntile)
     switch (srck) {
       case SRC_WORKER: DSQ_P1(SRC_WORKER); break;
       case SRC_SRV_IDENTITY: DSQ_P1(SRC_SRV_IDENTITY); break;
@@ -907,17 +1040,24 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
 #undef DSQ_P1
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(bm_eq, 0, (uint64_t)rows * pl.bm_stride * 4, st)) != cudaSuccess) return e;  // tie bitmap
-    k_topk_pick1<<<rows, 1024, 0, st>>>(hist, state, k32, pred, list_count, 0);
+    dim3 gl((unsigned)(148ull * 2ull / rows ? 148ull * 2ull / rows : 1), rows, 1);
+    k_topk_lhist<1><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+                                         k32, pred);
     k_topk_hist<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, hist);
-    k_topk_pick1<<<rows, 1024, 0, st>>>(hist, state, k32, pred, list_count, 1);
-    k_topk_mark<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, bm_gt, pl.bm_stride, padded, list, list_count, cap);
-    k_topk_resolve<<<rows, 1024, 0, st>>>(list, list_count, cap, state);
+    k_topk_pick1<<<rows, 1024, 0, st>>>(hist, state, k32);
+    k_topk_mark<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, bm_gt, pl.bm_stride, padded, list, cap, tile_info,
+                                         pl.ntile);
+    k_topk_compact<<<gm, kThreads, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, state);
+    k_topk_lhist<2><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+                                         k32, pred);
+    k_topk_lhist<3><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+                                         k32, pred);
     dim3 gc((unsigned)(148ull * 8ull / rows ? 148ull * 8ull / rows : 1), rows, 1);
-    k_topk_classify<<<gc, kThreads, 0, st>>>(list, list_count, cap, state, bm_gt, bm_eq, pl.bm_stride);
+    k_topk_classify<<<gc, kThreads, 0, st>>>(dense, list_count, cap, state, bm_gt, bm_eq, pl.bm_stride);
     k_topk_count<<<gs, kThreads, 0, st>>>(bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
-    count_launches(8);
+    count_launches(11);
   } else {
-#define DSQ_P1(S) k_topk_pass1_basic<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, hist, span)
+#define DSQ_P1(S) k_topk_pass1_basic<S><<<g1b, kThreads, 0, st>>>(src, io.v_inout, hist, span)
     switch (srck) {
       case SRC_WORKER: DSQ_P1(SRC_WORKER); break;
       case SRC_SRV_IDENTITY: DSQ_P1(SRC_SRV_IDENTITY); break;
