@@ -276,13 +276,9 @@ int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, voi
     // (1/n) sum_i Q[v_i] for sparse payloads: dense accumulator, workers added in order 0..n-1
     cudaError_t e = cudaMemsetAsync(h->acc, 0, h->cfg.d * 4, st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-    const uint8_t* wp = static_cast<const uint8_t*>(h->buf.worker_payload);
-    for (uint32_t i = 0; i < h->cfg.n; ++i) {
-      const uint8_t* pl = wp + (uint64_t)i * h->wl.stride;
-      e = launch_sparse_accumulate(reinterpret_cast<const uint32_t*>(pl + h->wl.off[0]),
-                                   reinterpret_cast<const float*>(pl + h->wl.off[1]), h->cfg.worker_q.k, h->acc, st);
-      if (e != cudaSuccess) return cuda_fail(e, "sparse accumulate");
-    }
+    e = launch_sparse_accumulate(static_cast<const uint8_t*>(h->buf.worker_payload), h->wl.stride, h->wl.off[0], h->wl.off[1],
+                                 h->cfg.n, h->cfg.worker_q.k, h->cfg.d, h->acc, st);
+    if (e != cudaSuccess) return cuda_fail(e, "sparse accumulate");
   }
   const bool fuse = (flags & DS_FUSE_APPLY) != 0;
   const int rc = run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload),

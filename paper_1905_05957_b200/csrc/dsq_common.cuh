@@ -29,7 +29,7 @@ struct SrcParams {
   uint64_t wp_off[3];      // sub-array offsets inside a payload
   uint32_t w_log2_chunk;   // worker chunk length (SIGN1, QSGD)
   float w_levels;          // worker QSGD level count as a float
-  float* acc;              // SRC_SRV_TOPK: dense accumulator [d]; cleared as it is consumed
+  const float* acc;        // SRC_SRV_TOPK: dense accumulator [d] holding the sum of the sparse payloads
   int vec;                 // 1 if every row starts 16-byte aligned (d % 4 == 0)
 };
 
@@ -167,12 +167,9 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
           }
         }
       }
-    } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc; consume and clear it
+    } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc (cleared before every use)
 #pragma unroll
-      for (int j = 0; j < V; ++j) {
-        acc[j] = load_row4(p.acc, e[j], cnt[j], p.vec);
-        store_row4(p.acc, e[j], cnt[j], p.vec, make_float4(0.f, 0.f, 0.f, 0.f));
-      }
+      for (int j = 0; j < V; ++j) acc[j] = load_row4(p.acc, e[j], cnt[j], p.vec);
     }
 #pragma unroll
     for (int j = 0; j < V; ++j) {

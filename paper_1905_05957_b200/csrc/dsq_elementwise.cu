@@ -106,20 +106,53 @@ cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamm
   return cudaGetLastError();
 }
 
-// acc[idx[m]] = acc[idx[m]] + val[m].  Indices inside one payload are distinct, so there is no
-// conflict; the launches for workers 0..n-1 are issued in that order on one stream, which makes
-// the sum over workers sequential in worker order as Eq. 4 is evaluated.
-__global__ void __launch_bounds__(kThreads) k_sparse_accumulate(const uint32_t* __restrict__ idx,
-                                                                const float* __restrict__ val, uint64_t k, float* acc) {
-  for (uint64_t m = (uint64_t)blockIdx.x * kThreads + threadIdx.x; m < k; m += (uint64_t)gridDim.x * kThreads) {
-    const uint32_t j = idx[m];
-    acc[j] = __fadd_rn(acc[j], val[m]);
+// Sum of the n sparse worker payloads into the dense accumulator, workers added in order
+// 0..n-1 as Eq. 4 is evaluated.  A CTA owns a span of indices: it first finds, for up to 128
+// workers at a time, where that span begins and ends in each worker's ascending index list
+// (binary searches, all in parallel), then walks the workers in order with a barrier in between.
+// Indices inside one payload are distinct, so the additions of one worker never collide, and no
+// other CTA touches this span.
+constexpr uint32_t kAccSpan = 8192;
+
+__global__ void __launch_bounds__(kThreads) k_sparse_accumulate_all(const uint8_t* __restrict__ wp, uint64_t stride,
+                                                                    uint64_t off_idx, uint64_t off_val, uint32_t n,
+                                                                    uint64_t k, uint64_t d, float* acc) {
+  __shared__ uint64_t s_bound[2 * 128];
+  const uint32_t tid = threadIdx.x;
+  const uint64_t span_lo = (uint64_t)blockIdx.x * kAccSpan;
+  const uint64_t span_hi = min(span_lo + kAccSpan, d);
+  for (uint32_t i0 = 0; i0 < n; i0 += 128) {
+    const uint32_t nb = min(128u, n - i0);
+    if (tid < 2 * nb) {
+      const uint32_t* idx = reinterpret_cast<const uint32_t*>(wp + (uint64_t)(i0 + (tid >> 1)) * stride + off_idx);
+      const uint64_t bound = (tid & 1u) ? span_hi : span_lo;
+      uint64_t lo = 0, hi = k;  // first m with idx[m] >= bound
+      while (lo < hi) {
+        const uint64_t mid = (lo + hi) >> 1;
+        if (idx[mid] < bound) lo = mid + 1; else hi = mid;
+      }
+      s_bound[tid] = lo;
+    }
+    __syncthreads();
+    for (uint32_t u = 0; u < nb; ++u) {
+      const uint8_t* pl = wp + (uint64_t)(i0 + u) * stride;
+      const uint32_t* idx = reinterpret_cast<const uint32_t*>(pl + off_idx);
+      const float* val = reinterpret_cast<const float*>(pl + off_val);
+      const uint64_t hi = s_bound[2 * u + 1];
+      for (uint64_t m = s_bound[2 * u] + tid; m < hi; m += kThreads) {
+        const uint32_t j = idx[m];
+        acc[j] = __fadd_rn(acc[j], val[m]);
+      }
+      __syncthreads();  // the next worker may add to the same entries
+    }
   }
 }
 
-cudaError_t launch_sparse_accumulate(const uint32_t* idx, const float* val, uint64_t k, float* acc, cudaStream_t st) {
-  if (k == 0) return cudaSuccess;
-  k_sparse_accumulate<<<grid_for(k), kThreads, 0, st>>>(idx, val, k, acc);
+cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_t off_idx, uint64_t off_val, uint32_t n,
+                                     uint64_t k, uint64_t d, float* acc, cudaStream_t st) {
+  if (k == 0 || n == 0) return cudaSuccess;
+  k_sparse_accumulate_all<<<(unsigned)((d + kAccSpan - 1) / kAccSpan), kThreads, 0, st>>>(wp, stride, off_idx, off_val, n, k,
+                                                                                          d, acc);
   count_launches(1);
   return cudaGetLastError();
 }

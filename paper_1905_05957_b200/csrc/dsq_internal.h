@@ -95,7 +95,8 @@ cudaError_t launch_identity(int src_kind, const SrcParams& src, float* out_c, ui
 // x = x - gamma * decode(payload)
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);
 
-// acc[idx[m]] += val[m] for one worker's sparse payload (indices are unique within a payload)
-cudaError_t launch_sparse_accumulate(const uint32_t* idx, const float* val, uint64_t k, float* acc, cudaStream_t st);
+// acc[j] = sum over workers i = 0..n-1, in that order, of the value worker i's sparse payload holds for j
+cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_t off_idx, uint64_t off_val, uint32_t n,
+                                     uint64_t k, uint64_t d, float* acc, cudaStream_t st);
 
 }  // namespace dsq
