@@ -31,7 +31,14 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/; valid only for the kernel sources with this digest.
 NCU_TRAFFIC = {
-    # workload id: (kernel, bytes per launch, digest of csrc/ at capture time)
+    # workload id: (kernel, bytes per launch, digest of the kernel's source files at capture time)
+    2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748170240 + 333396480, "7c901e443460a549"),
+}
+KERNEL_SOURCES = {  # files whose change invalidates the captured counters
+    "sign1": ("dsq_chunked.cu", "dsq_common.cuh", "dsq_internal.h"),
+    "qsgd": ("dsq_chunked.cu", "dsq_common.cuh", "dsq_internal.h"),
+    "topk": ("dsq_topk.cu", "dsq_common.cuh", "dsq_internal.h"),
+    "identity": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
 }
 
 
@@ -58,12 +65,11 @@ def algorithmic_bytes(wl) -> dict:
     return {"worker": worker, "server": server, "total": worker + server}
 
 
-def csrc_digest() -> str:
+def csrc_digest(op: str) -> str:
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_1905_05957_b200", "csrc")
-    for f in sorted(os.listdir(csrc)):
-        if f.endswith((".cu", ".cuh", ".h")):
-            h.update(open(os.path.join(csrc, f), "rb").read())
+    for f in KERNEL_SOURCES[op]:
+        h.update(open(os.path.join(csrc, f), "rb").read())
     return h.hexdigest()[:16]
 
 
@@ -282,7 +288,7 @@ def run_ours(args, wl):
         peak, peak_kind = measured_peak()
         wk_ms = statistics.mean(worker_ms)
         achieved = ab["worker"] / (wk_ms * 1e-3) / 1e9
-        digest = csrc_digest()
+        digest = csrc_digest(wl.worker_q.op)
         traffic = None
         if wl.wid in NCU_TRAFFIC and NCU_TRAFFIC[wl.wid][2] == digest:
             traffic = NCU_TRAFFIC[wl.wid][1]
