@@ -203,6 +203,7 @@ def run_ours(args, wl):
     import torch.distributed as dist
 
     from paper_1905_05957_b200 import DoubleSqueeze, load_library
+    from paper_1905_05957_b200.replicas import aggregate_throughput, max_over_ranks
     from paper_1905_05957_b200.workloads import make_gradients
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -278,10 +279,7 @@ def run_ours(args, wl):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    times = torch.tensor([t_total, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_total, e2e_ms = float(times[0]), float(times[1])
+    t_total, e2e_ms = max_over_ranks([t_total, e2e_ms], device=dev)
 
     if rank == 0:
         ab = algorithmic_bytes(wl)
@@ -295,13 +293,12 @@ def run_ours(args, wl):
         dominant = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
                     "topk": "top-k worker pass (pass1, mark, refine, finalize, emit)",
                     "identity": "k_identity<WORKER>"}[wl.worker_q.op]
-        elems = world * wl.n * wl.d
         line = {
-            "metric": METRIC, "value": elems * K / (t_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "metric": METRIC, "value": aggregate_throughput(wl.n * wl.d, K, t_total, world), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": t_total / K, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl),
             "clocks": clocks,
-            "e2e": {"value": elems * Ke / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": wl.n * wl.d * 4,
+            "e2e": {"value": aggregate_throughput(wl.n * wl.d, Ke, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": wl.n * wl.d * 4,
                     "d2h_bytes_per_step": int(ds.server_payload.numel()), "steps": Ke},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",

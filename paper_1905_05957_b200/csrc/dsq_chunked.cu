@@ -78,7 +78,7 @@ __device__ __forceinline__ uint32_t octet_sign_words(const uint32_t (&nib)[V], u
 }
 
 template <int OP, int SRC, int V, int LOG2G, bool FULL>
-__device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkParams& p, float* s_red) {
+__device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkParams& p, float* s_red, float* s_scal) {
   constexpr uint32_t G = 1u << LOG2G;
   constexpr uint32_t L = (uint32_t)V * G * 4u;
   constexpr uint32_t NG = (V * G) >> 5;   // 128-entry groups per chunk
@@ -164,15 +164,24 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
     s_or_q = __fdiv_rn(total, (float)len);  // mean |v| over the true chunk length
     if (chunk_live && t == 0) p.out_scale[(uint64_t)row * p.scale_stride + c] = s_or_q;
   } else {
-    float N = __fsqrt_rn(total);
+    // square root and the two divisions once per chunk (its first warp), not once per thread
     float q = 0.f;
-    bool live = (N > 0.f) && (N < __int_as_float(0x7f800000));
-    if (live) {
-      inv_q = __fdiv_rn(p.levels_f, N);
-      q = __fdiv_rn(N, p.levels_f);
-      live = inv_q < __int_as_float(0x7f800000);
+    if (G == 32 || (t >> 5) == 0) {
+      float N = __fsqrt_rn(total);
+      bool live = (N > 0.f) && (N < __int_as_float(0x7f800000));
+      if (live) {
+        inv_q = __fdiv_rn(p.levels_f, N);
+        q = __fdiv_rn(N, p.levels_f);
+        live = inv_q < __int_as_float(0x7f800000);
+      }
+      if (!live) { q = 0.f; inv_q = 0.f; }
+      if (G > 32 && lane == 0) { s_scal[2 * sub] = q; s_scal[2 * sub + 1] = inv_q; }
     }
-    if (!live) { N = 0.f; q = 0.f; inv_q = 0.f; }
+    if constexpr (G > 32) {
+      __syncthreads();
+      q = s_scal[2 * sub];
+      inv_q = s_scal[2 * sub + 1];
+    }
     s_or_q = q;
     if (chunk_live && t == 0) p.out_scale[(uint64_t)row * p.scale_stride + c] = q;  // the grid step is what is sent
   }
@@ -253,12 +262,13 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
 template <int OP, int SRC, int V, int LOG2G>
 __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const ChunkParams p) {
   __shared__ float s_red[64];
+  __shared__ float s_scal[16];
   constexpr uint64_t span = (uint64_t)V * 4u * kThreads;  // entries per CTA
   // interior CTA of an aligned row: no bounds logic anywhere
   if (src.vec && ((uint64_t)blockIdx.x + 1) * span <= src.d) {
-    chunk_body<OP, SRC, V, LOG2G, true>(src, p, s_red);
+    chunk_body<OP, SRC, V, LOG2G, true>(src, p, s_red, s_scal);
   } else {
-    chunk_body<OP, SRC, V, LOG2G, false>(src, p, s_red);
+    chunk_body<OP, SRC, V, LOG2G, false>(src, p, s_red, s_scal);
   }
 }
 
