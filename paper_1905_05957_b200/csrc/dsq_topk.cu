@@ -873,6 +873,13 @@ __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, uint64_t nse
   }
 }
 
+// A scattered 4-byte read: ask L2 to fetch no more than 64 bytes around it.
+__device__ __forceinline__ float gather_f32(const float* p) {
+  float v;
+  asm volatile("ld.global.L2::64B.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+
 __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d, const TopkState* state,
                                                         const uint32_t* bm_gt, const uint32_t* bm_eq, uint64_t bm_stride,
                                                         const uint2* seg_pre, uint64_t nseg, uint8_t* payload,
@@ -882,10 +889,26 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.y;
   const uint64_t widx = (uint64_t)blockIdx.x * kSegWords + tid * kWordsPerThread;
   const uint64_t at = (uint64_t)row * bm_stride + widx;
+  // everything that does not depend on the scan is fetched first, so that a thread has one round
+  // of bitmap loads and then up to eight value gathers in flight while the scan runs
+  const uint2 pre = seg_pre[(uint64_t)row * nseg + blockIdx.x];
+  const uint32_t r = state[row].r;
   const uint4 g4 = *reinterpret_cast<const uint4*>(bm_gt + at);
   const uint4 t4 = *reinterpret_cast<const uint4*>(bm_eq + at);
   const uint32_t gt[4] = {g4.x, g4.y, g4.z, g4.w};
   const uint32_t tie[4] = {t4.x, t4.y, t4.z, t4.w};
+  float* vrow = v_io + (uint64_t)row * d;
+  // the first two kept entries of every word (ties aside, which are rare and wait for the scan)
+  uint32_t b0[4], b1[4];
+  float v0[4], v1[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t s0 = gt[i], s1 = s0 & (s0 - 1u);
+    b0[i] = s0 ? __ffs(s0) - 1u : 32u;
+    b1[i] = s1 ? __ffs(s1) - 1u : 32u;
+    v0[i] = b0[i] < 32u ? gather_f32(vrow + (widx + i) * 32u + b0[i]) : 0.f;
+    v1[i] = b1[i] < 32u ? gather_f32(vrow + (widx + i) * 32u + b1[i]) : 0.f;
+  }
   // exclusive scan inside the segment; kept count in the low 16 bits, tie count in the high 16
   uint32_t cw[4], mine = 0;
 #pragma unroll
@@ -905,64 +928,48 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
   for (uint32_t i = 0; i < wrp; ++i) warp_pre += s_warp[i];
   uint32_t excl = warp_pre + incl - mine;
   if (!mine) return;
-  const uint2 pre = seg_pre[(uint64_t)row * nseg + blockIdx.x];
-  const uint32_t r = state[row].r;
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(payload + (uint64_t)row * payload_stride + off_idx);
   float* out_val = reinterpret_cast<float*>(payload + (uint64_t)row * payload_stride + off_val);
-  float* vrow = v_io + (uint64_t)row * d;
-  // which bits of each word are emitted, and the output slot of the first of them
-  uint32_t selw[4], posw[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const uint32_t ties_before = pre.y + (excl >> 16);
-    uint32_t keep = tie[i];
-    const uint32_t room = r > ties_before ? r - ties_before : 0u;
-    while ((uint32_t)__popc(keep) > room) keep &= ~(0x80000000u >> __clz(keep));  // drop the highest tie
-    selw[i] = gt[i] | keep;
-    posw[i] = pre.x + (excl & 0xFFFFu) + min(ties_before, r);
+    if (cw[i]) {
+      const uint32_t ties_before = pre.y + (excl >> 16);
+      uint32_t keep = tie[i];
+      const uint32_t room = r > ties_before ? r - ties_before : 0u;
+      while ((uint32_t)__popc(keep) > room) keep &= ~(0x80000000u >> __clz(keep));  // drop the highest tie
+      uint32_t pos = pre.x + (excl & 0xFFFFu) + min(ties_before, r);
+      uint32_t sel = gt[i] | keep;
+      if (!keep) {
+        // no tie in this word: the prefetched values are its first two entries
+        if (b0[i] < 32u) {
+          const uint64_t j = (widx + i) * 32u + b0[i];
+          if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v0[i]; }  // pos < k whenever the counts are consistent
+          vrow[j] = 0.f;                                                      // delta = v - Q[v] at a kept entry
+          if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v0[i]));
+          ++pos;
+        }
+        if (b1[i] < 32u) {
+          const uint64_t j = (widx + i) * 32u + b1[i];
+          if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v1[i]; }
+          vrow[j] = 0.f;
+          if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v1[i]));
+          ++pos;
+        }
+        sel &= sel - 1u;
+        sel &= sel - 1u;  // what is left after the first two (clearing bits of 0 leaves 0)
+      }
+      while (sel) {
+        const uint32_t b = __ffs(sel) - 1u;
+        sel &= sel - 1u;
+        const uint64_t j = (widx + i) * 32u + b;
+        const float val = vrow[j];
+        if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = val; }
+        vrow[j] = 0.f;
+        if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
+        ++pos;
+      }
+    }
     excl += cw[i];
-  }
-  // the first two kept entries of every word are fetched before anything is stored, so that a
-  // thread has up to eight gathers in flight; words with more (rare) finish in the loop below
-  uint32_t b0[4], b1[4];
-  float v0[4], v1[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint32_t s0 = selw[i], s1 = s0 & (s0 - 1u);
-    b0[i] = s0 ? __ffs(s0) - 1u : 32u;
-    b1[i] = s1 ? __ffs(s1) - 1u : 32u;
-    v0[i] = b0[i] < 32u ? vrow[(widx + i) * 32u + b0[i]] : 0.f;
-    v1[i] = b1[i] < 32u ? vrow[(widx + i) * 32u + b1[i]] : 0.f;
-  }
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    uint32_t pos = posw[i];
-    if (b0[i] < 32u) {
-      const uint64_t j = (widx + i) * 32u + b0[i];
-      if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v0[i]; }  // pos < k whenever the counts are consistent
-      vrow[j] = 0.f;                                                      // delta = v - Q[v] at a kept entry
-      if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v0[i]));
-      ++pos;
-    }
-    if (b1[i] < 32u) {
-      const uint64_t j = (widx + i) * 32u + b1[i];
-      if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v1[i]; }
-      vrow[j] = 0.f;
-      if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v1[i]));
-      ++pos;
-    }
-    uint32_t sel = selw[i] & (selw[i] - 1u);
-    sel &= sel - 1u;  // the entries after the first two
-    while (sel) {
-      const uint32_t b = __ffs(sel) - 1u;
-      sel &= sel - 1u;
-      const uint64_t j = (widx + i) * 32u + b;
-      const float val = vrow[j];
-      if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = val; }
-      vrow[j] = 0.f;
-      if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
-      ++pos;
-    }
   }
 }
 
@@ -1019,9 +1026,10 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   dim3 g1b((unsigned)((padded + span - 1) / span), rows, 1);
   const uint32_t k32 = (uint32_t)k;
   dim3 gs((unsigned)pl.nseg, rows, 1);
-  // kernels that re-read a whole vector after a miss: a grid that fills the GPU and strides over tiles
-  uint64_t stride_ctas = 148ull * 8ull / rows;
-  if (stride_ctas < 1) stride_ctas = 1;
+  // kernels that re-read a whole vector after a miss: per vector a grid that fills the GPU by itself
+  // and strides over the tiles, so that a single vector that missed is not left to a sliver of
+  // the machine; the CTAs of the vectors that hit leave at once
+  uint64_t stride_ctas = 148ull * 4ull;
   if (stride_ctas > padded / kTile) stride_ctas = padded / kTile;
   dim3 gm((unsigned)stride_ctas, rows, 1);
 
