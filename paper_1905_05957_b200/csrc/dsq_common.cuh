@@ -67,10 +67,8 @@ __device__ __forceinline__ float signed_by_bit(float m, uint32_t w, int k) {
   return __uint_as_float(__float_as_uint(m) ^ ((~w << (31 - k)) & 0x80000000u));
 }
 
-// Exact float value of byte `k` of `x`: place the byte in the mantissa of 2^23 and subtract 2^23.
-__device__ __forceinline__ float byte_to_float(uint32_t x, int k) {
-  return __fadd_rn(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7440u + k)), -8388608.0f);
-}
+// Exact float value of byte `k` of `x` (one conversion instruction with a byte selector).
+__device__ __forceinline__ float byte_to_float(uint32_t x, int k) { return __uint2float_rn((x >> (8 * k)) & 0xFFu); }
 
 // The vector to compress, for a tile of V rows: row j of the calling thread is the float4 at entry
 // e[j] of vector `row`; cnt[j] in [0, 4] says how many of its entries exist (the others, and whole
