@@ -72,6 +72,7 @@ struct ds_ctx {
   ds_payload_layout wl, sl;
   TopkPlan wplan, splan;  // workspace carving of the top-k path (worker rows / server row)
   float* acc;             // dense accumulator for sparse worker payloads (inside workspace), or NULL
+  uint32_t* acc_offsets;  // span offsets of the sparse payloads (inside workspace), or NULL
   int phase;              // 0: step complete, 1: worker pass done, 2: unfused server pass done
 };
 
@@ -94,9 +95,14 @@ uint64_t plan_workspace(ds_ctx* c) {
   uint64_t total = round16(topk_bytes);
   const uint64_t acc_off = total;
   if (cfg.worker_q.op == DS_Q_TOPK) total += round16(cfg.d * 4);
+  const uint64_t accoff_off = total;
+  if (cfg.worker_q.op == DS_Q_TOPK) total += round16(sparse_offsets_bytes(cfg.n, cfg.d));
   c->acc = (cfg.worker_q.op == DS_Q_TOPK && c->buf.workspace)
                ? reinterpret_cast<float*>(static_cast<uint8_t*>(c->buf.workspace) + acc_off)
                : nullptr;
+  c->acc_offsets = (cfg.worker_q.op == DS_Q_TOPK && c->buf.workspace)
+                       ? reinterpret_cast<uint32_t*>(static_cast<uint8_t*>(c->buf.workspace) + accoff_off)
+                       : nullptr;
   uint8_t* ws = static_cast<uint8_t*>(c->buf.workspace);
   if (cfg.worker_q.op == DS_Q_TOPK) {
     c->wplan.pred = ws ? reinterpret_cast<TopkPred*>(ws + total) : nullptr;
@@ -274,10 +280,9 @@ int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, voi
   const SrcParams src = server_src(h, &kind);
   if (kind == SRC_SRV_TOPK) {
     // (1/n) sum_i Q[v_i] for sparse payloads: dense accumulator, workers added in order 0..n-1
-    cudaError_t e = cudaMemsetAsync(h->acc, 0, h->cfg.d * 4, st);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
-    e = launch_sparse_accumulate(static_cast<const uint8_t*>(h->buf.worker_payload), h->wl.stride, h->wl.off[0], h->wl.off[1],
-                                 h->cfg.n, h->cfg.worker_q.k, h->cfg.d, h->acc, st);
+    const cudaError_t e = launch_sparse_accumulate(static_cast<const uint8_t*>(h->buf.worker_payload), h->wl.stride,
+                                                   h->wl.off[0], h->wl.off[1], h->cfg.n, h->cfg.worker_q.k, h->cfg.d,
+                                                   h->acc_offsets, h->acc, st);
     if (e != cudaSuccess) return cuda_fail(e, "sparse accumulate");
   }
   const bool fuse = (flags & DS_FUSE_APPLY) != 0;

@@ -107,53 +107,99 @@ cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamm
 }
 
 // Sum of the n sparse worker payloads into the dense accumulator, workers added in order
-// 0..n-1 as Eq. 4 is evaluated.  A CTA owns a span of indices: it first finds, for up to 128
-// workers at a time, where that span begins and ends in each worker's ascending index list
-// (binary searches, all in parallel), then walks the workers in order with a barrier in between.
-// Indices inside one payload are distinct, so the additions of one worker never collide, and no
-// other CTA touches this span.
+// 0..n-1 as Eq. 4 is evaluated.
+//
+// k_sparse_offsets: for every worker, where each span of kAccSpan indices begins in its ascending
+// index list (off[i][s] = first m with idx[m] >= s * kAccSpan; off[i][nspan] = k).
+// k_sparse_accumulate: a CTA owns one span and builds its slice of the sum in shared memory: the
+// entries of eight workers are fetched at once, then added worker by worker with a barrier in
+// between (indices inside one payload are distinct, so one worker's additions never collide), and
+// the finished slice is written out whole -- the accumulator needs no clearing beforehand.
 constexpr uint32_t kAccSpan = 8192;
 
-__global__ void __launch_bounds__(kThreads) k_sparse_accumulate_all(const uint8_t* __restrict__ wp, uint64_t stride,
-                                                                    uint64_t off_idx, uint64_t off_val, uint32_t n,
-                                                                    uint64_t k, uint64_t d, float* acc) {
-  __shared__ uint64_t s_bound[2 * 128];
+__global__ void __launch_bounds__(kThreads) k_sparse_offsets(const uint8_t* __restrict__ wp, uint64_t stride, uint64_t off_idx,
+                                                             uint64_t k, uint64_t nspan, uint32_t* off) {
+  const uint32_t i = blockIdx.y;
+  const uint32_t* idx = reinterpret_cast<const uint32_t*>(wp + (uint64_t)i * stride + off_idx);
+  uint32_t* o = off + (uint64_t)i * (nspan + 1);
+  for (uint64_t m = (uint64_t)blockIdx.x * kThreads + threadIdx.x; m <= k; m += (uint64_t)gridDim.x * kThreads) {
+    // entry m opens every span after the one entry m-1 lies in, up to and including its own
+    const uint64_t first = m == 0 ? 0 : (uint64_t)(idx[m - 1] / kAccSpan) + 1;
+    uint64_t last = m == k ? nspan : (uint64_t)(idx[m] / kAccSpan);
+    if (last > nspan) last = nspan;  // an index beyond d in a foreign payload must not leave the table
+    for (uint64_t s = first; s <= last; ++s) o[s] = (uint32_t)m;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) k_sparse_accumulate(const uint8_t* __restrict__ wp, uint64_t stride,
+                                                                uint64_t off_idx, uint64_t off_val, uint32_t n, uint64_t d,
+                                                                uint64_t nspan, const uint32_t* __restrict__ off,
+                                                                float* acc) {
+  __shared__ float s_acc[kAccSpan];
   const uint32_t tid = threadIdx.x;
-  const uint64_t span_lo = (uint64_t)blockIdx.x * kAccSpan;
-  const uint64_t span_hi = min(span_lo + kAccSpan, d);
-  for (uint32_t i0 = 0; i0 < n; i0 += 128) {
-    const uint32_t nb = min(128u, n - i0);
-    if (tid < 2 * nb) {
-      const uint32_t* idx = reinterpret_cast<const uint32_t*>(wp + (uint64_t)(i0 + (tid >> 1)) * stride + off_idx);
-      const uint64_t bound = (tid & 1u) ? span_hi : span_lo;
-      uint64_t lo = 0, hi = k;  // first m with idx[m] >= bound
-      while (lo < hi) {
-        const uint64_t mid = (lo + hi) >> 1;
-        if (idx[mid] < bound) lo = mid + 1; else hi = mid;
+  const uint64_t span = blockIdx.x;
+  const uint32_t base = (uint32_t)(span * kAccSpan);
+  for (uint32_t j = tid; j < kAccSpan; j += kThreads) s_acc[j] = 0.f;
+  __syncthreads();
+  for (uint32_t i0 = 0; i0 < n; i0 += 8) {
+    // first entry of this thread in each of eight workers' slices, fetched before any is used
+    uint32_t lo[8], hi[8], ji[8];
+    float vi[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      lo[u] = 0; hi[u] = 0; ji[u] = 0; vi[u] = 0.f;
+      if (i0 + u < n) {
+        const uint32_t* o = off + (uint64_t)(i0 + u) * (nspan + 1) + span;
+        lo[u] = o[0];
+        hi[u] = o[1];
       }
-      s_bound[tid] = lo;
     }
-    __syncthreads();
-    for (uint32_t u = 0; u < nb; ++u) {
-      const uint8_t* pl = wp + (uint64_t)(i0 + u) * stride;
-      const uint32_t* idx = reinterpret_cast<const uint32_t*>(pl + off_idx);
-      const float* val = reinterpret_cast<const float*>(pl + off_val);
-      const uint64_t hi = s_bound[2 * u + 1];
-      for (uint64_t m = s_bound[2 * u] + tid; m < hi; m += kThreads) {
-        const uint32_t j = idx[m];
-        acc[j] = __fadd_rn(acc[j], val[m]);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (lo[u] + tid < hi[u]) {
+        const uint8_t* pl = wp + (uint64_t)(i0 + u) * stride;
+        ji[u] = reinterpret_cast<const uint32_t*>(pl + off_idx)[lo[u] + tid];
+        vi[u] = reinterpret_cast<const float*>(pl + off_val)[lo[u] + tid];
       }
-      __syncthreads();  // the next worker may add to the same entries
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (i0 + u < n) {
+        if (lo[u] + tid < hi[u]) {
+          const uint32_t j = (ji[u] - base) & (kAccSpan - 1u);  // masked: never leaves the slice
+          s_acc[j] = __fadd_rn(s_acc[j], vi[u]);
+        }
+        // a slice with more entries than threads (dense payloads) finishes here
+        const uint8_t* pl = wp + (uint64_t)(i0 + u) * stride;
+        for (uint32_t m = lo[u] + tid + kThreads; m < hi[u]; m += kThreads) {
+          const uint32_t j = (reinterpret_cast<const uint32_t*>(pl + off_idx)[m] - base) & (kAccSpan - 1u);
+          s_acc[j] = __fadd_rn(s_acc[j], reinterpret_cast<const float*>(pl + off_val)[m]);
+        }
+        __syncthreads();  // the next worker may add to the same entries
+      }
+    }
+  }
+  for (uint32_t j = tid * 4; j < kAccSpan; j += kThreads * 4) {
+    const uint64_t e = (uint64_t)base + j;
+    if (e + 4 <= d) {
+      *reinterpret_cast<float4*>(acc + e) = make_float4(s_acc[j], s_acc[j + 1], s_acc[j + 2], s_acc[j + 3]);
+    } else {
+      for (uint32_t q = 0; q < 4; ++q)
+        if (e + q < d) acc[e + q] = s_acc[j + q];
     }
   }
 }
 
+uint64_t sparse_offsets_bytes(uint32_t n, uint64_t d) { return (uint64_t)n * ((d + kAccSpan - 1) / kAccSpan + 1) * 4; }
+
 cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_t off_idx, uint64_t off_val, uint32_t n,
-                                     uint64_t k, uint64_t d, float* acc, cudaStream_t st) {
-  if (k == 0 || n == 0) return cudaSuccess;
-  k_sparse_accumulate_all<<<(unsigned)((d + kAccSpan - 1) / kAccSpan), kThreads, 0, st>>>(wp, stride, off_idx, off_val, n, k,
-                                                                                          d, acc);
-  count_launches(1);
+                                     uint64_t k, uint64_t d, uint32_t* offsets, float* acc, cudaStream_t st) {
+  const uint64_t nspan = (d + kAccSpan - 1) / kAccSpan;
+  uint64_t ctas = (k + kThreads) / kThreads;
+  if (ctas > 148 * 8) ctas = 148 * 8;
+  k_sparse_offsets<<<dim3((unsigned)ctas, n, 1), kThreads, 0, st>>>(wp, stride, off_idx, k, nspan, offsets);
+  k_sparse_accumulate<<<(unsigned)nspan, kThreads, 0, st>>>(wp, stride, off_idx, off_val, n, d, nspan, offsets, acc);
+  count_launches(2);
   return cudaGetLastError();
 }
 

@@ -96,7 +96,9 @@ cudaError_t launch_identity(int src_kind, const SrcParams& src, float* out_c, ui
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);
 
 // acc[j] = sum over workers i = 0..n-1, in that order, of the value worker i's sparse payload holds for j
+// (every entry of acc is written).  offsets: scratch of sparse_offsets_bytes(n, d) bytes.
+uint64_t sparse_offsets_bytes(uint32_t n, uint64_t d);
 cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_t off_idx, uint64_t off_val, uint32_t n,
-                                     uint64_t k, uint64_t d, float* acc, cudaStream_t st);
+                                     uint64_t k, uint64_t d, uint32_t* offsets, float* acc, cudaStream_t st);
 
 }  // namespace dsq

@@ -421,14 +421,26 @@ __device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint2*
     uint32_t base = 0;
     if (lane == 0) base = atomicAdd(dense_count, total);
     base = __shfl_sync(0xffffffffu, base, 0);
+    // the first 32 entries of all eight regions are fetched before any is used
+    uint2 first[8];
+    uint32_t ns[8], offs[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const uint32_t n = __shfl_sync(0xffffffffu, mine.x, u);
-      const uint32_t off = __shfl_sync(0xffffffffu, incl - mine.x, u);
+      ns[u] = __shfl_sync(0xffffffffu, mine.x, u);
+      offs[u] = __shfl_sync(0xffffffffu, incl - mine.x, u);
+      first[u] = make_uint2(0u, 0u);
+      if (lane < ns[u]) first[u] = lrow[(t0 + u) * kTile + lane];
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (lane < ns[u]) {
+        drow[(uint64_t)base + offs[u] + lane] = first[u];
+        if (HIST) atomicAdd(&s_hist[(first[u].x >> 19) & 0xFFFu], 1u);
+      }
       const uint2* reg = lrow + (t0 + u) * kTile;
-      for (uint32_t i = lane; i < n; i += 32) {
+      for (uint32_t i = lane + 32; i < ns[u]; i += 32) {
         const uint2 e = reg[i];
-        drow[(uint64_t)base + off + i] = e;
+        drow[(uint64_t)base + offs[u] + i] = e;
         if (HIST) atomicAdd(&s_hist[(e.x >> 19) & 0xFFFu], 1u);
       }
     }
@@ -1026,10 +1038,11 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   dim3 g1b((unsigned)((padded + span - 1) / span), rows, 1);
   const uint32_t k32 = (uint32_t)k;
   dim3 gs((unsigned)pl.nseg, rows, 1);
-  // kernels that re-read a whole vector after a miss: per vector a grid that fills the GPU by itself
-  // and strides over the tiles, so that a single vector that missed is not left to a sliver of
-  // the machine; the CTAs of the vectors that hit leave at once
-  uint64_t stride_ctas = 148ull * 4ull;
+  // kernels that re-read a whole vector after a miss: per vector a grid that (nearly) fills the GPU by
+  // itself and strides over the tiles, so that a single vector that missed is not left to a sliver
+  // of the machine; the CTAs of the vectors that hit leave at once, so with many vectors the grid
+  // per vector is halved to keep those empty launches short
+  uint64_t stride_ctas = rows >= 8 ? 148ull * 2ull : 148ull * 4ull;
   if (stride_ctas > padded / kTile) stride_ctas = padded / kTile;
   dim3 gm((unsigned)stride_ctas, rows, 1);
 
