@@ -20,32 +20,37 @@ SERVER_WID = 0xFFFFFFFF
 _lib = None
 
 
+def load(path: str):
+    """Opens an oracle shared library and declares its signatures."""
+    L = C.CDLL(path)
+    f32p, u32p, u8p = C.POINTER(C.c_float), C.POINTER(C.c_uint32), C.POINTER(C.c_uint8)
+    u64, u32 = C.c_uint64, C.c_uint32
+    L.orc_pairwise_sum.restype = C.c_float
+    L.orc_pairwise_sum.argtypes = [f32p, u64]
+    L.orc_philox4x32_10.restype = None
+    L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
+    L.orc_ef_add.restype = None
+    L.orc_ef_add.argtypes = [f32p, f32p, u64, f32p]
+    L.orc_residual.restype = None
+    L.orc_residual.argtypes = [f32p, f32p, u64, f32p]
+    L.orc_server_mean_add.restype = None
+    L.orc_server_mean_add.argtypes = [f32p, u32, u64, f32p, f32p]
+    L.orc_apply_update.restype = None
+    L.orc_apply_update.argtypes = [f32p, f32p, C.c_float, u64]
+    L.orc_q_identity.argtypes = [f32p, u64, f32p]
+    L.orc_q_sign1.argtypes = [f32p, u64, u32, u32p, f32p, f32p]
+    L.orc_decode_sign1.argtypes = [u32p, f32p, u64, u32, f32p]
+    L.orc_q_topk.argtypes = [f32p, u64, u64, u32p, f32p, f32p]
+    L.orc_decode_topk.argtypes = [u32p, f32p, u64, u64, f32p]
+    L.orc_q_qsgd.argtypes = [f32p, u64, u32, u32, u64, u32, u32, u8p, u32p, f32p, f32p, f32p]
+    L.orc_decode_qsgd.argtypes = [u8p, u32p, f32p, u64, u32, f32p]
+    return L
+
+
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(_build.build())
-        f32p, u32p, u8p = C.POINTER(C.c_float), C.POINTER(C.c_uint32), C.POINTER(C.c_uint8)
-        u64, u32 = C.c_uint64, C.c_uint32
-        L.orc_pairwise_sum.restype = C.c_float
-        L.orc_pairwise_sum.argtypes = [f32p, u64]
-        L.orc_philox4x32_10.restype = None
-        L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
-        L.orc_ef_add.restype = None
-        L.orc_ef_add.argtypes = [f32p, f32p, u64, f32p]
-        L.orc_residual.restype = None
-        L.orc_residual.argtypes = [f32p, f32p, u64, f32p]
-        L.orc_server_mean_add.restype = None
-        L.orc_server_mean_add.argtypes = [f32p, u32, u64, f32p, f32p]
-        L.orc_apply_update.restype = None
-        L.orc_apply_update.argtypes = [f32p, f32p, C.c_float, u64]
-        L.orc_q_identity.argtypes = [f32p, u64, f32p]
-        L.orc_q_sign1.argtypes = [f32p, u64, u32, u32p, f32p, f32p]
-        L.orc_decode_sign1.argtypes = [u32p, f32p, u64, u32, f32p]
-        L.orc_q_topk.argtypes = [f32p, u64, u64, u32p, f32p, f32p]
-        L.orc_decode_topk.argtypes = [u32p, f32p, u64, u64, f32p]
-        L.orc_q_qsgd.argtypes = [f32p, u64, u32, u32, u64, u32, u32, u8p, u32p, f32p, f32p, f32p]
-        L.orc_decode_qsgd.argtypes = [u8p, u32p, f32p, u64, u32, f32p]
-        _lib = L
+        _lib = load(_build.build())
     return _lib
 
 

@@ -160,3 +160,44 @@ def test_workload_recipes_scaled(wid):
     wl = wl if wid == 1 else wl.scaled(d=200_000 + 40, n=min(wl.n, 8), steps=4)
     gs = [make_gradients(wl, t, device="cpu") for t in range(min(wl.steps, 4))]
     run_lockstep(wl.n, wl.d, wl.worker_q, wl.server_q, gs, gamma=wl.gamma, seed=wl.seed)
+
+
+def test_state_copied_into_a_fresh_instance_continues_identically():
+    """x, delta_w and delta_s are the whole state (Algorithm 1): T steps, copy them into a new
+    instance (which has no threshold history), T more steps -- same bits as 2T steps in one go."""
+    n, d, T = 4, 60_000, 4
+    for wq, sq in [(TOPK(600), TOPK(600)), (QSGD(2048), QSGD(2048)), (SIGN(4096), TOPK(300))]:
+        gs = [g.cuda() for g in randn_steps(n, d, 2 * T, seed=17)]
+        one = DoubleSqueeze(n, d, 0.1, wq, sq, seed=5)
+        for t, g in enumerate(gs):
+            one.step(g, t)
+        first = DoubleSqueeze(n, d, 0.1, wq, sq, seed=5)
+        for t, g in enumerate(gs[:T]):
+            first.step(g, t)
+        second = DoubleSqueeze(n, d, 0.1, wq, sq, seed=5, x0=first.x)
+        second.delta_w.copy_(first.delta_w)
+        second.delta_s.copy_(first.delta_s)
+        for t, g in enumerate(gs[T:]):
+            second.step(g, T + t)
+        torch.cuda.synchronize()
+        for a, b in ((one.x, second.x), (one.delta_w, second.delta_w), (one.delta_s, second.delta_s),
+                     (one.server_payload, second.server_payload), (one.worker_payload, second.worker_payload)):
+            assert torch.equal(a.view(torch.uint8) if a.dtype == torch.uint8 else a.view(torch.int32),
+                               b.view(torch.uint8) if b.dtype == torch.uint8 else b.view(torch.int32))
+        assert one.device_status() == 0 and second.device_status() == 0
+
+
+def test_calls_out_of_order_are_refused_on_a_live_handle():
+    ds = DoubleSqueeze(2, 5000, 0.1, SIGN(1024), SIGN(1024))
+    g = torch.randn(2, 5000, device="cuda")
+    with pytest.raises(Exception, match="-4"):
+        ds.server_aggregate_compress(0)
+    ds.worker_compress(g, 0)
+    with pytest.raises(Exception, match="-4"):
+        ds.worker_compress(g, 0)
+    with pytest.raises(Exception, match="-4"):
+        ds.apply_update()
+    ds.server_aggregate_compress(0, fuse_apply=False)
+    ds.apply_update()
+    ds.step(g, 1)
+    torch.cuda.synchronize()
