@@ -201,3 +201,31 @@ def test_calls_out_of_order_are_refused_on_a_live_handle():
     ds.apply_update()
     ds.step(g, 1)
     torch.cuda.synchronize()
+
+
+def test_host_buffer_step_equals_device_step_and_counts_launches():
+    from paper_1905_05957_b200 import load_library
+    n, d = 3, 40_000 + 8
+    wq, sq = SIGN(4096), TOPK(400)
+    gs = randn_steps(n, d, 3, seed=23)
+    a = DoubleSqueeze(n, d, 0.1, wq, sq, seed=9)
+    b = DoubleSqueeze(n, d, 0.1, wq, sq, seed=9)
+    stage = torch.empty(n, d, device="cuda")
+    out = torch.empty(b.server_payload.numel(), dtype=torch.uint8).pin_memory()
+    x_host = torch.empty(d).pin_memory()
+    before = load_library().ds_kernel_launches()
+    for t, g in enumerate(gs):
+        a.step(g.cuda(), t)
+        b.step_host(g.contiguous().pin_memory(), stage, t, server_payload_host=out, x_host=x_host)
+        torch.cuda.synchronize()
+        assert torch.equal(a.x.view(torch.int32), b.x.view(torch.int32))
+        assert torch.equal(a.server_payload, b.server_payload)
+        assert torch.equal(out, b.server_payload.cpu())
+        assert torch.equal(x_host.view(torch.int32), b.x.cpu().view(torch.int32))
+    assert load_library().ds_kernel_launches() > before
+
+
+def test_more_workers_than_one_batch_of_the_server_loops():
+    # 150 sparse payloads (the ordered sum walks them in batches of 128) and 150 one-bit payloads
+    run_lockstep(150, 9000, TOPK(90), TOPK(90), randn_steps(150, 9000, 2, seed=31))
+    run_lockstep(150, 4096 + 100, SIGN(1024), QSGD(512, 63), randn_steps(150, 4096 + 100, 2, seed=32))
