@@ -104,8 +104,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
 #pragma unroll
     for (int j = 0; j < V; ++j) {
       cnt[j] = 4;
-      v[j] = make_float4(__fadd_rn(a[j].x, b[j].x), __fadd_rn(a[j].y, b[j].y), __fadd_rn(a[j].z, b[j].z),
-                         __fadd_rn(a[j].w, b[j].w));
+      v[j] = add4_rn(a[j], b[j]);
     }
   } else {
     uint64_t e[V];
@@ -134,8 +133,8 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
     if constexpr (OP == DS_Q_SIGN1) {
       m0 = fabsf(v[j].x); m1 = fabsf(v[j].y); m2 = fabsf(v[j].z); m3 = fabsf(v[j].w);
     } else {
-      m0 = __fmul_rn(v[j].x, v[j].x); m1 = __fmul_rn(v[j].y, v[j].y);
-      m2 = __fmul_rn(v[j].z, v[j].z); m3 = __fmul_rn(v[j].w, v[j].w);
+      const float4 sq = mul4_rn(v[j], v[j]);
+      m0 = sq.x; m1 = sq.y; m2 = sq.z; m3 = sq.w;
     }
     part[j] = __fadd_rn(__fadd_rn(m0, m1), __fadd_rn(m2, m3));
   }
@@ -206,25 +205,37 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
       const uint4 rnd = philox4x32_10(make_uint4(tq, (uint32_t)c, p.server_pass ? 0xFFFFFFFFu : row, p.step), p.keys);
       const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
       uint32_t lb[4];
+      // r = |v| * (s / N), clamped to s
+      float4 r4 = mul4_rn(make_float4(fabsf(v[j].x), fabsf(v[j].y), fabsf(v[j].z), fabsf(v[j].w)),
+                          make_float4(inv_q, inv_q, inv_q, inv_q));
+      r4 = make_float4(fminf(r4.x, p.levels_f), fminf(r4.y, p.levels_f), fminf(r4.z, p.levels_f), fminf(r4.w, p.levels_f));
+      // floor(r) for 0 <= r <= 255 without a conversion: adding 2^23 with rounding toward zero
+      // leaves 2^23 + floor(r), whose low mantissa byte is the integer and whose difference
+      // from 2^23 is the float
+      float4 tz4, f4;
+      {
+        const f32x2 big = pack2(8388608.0f, 8388608.0f), nbig = pack2(-8388608.0f, -8388608.0f);
+        const f32x2 t01 = add2_rz(pack2(r4.x, r4.y), big), t23 = add2_rz(pack2(r4.z, r4.w), big);
+        unpack2(t01, tz4.x, tz4.y);
+        unpack2(t23, tz4.z, tz4.w);
+        unpack2(add2_rn(t01, nbig), f4.x, f4.y);
+        unpack2(add2_rn(t23, nbig), f4.z, f4.w);
+      }
+      const float4 pr4 = sub4_rn(r4, f4);  // exact
+      float4 lf4;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const float val = compc(v[j], k);
         const float u = __fmul_rn(__uint2float_rn(w[k] >> 8), 5.9604644775390625e-08f);  // 2^-24, exact
-        float r = __fmul_rn(fabsf(val), inv_q);
-        r = fminf(r, p.levels_f);
-        // floor(r) for 0 <= r <= 255 without a conversion: adding 2^23 with rounding toward zero
-        // leaves 2^23 + floor(r), whose low mantissa byte is the integer and whose difference
-        // from 2^23 is the float
-        const float tz = __fadd_rz(r, 8388608.0f);
-        const float f = __fadd_rn(tz, -8388608.0f);
-        const float pr = __fsub_rn(r, f);  // exact
-        const bool up = u < pr;
-        lb[k] = __float_as_uint(tz) + (up ? 1u : 0u);      // low byte = level (no carry: r = 255 has pr = 0)
-        const float lf = up ? __fadd_rn(f, 1.0f) : f;      // the level as a float, exact
-        const float mag = __fmul_rn(lf, s_or_q);
-        const bool nonneg = val >= 0.f;
+        const bool up = u < compc(pr4, k);
+        lb[k] = __float_as_uint(compc(tz4, k)) + (up ? 1u : 0u);      // low byte = level (no carry: r = 255 has pr = 0)
+        comp(lf4, k) = up ? __fadd_rn(compc(f4, k), 1.0f) : compc(f4, k);  // the level as a float, exact
+      }
+      const float4 mag4 = mul4_rn(lf4, make_float4(s_or_q, s_or_q, s_or_q, s_or_q));
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const bool nonneg = compc(v[j], k) >= 0.f;
         nib[j] |= (nonneg ? 1u : 0u) << k;
-        comp(C, k) = nonneg ? mag : -mag;
+        comp(C, k) = nonneg ? compc(mag4, k) : -compc(mag4, k);
       }
       const uint32_t packed = __byte_perm(__byte_perm(lb[0], lb[1], 0x0040), __byte_perm(lb[2], lb[3], 0x0040), 0x5410);
       if (cnt[j]) *reinterpret_cast<uint32_t*>(p.out_lvl + (uint64_t)row * p.lvl_stride + e) = packed;
@@ -232,9 +243,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
     if constexpr (!FULL) nib[j] &= (1u << cnt[j]) - 1u;  // pad bits are 0
 
     if (cnt[j]) {
-      float4 dl;
-      dl.x = __fsub_rn(v[j].x, C.x); dl.y = __fsub_rn(v[j].y, C.y);
-      dl.z = __fsub_rn(v[j].z, C.z); dl.w = __fsub_rn(v[j].w, C.w);
+      const float4 dl = sub4_rn(v[j], C);
       if constexpr (FULL) {
         st_stream4(delta_chunk + tq * 4u, dl);
       } else {
@@ -242,7 +251,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
       }
       if (kServer && p.x) {  // fused model update (server pass only): x = x - gamma * Q[v]
         const float4 xo = xv[kServer ? j : 0];
-        float4 xn;
+        float4 xn;  // scalar: a multiply that feeds a subtract must not be contracted
         xn.x = __fsub_rn(xo.x, __fmul_rn(p.gamma, C.x)); xn.y = __fsub_rn(xo.y, __fmul_rn(p.gamma, C.y));
         xn.z = __fsub_rn(xo.z, __fmul_rn(p.gamma, C.z)); xn.w = __fsub_rn(xo.w, __fmul_rn(p.gamma, C.w));
         store_row4(p.x, e, cnt[j], 1, xn);

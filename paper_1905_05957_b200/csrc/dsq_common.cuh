@@ -62,6 +62,40 @@ __device__ __forceinline__ void store_row4(float* base, uint64_t e, uint32_t cnt
   }
 }
 
+// Packed pairs of binary32 (sm_100 adds .f32x2 arithmetic: one instruction, two IEEE results, each
+// rounded on its own exactly like the scalar instruction).  A pair lives in a 64-bit register.
+// Never let a packed multiply feed a packed add or subtract directly: that pair was observed to be
+// contracted into a fused multiply-add, which changes the rounding; such spots stay scalar.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 r, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r)); }
+__device__ __forceinline__ f32x2 add2_rn(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 add2_rz(f32x2 a, f32x2 b) { f32x2 d; asm("add.rz.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 sub2_rn(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 mul2_rn(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ float4 add4_rn(float4 a, float4 b) {
+  float4 r;
+  unpack2(add2_rn(pack2(a.x, a.y), pack2(b.x, b.y)), r.x, r.y);
+  unpack2(add2_rn(pack2(a.z, a.w), pack2(b.z, b.w)), r.z, r.w);
+  return r;
+}
+__device__ __forceinline__ float4 sub4_rn(float4 a, float4 b) {
+  float4 r;
+  unpack2(sub2_rn(pack2(a.x, a.y), pack2(b.x, b.y)), r.x, r.y);
+  unpack2(sub2_rn(pack2(a.z, a.w), pack2(b.z, b.w)), r.z, r.w);
+  return r;
+}
+__device__ __forceinline__ float4 mul4_rn(float4 a, float4 b) {
+  float4 r;
+  unpack2(mul2_rn(pack2(a.x, a.y), pack2(b.x, b.y)), r.x, r.y);
+  unpack2(mul2_rn(pack2(a.z, a.w), pack2(b.z, b.w)), r.z, r.w);
+  return r;
+}
+
 // +m or -m according to bit `k` of the sign word `w` (1 = non-negative), without a branch.
 __device__ __forceinline__ float signed_by_bit(float m, uint32_t w, int k) {
   return __uint_as_float(__float_as_uint(m) ^ ((~w << (31 - k)) & 0x80000000u));
@@ -89,8 +123,7 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
     for (int j = 0; j < V; ++j) b[j] = load_row4(p.delta + off, e[j], cnt[j], p.vec);
 #pragma unroll
     for (int j = 0; j < V; ++j)
-      v[j] = make_float4(__fadd_rn(a[j].x, b[j].x), __fadd_rn(a[j].y, b[j].y), __fadd_rn(a[j].z, b[j].z),
-                         __fadd_rn(a[j].w, b[j].w));
+      v[j] = add4_rn(a[j], b[j]);
   } else {
     const uint32_t lane = threadIdx.x & 31u;
     float4 acc[V], ds[V];
@@ -107,8 +140,7 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
         for (int j = 0; j < V; ++j) ci[j] = load_row4(c, e[j], cnt[j], 1);
 #pragma unroll
         for (int j = 0; j < V; ++j) {
-          acc[j].x = __fadd_rn(acc[j].x, ci[j].x); acc[j].y = __fadd_rn(acc[j].y, ci[j].y);
-          acc[j].z = __fadd_rn(acc[j].z, ci[j].z); acc[j].w = __fadd_rn(acc[j].w, ci[j].w);
+          acc[j] = add4_rn(acc[j], ci[j]);
         }
       }
     } else if constexpr (SRC == SRC_SRV_SIGN1 || SRC == SRC_SRV_QSGD) {
@@ -150,16 +182,15 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
             const float sc = __shfl_sync(0xffffffffu, sreg[j], u);
             if (i0 + u < p.n) {
               if constexpr (SRC == SRC_SRV_SIGN1) {
-                acc[j].x = __fadd_rn(acc[j].x, signed_by_bit(sc, ww, 0));
-                acc[j].y = __fadd_rn(acc[j].y, signed_by_bit(sc, ww, 1));
-                acc[j].z = __fadd_rn(acc[j].z, signed_by_bit(sc, ww, 2));
-                acc[j].w = __fadd_rn(acc[j].w, signed_by_bit(sc, ww, 3));
+                acc[j] = add4_rn(acc[j], make_float4(signed_by_bit(sc, ww, 0), signed_by_bit(sc, ww, 1),
+                                                     signed_by_bit(sc, ww, 2), signed_by_bit(sc, ww, 3)));
               } else {
                 const uint32_t l4 = lv[j][u];
-                acc[j].x = __fadd_rn(acc[j].x, signed_by_bit(__fmul_rn(byte_to_float(l4, 0), sc), ww, 0));
-                acc[j].y = __fadd_rn(acc[j].y, signed_by_bit(__fmul_rn(byte_to_float(l4, 1), sc), ww, 1));
-                acc[j].z = __fadd_rn(acc[j].z, signed_by_bit(__fmul_rn(byte_to_float(l4, 2), sc), ww, 2));
-                acc[j].w = __fadd_rn(acc[j].w, signed_by_bit(__fmul_rn(byte_to_float(l4, 3), sc), ww, 3));
+                const float4 mag = mul4_rn(make_float4(byte_to_float(l4, 0), byte_to_float(l4, 1), byte_to_float(l4, 2),
+                                                       byte_to_float(l4, 3)),
+                                           make_float4(sc, sc, sc, sc));
+                acc[j] = add4_rn(acc[j], make_float4(signed_by_bit(mag.x, ww, 0), signed_by_bit(mag.y, ww, 1),
+                                                     signed_by_bit(mag.z, ww, 2), signed_by_bit(mag.w, ww, 3)));
               }
             }
           }
@@ -171,6 +202,7 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
     }
 #pragma unroll
     for (int j = 0; j < V; ++j) {
+      // scalar on purpose: a packed multiply feeding a packed add was seen to come out fused
       v[j].x = __fadd_rn(__fmul_rn(acc[j].x, p.inv_n), ds[j].x); v[j].y = __fadd_rn(__fmul_rn(acc[j].y, p.inv_n), ds[j].y);
       v[j].z = __fadd_rn(__fmul_rn(acc[j].z, p.inv_n), ds[j].z); v[j].w = __fadd_rn(__fmul_rn(acc[j].w, p.inv_n), ds[j].w);
       // entries past the end must read as +0 whatever the payload padding holds

@@ -143,8 +143,7 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       cnt[j] = 4;
-      v[j] = make_float4(__fadd_rn(a[j].x, b[j].x), __fadd_rn(a[j].y, b[j].y), __fadd_rn(a[j].z, b[j].z),
-                         __fadd_rn(a[j].w, b[j].w));
+      v[j] = add4_rn(a[j], b[j]);
     }
   } else {
     uint64_t ee[4];
