@@ -55,7 +55,7 @@ struct TopkState {
 // Threshold history of one vector (the keys tau of the two previous steps), kept across steps so
 // that pass1 can mark candidates itself.
 struct TopkPred {
-  uint32_t magic, tau_last, tau_prev, pad;
+  uint32_t magic, tau_last, tau_prev, err;
 };
 
 // Carving of the workspace for `rows` simultaneous selections over d-vectors.

@@ -45,7 +45,9 @@ constexpr uint32_t kSegWords = kThreads * kWordsPerThread;  // 1024 bitmap words
 constexpr uint32_t kSegElems = kSegWords * 32;     // 32768 entries
 constexpr uint64_t kTile = 4096;                   // entries a CTA handles per loop trip
 constexpr uint32_t kPredMagic = 0x70D1C7EDu;
-constexpr uint32_t kBandHalf = 1u << 16;           // half-width of the band in key units (0.5 % of magnitude)
+constexpr uint32_t kBandHalf = 1u << 16;           // least half-width of the band in key units (0.5 % of magnitude)
+constexpr uint32_t kMaxErr = 1u << 21;             // widest extrapolation error followed (band: half an octave each way)
+constexpr uint32_t kFirstErr = kMaxErr;            // error assumed before any extrapolation has been checked
 constexpr int kMaxTrend = 1 << 20;                 // largest step-to-step drift that is extrapolated (9 %)
 
 __device__ __forceinline__ uint32_t key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
@@ -54,17 +56,22 @@ inline uint64_t round16(uint64_t b) { return (b + 15u) & ~uint64_t(15); }
 
 // Keys are monotone in log-magnitude (2^23 units per octave), so a threshold that drifts by a
 // steady factor moves by a steady key difference.  The band is the last threshold, extrapolated by
-// the last change (the drift itself changes slowly), widened on both sides by the larger of a
-// quarter of that change and 0.5 % of magnitude.
+// the last change (the drift itself changes slowly), widened on both sides by the largest of a
+// quarter of that change, 0.5 % of magnitude, and twice the recent extrapolation error (a decaying
+// maximum kept beside the thresholds), so the band is wide while the error memories are still
+// filling and narrows once the threshold settles.
 // Candidates are the entries with lo <= key <= hi; returns false when there is no usable history.
-__device__ __forceinline__ bool predicted_band(const TopkPred* pred, uint32_t row, uint32_t* lo, uint32_t* hi) {
+__device__ __forceinline__ bool predicted_band(const TopkPred* pred, uint32_t row, uint32_t* lo, uint32_t* hi,
+                                               uint32_t* centre = nullptr) {
   if (!pred) return false;
   const TopkPred p = pred[row];
   if (p.magic != kPredMagic || (p.tau_last | p.tau_prev) >> 31) return false;
   long long trend = (long long)p.tau_last - (long long)p.tau_prev;
   trend = max((long long)-kMaxTrend, min((long long)kMaxTrend, trend));
   const long long c = (long long)p.tau_last + trend;
-  const long long half = max((long long)kBandHalf, (trend < 0 ? -trend : trend) / 4);
+  const long long err = min(p.err, kMaxErr);
+  const long long half = max(max((long long)kBandHalf, 2 * err), (trend < 0 ? -trend : trend) / 4);
+  if (centre) *centre = (uint32_t)max(0ll, min(0x7fffffffll, c));
   const long long l = min((long long)p.tau_last, c) - half, h = max((long long)p.tau_last, c) + half;
   *lo = (uint32_t)max(0ll, l);
   *hi = (uint32_t)min(0x7fffffffll, h);
@@ -560,13 +567,19 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
     st->r = s_out[1];
     st->k_rem = s_out[1];
     if (pred) {
-      uint32_t lo = 1, hi = 0;
-      const bool had = predicted_band(pred, row, &lo, &hi);
+      uint32_t lo = 1, hi = 0, centre = 0;
+      const bool had = predicted_band(pred, row, &lo, &hi, &centre);
       TopkPred np;
       np.magic = kPredMagic;
       np.tau_prev = had ? pred[row].tau_last : tau;
       np.tau_last = tau;
-      np.pad = 0;
+      if (had) {
+        const uint32_t e = tau > centre ? tau - centre : centre - tau;
+        const uint32_t old = min(pred[row].err, kMaxErr);
+        np.err = min(kMaxErr, max(old - (old >> 2), e));
+      } else {
+        np.err = kFirstErr;
+      }
       pred[row] = np;
     }
   }
