@@ -218,7 +218,11 @@ def run_ours(args, wl):
     K, W = args.steps, max(args.warmup, 3)
 
     ds = DoubleSqueeze.for_workload(wl, dev)
-    ring = [make_gradients(wl, t, device=dev) for t in range(2)]     # distinct g_t, resident in HBM
+    # distinct g_t resident in HBM: a fresh draw for every step where 48 GB hold them, else a ring of
+    # as many as fit (a training run never sees the same gradient twice; a short ring makes the
+    # top-k threshold oscillate with the ring's period)
+    R = max(2, min(K + W, int(48e9 // (wl.n * wl.d * 4))))
+    ring = [make_gradients(wl, t, device=dev) for t in range(R)]
     need_flush = wl.n * wl.d * 8 <= 2 * 126e6
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
     stream = torch.cuda.current_stream(dev)
@@ -230,7 +234,7 @@ def run_ours(args, wl):
 
     # ---- device-resident timing
     for t in range(W):
-        ds.step(ring[t % 2], t)
+        ds.step(ring[t % R], t)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     sampler = ClockSampler(local)
     barrier()
@@ -247,7 +251,7 @@ def run_ours(args, wl):
         if need_flush:
             flush.fill_(t & 0xFF)
         ev[t][0].record(stream)
-        ds.worker_compress(ring[t % 2], W + t)
+        ds.worker_compress(ring[(W + t) % R], W + t)
         ev[t][1].record(stream)
         ds.server_aggregate_compress(W + t, fuse_apply=True)
         ev[t][2].record(stream)

@@ -45,7 +45,7 @@ constexpr uint32_t kSegWords = kThreads * kWordsPerThread;  // 1024 bitmap words
 constexpr uint32_t kSegElems = kSegWords * 32;     // 32768 entries
 constexpr uint64_t kTile = 4096;                   // entries a CTA handles per loop trip
 constexpr uint32_t kPredMagic = 0x70D1C7EDu;
-constexpr uint32_t kBandHalf = 1u << 16;           // least half-width of the band in key units (0.5 % of magnitude)
+constexpr uint32_t kBandHalf = 1u << 13;           // least half-width of the band in key units (0.07 % of magnitude)
 constexpr uint32_t kMaxErr = 1u << 21;             // widest extrapolation error followed (band: half an octave each way)
 constexpr uint32_t kFirstErr = kMaxErr;            // error assumed before any extrapolation has been checked
 constexpr int kMaxTrend = 1 << 20;                 // largest step-to-step drift that is extrapolated (9 %)
@@ -57,7 +57,7 @@ inline uint64_t round16(uint64_t b) { return (b + 15u) & ~uint64_t(15); }
 // Keys are monotone in log-magnitude (2^23 units per octave), so a threshold that drifts by a
 // steady factor moves by a steady key difference.  The band is the last threshold, extrapolated by
 // the last change (the drift itself changes slowly), widened on both sides by the largest of a
-// quarter of that change, 0.5 % of magnitude, and twice the recent extrapolation error (a decaying
+// quarter of that change, 0.07 % of magnitude, and twice the recent extrapolation error (a decaying
 // maximum kept beside the thresholds), so the band is wide while the error memories are still
 // filling and narrows once the threshold settles.
 // Candidates are the entries with lo <= key <= hi; returns false when there is no usable history.
@@ -97,45 +97,90 @@ __device__ __forceinline__ uint32_t octet_words4(const uint32_t (&nib)[4], uint3
   return u2 ? (recv2 | q << 16) : (q | recv2 << 16);
 }
 
-// Writes the candidates of one tile -- sel[j] bit k flags entry k of row j, whose key is
-// keys[4 j + k] and whose index is idx0[j] + k -- into the tile's own region of the list (kTile slots, enough for every entry of
-// the tile).  Slots are handed out by a shared-memory counter, one atomic per warp; the order
-// inside the region is irrelevant.  Called by all 32 lanes of every warp of the CTA.
-__device__ __forceinline__ void tile_append(uint2* region, uint32_t* s_count, const uint32_t (&keys)[16],
-                                            const uint32_t (&idx0)[4], const uint32_t (&sel)[4], uint32_t lane) {
-  const uint32_t c = __popc(sel[0]) + __popc(sel[1]) + __popc(sel[2]) + __popc(sel[3]);
-  if (__ballot_sync(0xffffffffu, c != 0) == 0) return;
-  uint32_t incl = c;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= (uint32_t)o) incl += y;
-  }
-  const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-  uint32_t base = 0;
-  if (lane == 0) base = atomicAdd(s_count, total);
-  base = __shfl_sync(0xffffffffu, base, 0);
-  uint32_t pos = base + incl - c;
-#pragma unroll
-  for (int j = 0; j < 4; ++j)
-#pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if ((sel[j] >> k) & 1u) {
-        if (pos < kTile) region[pos] = make_uint2(keys[4 * j + k], idx0[j] + k);
-        ++pos;
-      }
-}
-
 // ================================================================ list pipeline
 
+// ---------------------------------------------------------------- marking a tile
+// One 4096-entry tile held by a 256-thread CTA: thread t has the float4 groups at entries
+// base + (j * 256 + t) * 4, j < 4 (cnt[j] of each inside the vector).  Every entry with key >= lo
+// is "listed": its (value bits, index) goes to the tile's own region of the list (kTile slots,
+// enough for the whole tile, so CTAs never share a region), in index order.  Listed entries with
+// key > hi are certain to be kept; they are counted and already zeroed in the residual (their
+// value survives in the list).  info receives (listed, above hi, 0, 0); the two zeros are the
+// counters classify fills.  s_tot: one uint4 per warp, free for reuse after the call's barrier
+// has been passed by all threads a second time.  Called by all threads of the CTA.
+template <bool FULL>
+__device__ __forceinline__ void mark_tile(const float4 (&v)[4], const uint32_t (&cnt)[4], uint64_t base, uint32_t key_lo,
+                                          uint32_t key_hi, float* out_row, uint2* region, uint4* info, uint4* s_tot) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5;
+  uint32_t sel[4], kept = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    sel[j] = 0;
+    const uint32_t k0 = key_of(v[j].x), k1 = key_of(v[j].y), k2 = key_of(v[j].z), k3 = key_of(v[j].w);
+    if (max(max(k0, k1), max(k2, k3)) >= key_lo) {
+      // only groups with a listed entry get in here
+      uint32_t gt = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint32_t key = key_of(compc(v[j], k));
+        if (FULL || (uint32_t)k < cnt[j]) {  // entries past the end were loaded as +0 and are no entries
+          if (key >= key_lo) sel[j] |= 1u << k;
+          if (key > key_hi) gt |= 1u << k;
+        }
+      }
+      if (gt) {
+        float* o = out_row + base + (uint64_t)(j * kThreads + tid) * 4u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((gt >> k) & 1u) o[k] = 0.f;  // delta = v - Q[v] at an entry that is kept whatever tau turns out to be
+        kept += __popc(gt);
+      }
+    }
+  }
+  // index order is (j, thread, k): per-j counts, packed two to a word, scanned over the warp
+  const uint32_t ca = __popc(sel[0]) | (__popc(sel[1]) << 16), cb = __popc(sel[2]) | (__popc(sel[3]) << 16);
+  uint32_t ia = ca, ib = cb;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t ya = __shfl_up_sync(0xffffffffu, ia, o), yb = __shfl_up_sync(0xffffffffu, ib, o);
+    if (lane >= (uint32_t)o) { ia += ya; ib += yb; }
+  }
+  kept = __reduce_add_sync(0xffffffffu, kept);
+  if (lane == 31) s_tot[wrp] = make_uint4(ia, ib, kept, 0u);
+  __syncthreads();
+  uint32_t sa = 0, sb = 0, pa = 0, pb = 0, kt = 0;
+#pragma unroll
+  for (uint32_t w = 0; w < kThreads / 32; ++w) {
+    const uint4 t = s_tot[w];
+    if (w < wrp) { pa += t.x; pb += t.y; }
+    sa += t.x; sb += t.y; kt += t.z;
+  }
+  // a field holds at most 1024 (entries of one j in the tile), so the 16-bit fields never carry
+  const uint32_t t0 = sa & 0xFFFFu, t1 = sa >> 16, t2 = sb & 0xFFFFu, t3 = sb >> 16;
+  const uint32_t ea = pa + ia - ca, eb = pb + ib - cb;
+  uint32_t pos[4] = {ea & 0xFFFFu, t0 + (ea >> 16), t0 + t1 + (eb & 0xFFFFu), t0 + t1 + t2 + (eb >> 16)};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (sel[j]) {
+      const uint32_t i0 = (uint32_t)base + (uint32_t)(j * kThreads + tid) * 4u;  // indices fit 32 bits: d < 2^32
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if ((sel[j] >> k) & 1u) {
+          if (pos[j] < kTile) region[pos[j]] = make_uint2(__float_as_uint(compc(v[j], k)), i0 + k);
+          ++pos[j];
+        }
+    }
+  }
+  if (tid == 0) *info = make_uint4(t0 + t1 + t2 + t3, kt, 0u, 0u);
+}
+
 // ---------------------------------------------------------------- pass1
-// One CTA per 4096-entry tile; the grid covers the padded bitmap extent.  tile_info[tile] receives
-// (candidates written, entries above the band).
+// One CTA per 4096-entry tile: v = source, written over delta; with a predicted band the tile is
+// marked while v is still in registers.
 template <int SRC, bool FULL>
 __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, uint64_t base, float* out_row, bool marking,
-                                           uint32_t key_lo, uint32_t key_hi, uint32_t* bm_row, uint2* region,
-                                           uint32_t* s_count, uint32_t* s_kept) {
-  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+                                           uint32_t key_lo, uint32_t key_hi, uint2* region, uint4* info, uint4* s_tot) {
+  const uint32_t tid = threadIdx.x;
   const uint64_t d = src.d;
   float4 v[4];
   uint32_t cnt[4];
@@ -180,63 +225,25 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
       }
     }
   }
-  if (!marking) return;
-  uint32_t ngt[4], ncand[4], idx0[4], keys[16];
-  uint32_t kept = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    ngt[j] = 0;
-    ncand[j] = 0;
-    idx0[j] = (uint32_t)base + (uint32_t)(j * kThreads + tid) * 4u;  // indices fit 32 bits: d < 2^32
-    keys[4 * j] = key_of(v[j].x); keys[4 * j + 1] = key_of(v[j].y);
-    keys[4 * j + 2] = key_of(v[j].z); keys[4 * j + 3] = key_of(v[j].w);
-    if (max(max(keys[4 * j], keys[4 * j + 1]), max(keys[4 * j + 2], keys[4 * j + 3])) >= key_lo) {
-      // only the kept entries and the candidates get in here
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (FULL || (uint32_t)k < cnt[j]) {  // entries past the end were loaded as +0 and are no entries
-          if (keys[4 * j + k] > key_hi) ngt[j] |= 1u << k;
-          else if (keys[4 * j + k] >= key_lo) ncand[j] |= 1u << k;
-        }
-      }
-    }
-    kept += __popc(ngt[j]);
-  }
-  const uint32_t wg = octet_words4(ngt, lane);
-  const uint32_t r = lane & 7u;
-  if (r < 4) bm_row[(base >> 5) + r * 32u + (tid >> 3)] = wg;
-  tile_append(region, s_count, keys, idx0, ncand, lane);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
-  if (lane == 0 && kept) atomicAdd(s_kept, kept);
+  if (marking) mark_tile<FULL>(v, cnt, base, key_lo, key_hi, out_row, region, info, s_tot);
 }
 
 template <int SRC>
-__global__ void __launch_bounds__(kThreads) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred,
-                                                         uint32_t* bm_gt, uint64_t bm_stride, uint2* list, uint64_t cap,
-                                                         uint2* tile_info, uint64_t ntile) {
-  __shared__ uint32_t s_count, s_kept;
-  const uint32_t tid = threadIdx.x, row = blockIdx.y;
+__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER || SRC == SRC_SRV_TOPK ? 5 : 1) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred, uint2* list,
+                                                         uint64_t cap, uint4* tile_info, uint64_t ntile) {
+  __shared__ uint4 s_tot[kThreads / 32];
+  const uint32_t row = blockIdx.y;
   const uint64_t tile = blockIdx.x, base = tile * kTile;
   const uint64_t d = src.d;
   uint32_t key_lo = 1, key_hi = 0;
   const bool marking = predicted_band(pred, row, &key_lo, &key_hi);
-  if (!marking && base >= d) return;  // padding tile and no bitmap to clear
-  if (marking) {
-    if (tid == 0) { s_count = 0; s_kept = 0; }
-    __syncthreads();
-  }
   float* out_row = v_out + (uint64_t)row * d;
-  uint32_t* bm_row = bm_gt + (uint64_t)row * bm_stride;
   uint2* region = list + (uint64_t)row * cap + base;
+  uint4* info = tile_info + (uint64_t)row * ntile + tile;
   if (src.vec && base + kTile <= d) {
-    pass1_tile<SRC, true>(src, row, base, out_row, marking, key_lo, key_hi, bm_row, region, &s_count, &s_kept);
+    pass1_tile<SRC, true>(src, row, base, out_row, marking, key_lo, key_hi, region, info, s_tot);
   } else {
-    pass1_tile<SRC, false>(src, row, base, out_row, marking, key_lo, key_hi, bm_row, region, &s_count, &s_kept);
-  }
-  if (marking && base < d) {
-    __syncthreads();
-    if (tid == 0) tile_info[(uint64_t)row * ntile + tile] = make_uint2(min(s_count, (uint32_t)kTile), s_kept);
+    pass1_tile<SRC, false>(src, row, base, out_row, marking, key_lo, key_hi, region, info, s_tot);
   }
 }
 
@@ -301,19 +308,34 @@ __global__ void __launch_bounds__(1024) k_topk_pick1(uint32_t* hist, TopkState* 
   st->tb1 = s_out[0];
   st->k_rem = s_out[1];
   st->need_mark = 1;
+  st->zeroed_above = (s_out[0] << 19) | 0x7FFFFu;  // mark zeroes the bins above the threshold bin
 }
 
 // ---------------------------------------------------------------- full histogram (after a miss)
-__global__ void __launch_bounds__(kThreads) k_topk_hist(const float* v_in, uint64_t d, int vec, const TopkState* state,
-                                                        uint32_t* hist) {
+// If pass1 marked with a band that then missed, the entries it zeroed come back first: a tile's
+// region holds only entries of that tile, so the CTA that histograms a tile restores it itself.
+__global__ void __launch_bounds__(kThreads) k_topk_hist(float* v_io, uint64_t d, int vec, const TopkState* state,
+                                                        const TopkPred* pred, const uint2* list, uint64_t cap,
+                                                        const uint4* tile_info, uint32_t* hist) {
   __shared__ uint32_t s_hist[kBins1];
   const uint32_t tid = threadIdx.x, row = blockIdx.y;
   if (!state[row].need_full) return;
   for (uint32_t b = tid; b < kBins1; b += kThreads) s_hist[b] = 0;
-  __syncthreads();
-  const float* vrow = v_in + (uint64_t)row * d;
+  uint32_t band_lo = 1, band_hi = 0;
+  const bool marked = predicted_band(pred, row, &band_lo, &band_hi);  // what pass1 saw: pred changes only at the end
+  float* vrow = v_io + (uint64_t)row * d;
   const uint64_t ntile = (d + kTile - 1) / kTile;
   for (uint64_t tile = blockIdx.x; tile < ntile; tile += gridDim.x) {
+    if (marked) {
+      const uint4 info = tile_info[(uint64_t)row * ntile + tile];
+      const uint32_t n = min(info.x, (uint32_t)kTile);
+      const uint2* region = list + (uint64_t)row * cap + tile * kTile;
+      for (uint32_t i = tid; i < n; i += kThreads) {
+        const uint2 e = region[i];
+        if ((e.x & 0x7fffffffu) > band_hi && (e.y >> 12) == tile && e.y < d) vrow[e.y] = __uint_as_float(e.x);
+      }
+    }
+    __syncthreads();  // restored entries are read below by other threads; also orders s_hist clearing
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const uint64_t e = tile * kTile + (uint64_t)(j * kThreads + tid) * 4u;
@@ -341,27 +363,23 @@ __global__ void __launch_bounds__(kThreads) k_topk_hist(const float* v_in, uint6
 }
 
 // ---------------------------------------------------------------- mark (after a miss)
-// Bitmap of the entries above the exact threshold bin and the list of those inside it.  A small
-// grid strides over the tiles; every bitmap word up to the padded end is written.
-__global__ void __launch_bounds__(kThreads) k_topk_mark(const float* v_in, uint64_t d, int vec, const TopkState* state,
-                                                        uint32_t* bm_gt, uint64_t bm_stride, uint64_t padded, uint2* list,
-                                                        uint64_t cap, uint2* tile_info, uint64_t ntile) {
-  __shared__ uint32_t s_count;
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
+// Rebuilds the tile regions for the exact threshold bin: entries in bins above it are kept (and
+// zeroed), entries inside it are the candidates.  A small grid strides over the tiles.
+__global__ void __launch_bounds__(kThreads) k_topk_mark(float* v_io, uint64_t d, int vec, const TopkState* state, uint2* list,
+                                                        uint64_t cap, uint4* tile_info, uint64_t ntile) {
+  __shared__ uint4 s_tot[kThreads / 32];
+  const uint32_t tid = threadIdx.x, row = blockIdx.y;
   if (!state[row].need_mark) return;
-  const uint32_t tb = state[row].tb1;
-  const float* vrow = v_in + (uint64_t)row * d;
-  const uint64_t tiles = padded / kTile;
-  for (uint64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+  const uint32_t lo = state[row].tb1 << 19, hi = lo | 0x7FFFFu;
+  float* vrow = v_io + (uint64_t)row * d;
+  for (uint64_t tile = blockIdx.x; tile < ntile; tile += gridDim.x) {
     const uint64_t base = tile * kTile;
-    if (tid == 0) s_count = 0;
-    __syncthreads();
+    const bool full = vec && base + kTile <= d;
     float4 v[4];
-    uint32_t cnt[4], idx0[4];
+    uint32_t cnt[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const uint64_t e = base + (uint64_t)(j * kThreads + tid) * 4u;
-      idx0[j] = (uint32_t)e;
       cnt[j] = e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u;
       v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (cnt[j]) {
@@ -374,94 +392,137 @@ __global__ void __launch_bounds__(kThreads) k_topk_mark(const float* v_in, uint6
         }
       }
     }
-    uint32_t ngt[4], ncand[4], keys[16];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      ngt[j] = 0;
-      ncand[j] = 0;
-      keys[4 * j] = key_of(v[j].x); keys[4 * j + 1] = key_of(v[j].y);
-      keys[4 * j + 2] = key_of(v[j].z); keys[4 * j + 3] = key_of(v[j].w);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const uint32_t bin = keys[4 * j + k] >> 19;
-        const bool in = (uint32_t)k < cnt[j];
-        ngt[j] |= (in && bin > tb ? 1u : 0u) << k;
-        ncand[j] |= (in && bin == tb ? 1u : 0u) << k;
-      }
-    }
-    const uint32_t wg = octet_words4(ngt, lane);
-    const uint32_t r = lane & 7u;
-    if (r < 4) bm_gt[(uint64_t)row * bm_stride + tile * (kTile / 32) + r * 32u + (tid >> 3)] = wg;
-    if (base < d) tile_append(list + (uint64_t)row * cap + base, &s_count, keys, idx0, ncand, lane);
-    __syncthreads();
-    if (tid == 0 && base < d) tile_info[(uint64_t)row * ntile + tile] = make_uint2(min(s_count, (uint32_t)kTile), 0u);
+    uint2* region = list + (uint64_t)row * cap + base;
+    uint4* info = tile_info + (uint64_t)row * ntile + tile;
+    if (full) mark_tile<true>(v, cnt, base, lo, hi, vrow, region, info, s_tot);
+    else mark_tile<false>(v, cnt, base, lo, hi, vrow, region, info, s_tot);
+    __syncthreads();  // s_tot is written again for the next tile
   }
 }
 
 // ---------------------------------------------------------------- tile regions -> dense list
-// Copies the candidates out of the per-tile regions into one dense list per vector (order
-// irrelevant).  A warp takes eight tiles at a time: one read of their counts, one reservation in
-// the dense list for all eight, then the regions.  With HIST the top-12-bit histogram of the keys
-// is counted on the way (into s_hist) and the return value is this thread's share of the
-// "entries above the band" counts.  Called by whole CTAs.
+// Exclusive prefix of one value per thread over the CTA (blockDim a multiple of 32, at most 1024).
+// s_warp: 33 words.  *total = sum over the CTA.  Ends with a barrier; s_warp may be reused after
+// the next barrier the caller passes.
+__device__ __forceinline__ uint32_t cta_excl_scan(uint32_t val, uint32_t* s_warp, uint32_t* total) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, warps = blockDim.x >> 5;
+  uint32_t incl = val;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= (uint32_t)o) incl += y;
+  }
+  if (lane == 31) s_warp[wrp] = incl;
+  __syncthreads();
+  if (wrp == 0) {
+    const uint32_t w = lane < warps ? s_warp[lane] : 0u;
+    uint32_t wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= (uint32_t)o) wi += y;
+    }
+    s_warp[lane] = wi - w;
+    if (lane == 31) s_warp[32] = wi;
+  }
+  __syncthreads();
+  *total = s_warp[32];
+  return s_warp[wrp] + incl - val;
+}
+
+// One batch of up to 64 region entries, two neighbours per lane (q.x, q.y = first entry, q.z, q.w =
+// second): those not above the band (key <= fhi) are the candidates; they go to the dense list as
+// (key, index) from slot `run` on, in entry order.
 template <bool HIST>
-__device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint2* info, uint64_t ntile, uint2* drow,
-                                                 uint32_t* dense_count, uint32_t* s_hist) {
-  const uint32_t tid = threadIdx.x, lane = tid & 31u;
-  const uint32_t warps = blockDim.x >> 5;
+__device__ __forceinline__ void put_candidates(uint4 q, bool valid0, bool valid1, uint32_t fhi, uint32_t& run, uint2* drow,
+                                               uint64_t cap, uint32_t* s_hist, uint32_t lane) {
+  const uint32_t key0 = q.x & 0x7fffffffu, key1 = q.z & 0x7fffffffu;
+  const bool is0 = valid0 && key0 <= fhi, is1 = valid1 && key1 <= fhi;
+  const uint32_t b0 = __ballot_sync(0xffffffffu, is0), b1 = __ballot_sync(0xffffffffu, is1);
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t pos = run + __popc(b0 & lt) + __popc(b1 & lt);
+  if (is0) {
+    if (pos < cap) drow[pos] = make_uint2(key0, q.y);
+    if (HIST) atomicAdd(&s_hist[key0 >> 19], 1u);
+    ++pos;
+  }
+  if (is1) {
+    if (pos < cap) drow[pos] = make_uint2(key1, q.w);
+    if (HIST) atomicAdd(&s_hist[key1 >> 19], 1u);
+  }
+  run += __popc(b0) + __popc(b1);
+}
+
+// The first / a later 64-entry batch of a region of n entries (regions are 16-byte aligned).
+__device__ __forceinline__ uint4 region_batch(const uint2* region, uint32_t i0, uint32_t n, uint32_t lane) {
+  return i0 + 2u * lane < n ? reinterpret_cast<const uint4*>(region)[(i0 >> 1) + lane] : make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Copies the candidates out of the tile regions into one dense list per vector; a tile's
+// candidates stay together and in index order, the tiles of a CTA follow one another.  Each CTA
+// takes a contiguous run of tiles; the tile_info counts say how many candidates each region
+// holds, so one prefix sum per CTA and ONE reservation in the dense list place them all (the
+// counters of all vectors share a cache line, and atomics on one line are served one after the
+// other).  With HIST the top-12-bit histogram of the keys is counted on the way.  Returns this
+// thread's share of the "entries above the band" counts.  s_n, s_off: blockDim words each;
+// s_warp: 34 words.  Called by whole CTAs.
+template <bool HIST>
+__device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint4* info, uint64_t ntile, uint2* drow,
+                                                 uint64_t cap, uint32_t* dense_count, uint32_t fhi, uint32_t* s_hist,
+                                                 uint32_t* s_n, uint32_t* s_off, uint32_t* s_warp) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, nthr = blockDim.x, warps = nthr >> 5;
+  const uint64_t per = (ntile + gridDim.x - 1) / gridDim.x;
+  const uint64_t c0 = (uint64_t)blockIdx.x * per, c1 = min(ntile, c0 + per);
   uint32_t kept = 0;
-  const uint64_t wstep = (uint64_t)gridDim.x * warps * 8;
-  for (uint64_t t0 = ((uint64_t)blockIdx.x * warps + (tid >> 5)) * 8; t0 < ntile; t0 += wstep) {
-    uint2 mine = make_uint2(0, 0);
-    if (lane < 8 && t0 + lane < ntile) mine = info[t0 + lane];
-    mine.x = min(mine.x, (uint32_t)kTile);
-    kept += mine.y;
-    uint32_t incl = mine.x;
+  for (uint64_t r0 = c0; r0 < c1; r0 += nthr) {
+    uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+    if (r0 + tid < c1) mine = info[r0 + tid];
+    const uint32_t n = min(mine.x, (uint32_t)kTile), above = min(mine.y, n);
+    kept += above;
+    uint32_t total;
+    const uint32_t excl = cta_excl_scan(n - above, s_warp, &total);
+    s_n[tid] = n;
+    s_off[tid] = excl;
+    if (tid == 0) s_warp[33] = total ? atomicAdd(dense_count, total) : 0u;
+    __syncthreads();
+    const uint32_t base = s_warp[33];
+    const uint32_t ntl = (uint32_t)min((uint64_t)nthr, c1 - r0);
+    // a warp takes four tiles at a time and has the first 64 entries of each in flight at once
+    for (uint32_t i = wrp; i < ntl; i += 4 * warps) {
+      uint32_t nn[4];
+      uint4 q[4];
 #pragma unroll
-    for (int o = 1; o < 8; o <<= 1) {
-      const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= (uint32_t)o) incl += y;
-    }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 7);
-    if (total == 0) continue;
-    uint32_t base = 0;
-    if (lane == 0) base = atomicAdd(dense_count, total);
-    base = __shfl_sync(0xffffffffu, base, 0);
-    // the first 32 entries of all eight regions are fetched before any is used
-    uint2 first[8];
-    uint32_t ns[8], offs[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      ns[u] = __shfl_sync(0xffffffffu, mine.x, u);
-      offs[u] = __shfl_sync(0xffffffffu, incl - mine.x, u);
-      first[u] = make_uint2(0u, 0u);
-      if (lane < ns[u]) first[u] = lrow[(t0 + u) * kTile + lane];
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      if (lane < ns[u]) {
-        drow[(uint64_t)base + offs[u] + lane] = first[u];
-        if (HIST) atomicAdd(&s_hist[(first[u].x >> 19) & 0xFFFu], 1u);
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t iu = i + u * warps;
+        nn[u] = iu < ntl ? s_n[iu] : 0u;
+        q[u] = region_batch(lrow + (r0 + iu) * kTile, 0, nn[u], lane);  // no read where nn[u] == 0
       }
-      const uint2* reg = lrow + (t0 + u) * kTile;
-      for (uint32_t i = lane + 32; i < ns[u]; i += 32) {
-        const uint2 e = reg[i];
-        drow[(uint64_t)base + offs[u] + i] = e;
-        if (HIST) atomicAdd(&s_hist[(e.x >> 19) & 0xFFFu], 1u);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (nn[u] == 0) continue;
+        const uint32_t iu = i + u * warps;
+        const uint2* reg = lrow + (r0 + iu) * kTile;
+        uint32_t run = base + s_off[iu];
+        put_candidates<HIST>(q[u], 2u * lane < nn[u], 2u * lane + 1u < nn[u], fhi, run, drow, cap, s_hist, lane);
+        for (uint32_t i0 = 64; i0 < nn[u]; i0 += 64)
+          put_candidates<HIST>(region_batch(reg, i0, nn[u], lane), i0 + 2u * lane < nn[u], i0 + 2u * lane + 1u < nn[u], fhi,
+                               run, drow, cap, s_hist, lane);
       }
     }
+    __syncthreads();  // s_n, s_off and s_warp are rewritten by the next round
   }
   return kept;
 }
 
-// After a miss: the list that mark rebuilt, made dense.
-__global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, uint64_t cap, const uint2* tile_info,
+// After a miss: the candidates of the regions that mark rebuilt, made dense.
+__global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, uint64_t cap, const uint4* tile_info,
                                                            uint64_t ntile, uint2* dense, uint32_t* dense_count,
                                                            const TopkState* state) {
+  __shared__ uint32_t s_n[kThreads], s_off[kThreads], s_warp[34];
   const uint32_t row = blockIdx.y;
   if (!state[row].need_mark) return;
-  gather_tiles<false>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile, dense + (uint64_t)row * cap,
-                      &dense_count[row], nullptr);
+  gather_tiles<false>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile, dense + (uint64_t)row * cap, cap,
+                      &dense_count[row], (state[row].tb1 << 19) | 0x7FFFFu, nullptr, s_n, s_off, s_warp);
 }
 
 // ---------------------------------------------------------------- list histogram + pick
@@ -471,27 +532,31 @@ __global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, ui
 // vector's global histogram; the CTA that finishes last (a ticket counter, no waiting) picks the
 // digit and clears histogram and ticket.
 template <int LEVEL>
-__global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t cap, const uint2* tile_info, uint64_t ntile,
+__global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t cap, const uint4* tile_info, uint64_t ntile,
                                                      uint2* dense, uint32_t* dense_count, uint32_t* kept_count,
                                                      TopkState* state, uint32_t* hist, uint32_t* done, uint32_t k,
                                                      TopkPred* pred) {
   __shared__ uint32_t s_hist[kBins1];
-  __shared__ uint32_t s_warp[32], s_out[3];
-  __shared__ uint32_t s_last;
+  __shared__ uint32_t s_warp[34], s_out[3];
+  __shared__ uint32_t s_last, s_kept;
   constexpr uint32_t NB = LEVEL == 3 ? 128u : 4096u;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
-  const uint2* lrow = list + (uint64_t)row * cap;
-  const uint2* info = tile_info + (uint64_t)row * ntile;
   TopkState* st = state + row;
   uint32_t band_lo = 1, band_hi = 0;
   // LEVEL 1 reads what pass1 wrote, which exists only if pass1 had a band to work with
   const bool readable = LEVEL != 1 || predicted_band(pred, row, &band_lo, &band_hi);
   const uint32_t tb1 = st->tb1, top24 = (st->tb1 << 12) | st->tb2;
   for (uint32_t b = tid; b < NB; b += 1024) s_hist[b] = 0;
+  if (tid == 0) s_kept = 0;
   __syncthreads();
-  uint32_t kept = 0;
-  if (LEVEL == 1) {
-    if (readable) kept = gather_tiles<true>(lrow, info, ntile, dense + (uint64_t)row * cap, &dense_count[row], s_hist);
+  if constexpr (LEVEL == 1) {
+    __shared__ uint32_t s_n[1024], s_off[1024];
+    uint32_t kept = 0;
+    if (readable)
+      kept = gather_tiles<true>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile,
+                                dense + (uint64_t)row * cap, cap, &dense_count[row], band_hi, s_hist, s_n, s_off, s_warp);
+    kept = __reduce_add_sync(0xffffffffu, kept);
+    if (lane == 0 && kept) atomicAdd(&s_kept, kept);
   } else {
     const uint2* drow = dense + (uint64_t)row * cap;
     const uint64_t n = min((uint64_t)dense_count[row], cap);
@@ -513,17 +578,13 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
       }
     }
   }
-  if (LEVEL == 1) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
-    if (lane == 0 && kept) atomicAdd(&kept_count[row], kept);
-  }
   __syncthreads();
   uint32_t* h = hist + (uint64_t)row * kBins1;
   for (uint32_t b = tid; b < NB; b += 1024) {
     const uint32_t c = s_hist[b];
     if (c) atomicAdd(&h[b], c);
   }
+  if (LEVEL == 1 && tid == 0 && s_kept) atomicAdd(&kept_count[row], s_kept);
   __threadfence();
   __syncthreads();
   if (tid == 0) s_last = atomicAdd(&done[row], 1u) == gridDim.x - 1 ? 1u : 0u;
@@ -546,15 +607,15 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
   if (tid != 0) return;
   if (LEVEL == 1) {
     // the prediction holds iff the k-th largest entry is one of the listed candidates
-    uint32_t lo = 1, hi = 0;
-    const bool hit = predicted_band(pred, row, &lo, &hi) && want >= 1 && want <= s_out[2];
+    const bool hit = readable && want >= 1 && want <= s_out[2];
     if (hit) {
       st->tb1 = s_out[0];
       st->k_rem = s_out[1];
       st->need_full = 0;
       st->need_mark = 0;
+      st->zeroed_above = band_hi;
     } else {
-      st->need_full = 1;  // hist, pick, mark and compact rebuild bitmap and list for the exact bin
+      st->need_full = 1;  // hist, pick, mark and compact rebuild the regions and the list for the exact bin
       st->need_mark = 1;
       dense_count[row] = 0;
     }
@@ -586,20 +647,21 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
 }
 
 // ---------------------------------------------------------------- classify
-// Candidates above tau join the kept bitmap; candidates equal to tau are set in the tie bitmap
-// (which the launcher cleared).  Candidate bits are never set in bm_gt beforehand, so the ORs
-// commute with nothing else.
+// Per tile, how many of its candidates lie above tau (z) and how many equal it (w): the counters
+// pass1 / mark left at zero beside the tile's counts.  A tile's candidates are neighbours in the
+// dense list, so the lanes of a warp that count for the same counter send one atomic between
+// them.  Integer atomics: order-free.
 __global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* dense, const uint32_t* dense_count, uint64_t cap,
-                                                            const TopkState* state, uint32_t* bm_gt, uint32_t* bm_tie,
-                                                            uint64_t bm_stride) {
-  const uint32_t row = blockIdx.y;
+                                                            const TopkState* state, uint4* tile_info, uint64_t ntile) {
+  const uint32_t row = blockIdx.y, lane = threadIdx.x & 31u;
   const uint2* drow = dense + (uint64_t)row * cap;
   const uint64_t n = min((uint64_t)dense_count[row], cap);
   const uint32_t tau = state[row].tau;
-  uint32_t* g = bm_gt + (uint64_t)row * bm_stride;
-  uint32_t* t = bm_tie + (uint64_t)row * bm_stride;
+  uint32_t* counters = reinterpret_cast<uint32_t*>(tile_info + (uint64_t)row * ntile);
   const uint64_t step = (uint64_t)gridDim.x * kThreads * 4;
-  for (uint64_t i0 = (uint64_t)blockIdx.x * kThreads * 4 + threadIdx.x; i0 < n; i0 += step) {
+  // the loop bound is the same for all lanes of a warp (i0 - threadIdx.x is), as match needs
+  for (uint64_t c0 = (uint64_t)blockIdx.x * kThreads * 4; c0 < n; c0 += step) {
+    const uint64_t i0 = c0 + threadIdx.x;
     uint2 e[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -608,35 +670,80 @@ __global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* dense, 
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      if (i0 + (uint64_t)u * kThreads >= n) continue;
-      if (e[u].x > tau) atomicOr(&g[e[u].y >> 5], 1u << (e[u].y & 31u));
-      else if (e[u].x == tau) atomicOr(&t[e[u].y >> 5], 1u << (e[u].y & 31u));
+      const uint64_t t = e[u].y >> 12;
+      const bool live = i0 + (uint64_t)u * kThreads < n && t < ntile && e[u].x >= tau;
+      // word index of the counter inside the vector's tile_info: .z for "above", .w for "equal"
+      const uint32_t word = live ? (uint32_t)t * 4u + (e[u].x > tau ? 2u : 3u) : 0xFFFFFFFFu;
+      const uint32_t peers = __match_any_sync(0xffffffffu, word);
+      if (live && lane == (uint32_t)__ffs(peers) - 1u) atomicAdd(&counters[word], (uint32_t)__popc(peers));
     }
   }
 }
 
-// ---------------------------------------------------------------- count
-// Population counts per segment (x: kept, y: ties).
-__global__ void __launch_bounds__(kThreads) k_topk_count(const uint32_t* bm_gt, const uint32_t* bm_tie, uint64_t bm_stride,
-                                                         uint2* seg_cnt, uint64_t nseg) {
-  __shared__ uint32_t s_gt[kThreads / 32], s_tie[kThreads / 32];
+// ---------------------------------------------------------------- emit from the tile regions
+// A warp per tile.  The region lists, in index order, every entry that can be kept; the scan gave
+// the tile its first output slot (and the number of ties before it), so a ballot per 32 entries
+// places them.  Entries above `zeroed_above` were zeroed in the residual when they were listed;
+// the kept candidates are zeroed here (delta = v - Q[v], Eq. 3).
+__global__ void __launch_bounds__(kThreads) k_topk_emit_list(float* v_io, uint64_t d, const TopkState* state, const uint2* list,
+                                                             uint64_t cap, const uint4* tile_info, const uint2* tile_pre,
+                                                             uint64_t ntile, uint8_t* payload, uint64_t payload_stride,
+                                                             uint64_t off_idx, uint64_t off_val, uint32_t k, float* x,
+                                                             float gamma) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
-  const uint64_t at = (uint64_t)row * bm_stride + (uint64_t)blockIdx.x * kSegWords + tid * kWordsPerThread;
-  const uint4 g4 = *reinterpret_cast<const uint4*>(bm_gt + at);
-  const uint4 t4 = *reinterpret_cast<const uint4*>(bm_tie + at);
-  uint32_t ng = __popc(g4.x) + __popc(g4.y) + __popc(g4.z) + __popc(g4.w);
-  uint32_t nt = __popc(t4.x) + __popc(t4.y) + __popc(t4.z) + __popc(t4.w);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    ng += __shfl_xor_sync(0xffffffffu, ng, o);
-    nt += __shfl_xor_sync(0xffffffffu, nt, o);
-  }
-  if (lane == 0) { s_gt[tid >> 5] = ng; s_tie[tid >> 5] = nt; }
-  __syncthreads();
-  if (tid == 0) {
-    uint32_t a = 0, b = 0;
-    for (uint32_t i = 0; i < kThreads / 32; ++i) { a += s_gt[i]; b += s_tie[i]; }
-    seg_cnt[(uint64_t)row * nseg + blockIdx.x] = make_uint2(a, b);
+  const uint64_t tile = (uint64_t)blockIdx.x * (kThreads / 32) + (tid >> 5);
+  if (tile >= ntile) return;
+  const uint4 info = tile_info[(uint64_t)row * ntile + tile];
+  const uint32_t n = min(info.x, (uint32_t)kTile);
+  if (n == 0) return;
+  const uint2* region = list + (uint64_t)row * cap + tile * kTile;
+  uint4 q = region_batch(region, 0, n, lane);  // 64 entries per trip, two neighbours per lane
+  const uint2 pre = tile_pre[(uint64_t)row * ntile + tile];
+  const uint32_t tau = state[row].tau, r = state[row].r, zeroed_above = state[row].zeroed_above;
+  const bool ties = info.w != 0;  // the tile holds an entry equal to tau
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t ties_before = pre.y;
+  uint32_t run = pre.x + min(pre.y, r);
+  float* vrow = v_io + (uint64_t)row * d;
+  uint32_t* out_idx = reinterpret_cast<uint32_t*>(payload + (uint64_t)row * payload_stride + off_idx);
+  float* out_val = reinterpret_cast<float*>(payload + (uint64_t)row * payload_stride + off_val);
+  for (uint32_t i0 = 0; i0 < n; i0 += 64) {
+    const uint4 q_next = region_batch(region, i0 + 64, n, lane);
+    const bool valid0 = i0 + 2u * lane < n, valid1 = i0 + 2u * lane + 1u < n;
+    const uint32_t key0 = q.x & 0x7fffffffu, key1 = q.z & 0x7fffffffu;
+    bool sel0 = valid0 && key0 > tau, sel1 = valid1 && key1 > tau;
+    if (ties) {
+      // ties are kept lowest index first until r of them are in
+      const bool tie0 = valid0 && key0 == tau, tie1 = valid1 && key1 == tau;
+      const uint32_t b0 = __ballot_sync(0xffffffffu, tie0), b1 = __ballot_sync(0xffffffffu, tie1);
+      const uint32_t before = ties_before + __popc(b0 & lt) + __popc(b1 & lt);
+      if (tie0 && before < r) sel0 = true;
+      if (tie1 && before + (tie0 ? 1u : 0u) < r) sel1 = true;
+      ties_before += __popc(b0) + __popc(b1);
+    }
+    const uint32_t s0 = __ballot_sync(0xffffffffu, sel0), s1 = __ballot_sync(0xffffffffu, sel1);
+    uint32_t pos = run + __popc(s0 & lt) + __popc(s1 & lt);
+    if (sel0) {
+      const uint32_t j = q.y;
+      const float val = __uint_as_float(q.x);
+      if (pos < k) { out_idx[pos] = j; out_val[pos] = val; }  // pos < k whenever the counts are consistent
+      if (j < d) {
+        if (key0 <= zeroed_above) vrow[j] = 0.f;
+        if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
+      }
+      ++pos;
+    }
+    if (sel1) {
+      const uint32_t j = q.w;
+      const float val = __uint_as_float(q.z);
+      if (pos < k) { out_idx[pos] = j; out_val[pos] = val; }
+      if (j < d) {
+        if (key1 <= zeroed_above) vrow[j] = 0.f;
+        if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
+      }
+    }
+    run += __popc(s0) + __popc(s1);
+    q = q_next;
   }
 }
 
@@ -849,19 +956,36 @@ __global__ void __launch_bounds__(kThreads) k_topk_finalize(const float* v_in, u
 
 // ================================================================ shared tail
 
-// Exclusive prefix of the per-segment counts of one vector, in place; checks that exactly k
-// entries will be emitted.
-__global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, uint64_t nseg, TopkState* state, uint32_t k,
-                                                    uint32_t* dev_status) {
+// Exclusive prefix of the per-segment counts of one vector (in place), or with TILES of the
+// per-tile counts in tile_info (written to seg_cnt); checks that exactly k entries will be emitted.
+template <bool TILES>
+__global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4* tile_info, uint64_t nseg, TopkState* state,
+                                                    uint32_t k, uint32_t* dev_status) {
+  constexpr int ITEMS = TILES ? 8 : 1;  // consecutive counts per thread: one round trip to memory for all of them
   __shared__ uint2 s_warp[32];
   __shared__ uint2 s_carry;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.x;
   uint2* c = seg_cnt + (uint64_t)row * nseg;
   if (tid == 0) s_carry = make_uint2(0, 0);
   __syncthreads();
-  for (uint64_t base = 0; base < nseg; base += 1024) {
-    const uint64_t i = base + tid;
-    const uint2 mine = i < nseg ? c[i] : make_uint2(0, 0);
+  for (uint64_t base = 0; base < nseg; base += 1024 * ITEMS) {
+    uint2 item[ITEMS];
+    uint2 mine = make_uint2(0, 0);
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      const uint64_t i = base + (uint64_t)tid * ITEMS + u;
+      item[u] = make_uint2(0, 0);
+      if (i < nseg) {
+        if (TILES) {
+          const uint4 t = tile_info[(uint64_t)row * nseg + i];
+          item[u] = make_uint2(t.y + t.z, t.w);  // above the band + candidates above tau; candidates equal to tau
+        } else {
+          item[u] = c[i];
+        }
+      }
+      mine.x += item[u].x;
+      mine.y += item[u].y;
+    }
     uint2 incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -882,10 +1006,16 @@ __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, uint64_t nse
     }
     __syncthreads();
     const uint2 carry = s_carry;
-    const uint2 excl = make_uint2(carry.x + s_warp[wrp].x + incl.x - mine.x, carry.y + s_warp[wrp].y + incl.y - mine.y);
-    if (i < nseg) c[i] = excl;
+    uint2 excl = make_uint2(carry.x + s_warp[wrp].x + incl.x - mine.x, carry.y + s_warp[wrp].y + incl.y - mine.y);
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      const uint64_t i = base + (uint64_t)tid * ITEMS + u;
+      if (i < nseg) c[i] = excl;
+      excl.x += item[u].x;
+      excl.y += item[u].y;
+    }
     __syncthreads();
-    if (tid == 1023) s_carry = make_uint2(excl.x + mine.x, excl.y + mine.y);
+    if (tid == 1023) s_carry = excl;  // the prefix after this round's last item
     __syncthreads();
   }
   if (tid == 0) {
@@ -1012,11 +1142,12 @@ void topk_plan(uint64_t d, uint32_t rows, uint64_t k, bool with_list, TopkPlan* 
   p->off_hist = pos;       pos += (uint64_t)rows * kBins1 * 4;      // histogram and list counters are
   p->off_list_count = pos; pos = round16(pos + (uint64_t)rows * 12);  // tickets, kept counts: cleared by one memset
   p->off_state = pos;      pos = round16(pos + (uint64_t)rows * sizeof(TopkState));
-  p->off_bm_gt = pos;      pos = round16(pos + (uint64_t)rows * p->bm_stride * 4);
-  p->off_bm_eq = pos;      pos = round16(pos + (uint64_t)rows * p->bm_stride * 4);
-  p->off_seg = pos;        pos = round16(pos + (uint64_t)rows * p->nseg * sizeof(uint2));
+  // the bitmaps serve the pipeline without a list only; with a list the prefix runs over tiles
+  p->off_bm_gt = pos;      pos = round16(pos + (with_list ? 0 : (uint64_t)rows * p->bm_stride * 4));
+  p->off_bm_eq = pos;      pos = round16(pos + (with_list ? 0 : (uint64_t)rows * p->bm_stride * 4));
+  p->off_seg = pos;        pos = round16(pos + (uint64_t)rows * (with_list ? p->ntile : p->nseg) * sizeof(uint2));
   p->off_list = pos;       pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint2));
-  p->off_tile_info = pos;  pos = round16(pos + (with_list ? (uint64_t)rows * p->ntile * sizeof(uint2) : 0));
+  p->off_tile_info = pos;  pos = round16(pos + (with_list ? (uint64_t)rows * p->ntile * sizeof(uint4) : 0));
   p->off_dense = pos;      pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint2));
   p->bytes = pos;
   p->pred = nullptr;
@@ -1032,7 +1163,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   uint32_t* bm_eq = reinterpret_cast<uint32_t*>(ws + pl.off_bm_eq);  // candidates (no list) / ties
   uint2* seg = reinterpret_cast<uint2*>(ws + pl.off_seg);
   uint2* list = pl.list_cap ? reinterpret_cast<uint2*>(ws + pl.off_list) : nullptr;
-  uint2* tile_info = reinterpret_cast<uint2*>(ws + pl.off_tile_info);
+  uint4* tile_info = reinterpret_cast<uint4*>(ws + pl.off_tile_info);
   uint2* dense = reinterpret_cast<uint2*>(ws + pl.off_dense);
   const uint64_t d = src.d, cap = pl.list_cap;
   const uint64_t padded = pl.nseg * (uint64_t)kSegElems;
@@ -1041,9 +1172,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   cudaError_t e = cudaMemsetAsync(hist, 0, (uint64_t)rows * kBins1 * 4 + (uint64_t)rows * 12, st);
   if (e != cudaSuccess) return e;
 
-  // pass1: one CTA per tile of the padded extent
-  const uint64_t ntile_padded = padded / kTile;
-  dim3 g1((unsigned)ntile_padded, rows, 1);
+  dim3 g1((unsigned)pl.ntile, rows, 1);  // pass1 with a list: one CTA per tile
   // pass1 without a list keeps its span form
   uint64_t span = 16 * kTile;
   while (span > kTile && ((padded + span - 1) / span) * rows < 148ull * 16ull) span /= 2;
@@ -1055,13 +1184,13 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   // of the machine; the CTAs of the vectors that hit leave at once, so with many vectors the grid
   // per vector is halved to keep those empty launches short
   uint64_t stride_ctas = rows >= 8 ? 148ull * 2ull : 148ull * 4ull;
-  if (stride_ctas > padded / kTile) stride_ctas = padded / kTile;
+  if (stride_ctas > pl.ntile) stride_ctas = pl.ntile;
   dim3 gm((unsigned)stride_ctas, rows, 1);
+  const uint64_t off_val = (uint64_t)(reinterpret_cast<uint8_t*>(io.val) - reinterpret_cast<uint8_t*>(io.idx));
 
   if (list && k) {
     TopkPred* pred = pl.pred;
-#define DSQ_P1(S)                                                                                                 \
-  k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, pred, bm_gt, pl.bm_stride, list, cap, tile_info, pl.ntile)
+#define DSQ_P1(S) k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, pred, list, cap, tile_info, pl.ntile)
     switch (srck) {
       case SRC_WORKER: DSQ_P1(SRC_WORKER); break;
       case SRC_SRV_IDENTITY: DSQ_P1(SRC_SRV_IDENTITY); break;
@@ -1072,23 +1201,28 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     }
 #undef DSQ_P1
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(bm_eq, 0, (uint64_t)rows * pl.bm_stride * 4, st)) != cudaSuccess) return e;  // tie bitmap
+    // level 1 keeps a whole SM per CTA (registers), so its grid is one wave; levels 2 and 3 fit two per SM
+    dim3 gl1((unsigned)(148ull / rows ? 148ull / rows : 1), rows, 1);
     dim3 gl((unsigned)(148ull * 2ull / rows ? 148ull * 2ull / rows : 1), rows, 1);
-    k_topk_lhist<1><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+    k_topk_lhist<1><<<gl1, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred);
-    k_topk_hist<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, hist);
+    k_topk_hist<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, pred, list, cap, tile_info, hist);
     k_topk_pick1<<<rows, 1024, 0, st>>>(hist, state, k32);
-    k_topk_mark<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, bm_gt, pl.bm_stride, padded, list, cap, tile_info,
-                                         pl.ntile);
+    k_topk_mark<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, list, cap, tile_info, pl.ntile);
     k_topk_compact<<<gm, kThreads, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, state);
     k_topk_lhist<2><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred);
     k_topk_lhist<3><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred);
     dim3 gc((unsigned)(148ull * 8ull / rows ? 148ull * 8ull / rows : 1), rows, 1);
-    k_topk_classify<<<gc, kThreads, 0, st>>>(dense, list_count, cap, state, bm_gt, bm_eq, pl.bm_stride);
-    k_topk_count<<<gs, kThreads, 0, st>>>(bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
+    k_topk_classify<<<gc, kThreads, 0, st>>>(dense, list_count, cap, state, tile_info, pl.ntile);
+    k_topk_scan<true><<<rows, 1024, 0, st>>>(seg, tile_info, pl.ntile, state, k32, io.dev_status);
+    dim3 ge((unsigned)((pl.ntile + kThreads / 32 - 1) / (kThreads / 32)), rows, 1);
+    k_topk_emit_list<<<ge, kThreads, 0, st>>>(io.v_inout, d, state, list, cap, tile_info, seg, pl.ntile,
+                                              reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x,
+                                              io.gamma);
     count_launches(11);
+    return cudaGetLastError();
   } else {
 #define DSQ_P1(S) k_topk_pass1_basic<S><<<g1b, kThreads, 0, st>>>(src, io.v_inout, hist, span)
     switch (srck) {
@@ -1112,11 +1246,9 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     k_topk_finalize<<<gs, kThreads, 0, st>>>(io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
     count_launches(7);
   }
-  k_topk_scan<<<rows, 1024, 0, st>>>(seg, pl.nseg, state, k32, io.dev_status);
+  k_topk_scan<false><<<rows, 1024, 0, st>>>(seg, nullptr, pl.nseg, state, k32, io.dev_status);
   k_topk_emit<<<gs, kThreads, 0, st>>>(io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg,
-                                       reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0,
-                                       (uint64_t)(reinterpret_cast<uint8_t*>(io.val) - reinterpret_cast<uint8_t*>(io.idx)),
-                                       k32, io.x, io.gamma);
+                                       reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x, io.gamma);
   count_launches(2);
   return cudaGetLastError();
 }
