@@ -270,6 +270,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
 
 template <int OP, int SRC, int V, int LOG2G>
 __global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const ChunkParams p) {
+  pdl_prologue();
   __shared__ float s_red[64];
   __shared__ float s_scal[16];
   constexpr uint64_t span = (uint64_t)V * 4u * kThreads;  // entries per CTA
@@ -287,13 +288,13 @@ cudaError_t launch_v(const SrcParams& src, const ChunkParams& p, uint32_t rows, 
   const uint64_t span_entries = chunk <= 1024 ? 1024 : chunk;  // entries per CTA
   dim3 grid((unsigned)((src.d + span_entries - 1) / span_entries), rows, 1);
   switch (chunk) {
-    case 128: k_chunked<OP, SRC, 1, 5><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 256: k_chunked<OP, SRC, 1, 6><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 512: k_chunked<OP, SRC, 1, 7><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 1024: k_chunked<OP, SRC, 1, 8><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 2048: k_chunked<OP, SRC, 2, 8><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 4096: k_chunked<OP, SRC, 4, 8><<<grid, kThreads, 0, st>>>(src, p); break;
-    case 8192: k_chunked<OP, SRC, 8, 8><<<grid, kThreads, 0, st>>>(src, p); break;
+    case 128: launch_pdl(k_chunked<OP, SRC, 1, 5>, grid, kThreads, st, src, p); break;
+    case 256: launch_pdl(k_chunked<OP, SRC, 1, 6>, grid, kThreads, st, src, p); break;
+    case 512: launch_pdl(k_chunked<OP, SRC, 1, 7>, grid, kThreads, st, src, p); break;
+    case 1024: launch_pdl(k_chunked<OP, SRC, 1, 8>, grid, kThreads, st, src, p); break;
+    case 2048: launch_pdl(k_chunked<OP, SRC, 2, 8>, grid, kThreads, st, src, p); break;
+    case 4096: launch_pdl(k_chunked<OP, SRC, 4, 8>, grid, kThreads, st, src, p); break;
+    case 8192: launch_pdl(k_chunked<OP, SRC, 8, 8>, grid, kThreads, st, src, p); break;
     default: return cudaErrorInvalidValue;
   }
   count_launches(1);

@@ -9,6 +9,15 @@ namespace dsq {
 
 constexpr int kThreads = 256;  // every streaming kernel uses 256-thread CTAs
 
+// Kernels are launched with programmatic stream serialization: once every CTA of a kernel has
+// passed launch_dependents (or left), the CTAs of the next kernel in the stream may take free
+// slots; there they stop at wait until the earlier kernel has completed and its writes are
+// visible.  Every kernel starts with this prologue, so nothing before it touches memory.
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 enum Src : int {
   SRC_WORKER = 0,        // v = g[row] + delta_w[row]
   SRC_SRV_IDENTITY = 1,  // v = (sum_i c_i) * inv_n + delta_s

@@ -10,6 +10,7 @@ template <int SRC>
 __global__ void __launch_bounds__(kThreads) k_identity(const SrcParams src, float* out_c, uint64_t c_row_stride,
                                                        float* delta_out, uint64_t delta_row_stride, float* x,
                                                        float gamma) {
+  pdl_prologue();
   const uint32_t row = blockIdx.y;
   const uint64_t nq = (src.d + 3) / 4;
   // the loop bound is the same for all threads of the CTA: the source is read warp-cooperatively
@@ -42,7 +43,7 @@ static unsigned grid_for(uint64_t items) {
 cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64_t c_row_stride, float* delta_out,
                             uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st) {
   dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
-#define DSQ_ID(S) k_identity<S><<<grid, kThreads, 0, st>>>(src, out_c, c_row_stride, delta_out, delta_row_stride, x, gamma)
+#define DSQ_ID(S) launch_pdl(k_identity<S>, grid, kThreads, st, src, out_c, c_row_stride, delta_out, delta_row_stride, x, gamma)
   switch (srck) {
     case SRC_WORKER: DSQ_ID(SRC_WORKER); break;
     case SRC_SRV_IDENTITY: DSQ_ID(SRC_SRV_IDENTITY); break;
@@ -58,6 +59,7 @@ cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64
 
 // Dense decode of a server payload and update of x.
 __global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, float* x, uint64_t d, float gamma) {
+  pdl_prologue();
   const uint64_t nq = (d + 3) / 4;
   for (uint64_t qd = (uint64_t)blockIdx.x * kThreads + threadIdx.x; qd < nq; qd += (uint64_t)gridDim.x * kThreads) {
     const uint64_t e = qd * 4;
@@ -88,6 +90,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, 
 // Sparse payload: only the k listed entries of x change (the others would subtract gamma * 0).
 __global__ void __launch_bounds__(kThreads) k_apply_sparse(const uint32_t* __restrict__ idx, const float* __restrict__ val,
                                                            uint64_t k, float* x, float gamma) {
+  pdl_prologue();
   for (uint64_t m = (uint64_t)blockIdx.x * kThreads + threadIdx.x; m < k; m += (uint64_t)gridDim.x * kThreads) {
     const uint32_t j = idx[m];
     x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val[m]));
@@ -97,10 +100,10 @@ __global__ void __launch_bounds__(kThreads) k_apply_sparse(const uint32_t* __res
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st) {
   if (pv.op == DS_Q_TOPK) {
     if (pv.k == 0) return cudaSuccess;
-    k_apply_sparse<<<grid_for(pv.k), kThreads, 0, st>>>(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]),
+    launch_pdl(k_apply_sparse, grid_for(pv.k), kThreads, st, reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]),
                                                         reinterpret_cast<const float*>(pv.base + pv.off[1]), pv.k, x, gamma);
   } else {
-    k_apply_dense<<<grid_for((d + 3) / 4), kThreads, 0, st>>>(pv, x, d, gamma);
+    launch_pdl(k_apply_dense, grid_for((d + 3) / 4), kThreads, st, pv, x, d, gamma);
   }
   count_launches(1);
   return cudaGetLastError();
@@ -119,6 +122,7 @@ constexpr uint32_t kAccSpan = 8192;
 
 __global__ void __launch_bounds__(kThreads) k_sparse_offsets(const uint8_t* __restrict__ wp, uint64_t stride, uint64_t off_idx,
                                                              uint64_t k, uint64_t nspan, uint32_t* off) {
+  pdl_prologue();
   const uint32_t i = blockIdx.y;
   const uint32_t* idx = reinterpret_cast<const uint32_t*>(wp + (uint64_t)i * stride + off_idx);
   uint32_t* o = off + (uint64_t)i * (nspan + 1);
@@ -135,6 +139,7 @@ __global__ void __launch_bounds__(kThreads) k_sparse_accumulate(const uint8_t* _
                                                                 uint64_t off_idx, uint64_t off_val, uint32_t n, uint64_t d,
                                                                 uint64_t nspan, const uint32_t* __restrict__ off,
                                                                 float* acc) {
+  pdl_prologue();
   __shared__ float s_acc[kAccSpan];
   const uint32_t tid = threadIdx.x;
   const uint64_t span = blockIdx.x;
@@ -197,8 +202,8 @@ cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_
   const uint64_t nspan = (d + kAccSpan - 1) / kAccSpan;
   uint64_t ctas = (k + kThreads) / kThreads;
   if (ctas > 148 * 8) ctas = 148 * 8;
-  k_sparse_offsets<<<dim3((unsigned)ctas, n, 1), kThreads, 0, st>>>(wp, stride, off_idx, k, nspan, offsets);
-  k_sparse_accumulate<<<(unsigned)nspan, kThreads, 0, st>>>(wp, stride, off_idx, off_val, n, d, nspan, offsets, acc);
+  launch_pdl(k_sparse_offsets, dim3((unsigned)ctas, n, 1), kThreads, st, wp, stride, off_idx, k, nspan, offsets);
+  launch_pdl(k_sparse_accumulate, (unsigned)nspan, kThreads, st, wp, stride, off_idx, off_val, n, d, nspan, offsets, acc);
   count_launches(2);
   return cudaGetLastError();
 }

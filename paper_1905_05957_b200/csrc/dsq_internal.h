@@ -12,6 +12,23 @@ namespace dsq {
 extern uint64_t g_kernel_launches;
 inline void count_launches(uint64_t n) { g_kernel_launches += n; }
 
+// kernel<<<grid, block, 0, st>>>(args...) with programmatic stream serialization allowed (the
+// kernel begins with pdl_prologue()).  A failed launch shows in cudaGetLastError().
+template <typename... P, typename... A>
+inline void launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t st, A&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
 // Destination of a chunk-wise operator (SIGN1 or QSGD).
 struct ChunkParams {
   uint32_t* out_bits;        // sign words, row stride bits_stride (in words)

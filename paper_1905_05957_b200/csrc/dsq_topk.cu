@@ -231,6 +231,7 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
 template <int SRC>
 __global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER || SRC == SRC_SRV_TOPK ? 5 : 1) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred, uint2* list,
                                                          uint64_t cap, uint4* tile_info, uint64_t ntile) {
+  pdl_prologue();
   __shared__ uint4 s_tot[kThreads / 32];
   const uint32_t row = blockIdx.y;
   const uint64_t tile = blockIdx.x, base = tile * kTile;
@@ -295,6 +296,7 @@ __device__ __forceinline__ void cta_pick(const uint32_t* h, uint32_t want, uint3
 
 // Level-1 pick after a miss, one CTA per vector, on the full histogram written by k_topk_hist.
 __global__ void __launch_bounds__(1024) k_topk_pick1(uint32_t* hist, TopkState* state, uint32_t k) {
+  pdl_prologue();
   __shared__ uint32_t s_warp[32], s_out[3];
   const uint32_t tid = threadIdx.x, row = blockIdx.x;
   uint32_t* h = hist + (uint64_t)row * kBins1;
@@ -317,6 +319,7 @@ __global__ void __launch_bounds__(1024) k_topk_pick1(uint32_t* hist, TopkState* 
 __global__ void __launch_bounds__(kThreads) k_topk_hist(float* v_io, uint64_t d, int vec, const TopkState* state,
                                                         const TopkPred* pred, const uint2* list, uint64_t cap,
                                                         const uint4* tile_info, uint32_t* hist) {
+  pdl_prologue();
   __shared__ uint32_t s_hist[kBins1];
   const uint32_t tid = threadIdx.x, row = blockIdx.y;
   if (!state[row].need_full) return;
@@ -367,6 +370,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_hist(float* v_io, uint64_t d,
 // zeroed), entries inside it are the candidates.  A small grid strides over the tiles.
 __global__ void __launch_bounds__(kThreads) k_topk_mark(float* v_io, uint64_t d, int vec, const TopkState* state, uint2* list,
                                                         uint64_t cap, uint4* tile_info, uint64_t ntile) {
+  pdl_prologue();
   __shared__ uint4 s_tot[kThreads / 32];
   const uint32_t tid = threadIdx.x, row = blockIdx.y;
   if (!state[row].need_mark) return;
@@ -518,6 +522,7 @@ __device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint4*
 __global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, uint64_t cap, const uint4* tile_info,
                                                            uint64_t ntile, uint2* dense, uint32_t* dense_count,
                                                            const TopkState* state) {
+  pdl_prologue();
   __shared__ uint32_t s_n[kThreads], s_off[kThreads], s_warp[34];
   const uint32_t row = blockIdx.y;
   if (!state[row].need_mark) return;
@@ -536,6 +541,7 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
                                                      uint2* dense, uint32_t* dense_count, uint32_t* kept_count,
                                                      TopkState* state, uint32_t* hist, uint32_t* done, uint32_t k,
                                                      TopkPred* pred) {
+  pdl_prologue();
   __shared__ uint32_t s_hist[kBins1];
   __shared__ uint32_t s_warp[34], s_out[3];
   __shared__ uint32_t s_last, s_kept;
@@ -653,6 +659,7 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
 // them.  Integer atomics: order-free.
 __global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* dense, const uint32_t* dense_count, uint64_t cap,
                                                             const TopkState* state, uint4* tile_info, uint64_t ntile) {
+  pdl_prologue();
   const uint32_t row = blockIdx.y, lane = threadIdx.x & 31u;
   const uint2* drow = dense + (uint64_t)row * cap;
   const uint64_t n = min((uint64_t)dense_count[row], cap);
@@ -690,6 +697,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit_list(float* v_io, uint64
                                                              uint64_t ntile, uint8_t* payload, uint64_t payload_stride,
                                                              uint64_t off_idx, uint64_t off_val, uint32_t k, float* x,
                                                              float gamma) {
+  pdl_prologue();
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   const uint64_t tile = (uint64_t)blockIdx.x * (kThreads / 32) + (tid >> 5);
   if (tile >= ntile) return;
@@ -753,6 +761,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit_list(float* v_io, uint64
 template <int SRC>
 __global__ void __launch_bounds__(kThreads) k_topk_pass1_basic(const SrcParams src, float* v_out, uint32_t* hist,
                                                                uint64_t span) {
+  pdl_prologue();
   __shared__ uint32_t s_hist[kBins1];
   const uint32_t tid = threadIdx.x, row = blockIdx.y;
   for (uint32_t b = tid; b < kBins1; b += kThreads) s_hist[b] = 0;
@@ -799,6 +808,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_pass1_basic(const SrcParams s
 //   level 2: bins = (key >> 7) & 0xFFF   want = k_rem
 //   level 3: bins = key & 0x7F           want = k_rem   -> tau and r complete
 __global__ void __launch_bounds__(1024) k_topk_pick_basic(uint32_t* hist, TopkState* state, uint32_t level, uint32_t k) {
+  pdl_prologue();
   __shared__ uint32_t s_warp[32], s_out[3];
   const uint32_t tid = threadIdx.x, row = blockIdx.x;
   uint32_t* h = hist + (uint64_t)row * kBins1;
@@ -825,6 +835,7 @@ __global__ void __launch_bounds__(1024) k_topk_pick_basic(uint32_t* hist, TopkSt
 __global__ void __launch_bounds__(kThreads) k_topk_mark_basic(const float* v_in, uint64_t d, int vec, const TopkState* state,
                                                               uint32_t* bm_gt, uint32_t* bm_eq, uint64_t bm_stride,
                                                               uint64_t padded) {
+  pdl_prologue();
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   const uint32_t tb = state[row].tb1;
   const float* vrow = v_in + (uint64_t)row * d;
@@ -869,6 +880,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_mark_basic(const float* v_in,
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads) k_topk_refine(const float* v_in, uint64_t d, const TopkState* state,
                                                           const uint32_t* bm_eq, uint64_t bm_stride, uint32_t* hist) {
+  pdl_prologue();
   constexpr uint32_t NB = LEVEL == 2 ? 4096u : 128u;
   __shared__ uint32_t s_hist[NB];
   __shared__ uint32_t s_any;
@@ -912,6 +924,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_refine(const float* v_in, uin
 __global__ void __launch_bounds__(kThreads) k_topk_finalize(const float* v_in, uint64_t d, const TopkState* state,
                                                             uint32_t* bm_gt, uint32_t* bm_eq, uint64_t bm_stride,
                                                             uint2* seg_cnt, uint64_t nseg) {
+  pdl_prologue();
   __shared__ uint32_t s_gt[kThreads / 32], s_tie[kThreads / 32];
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   const uint64_t widx = (uint64_t)blockIdx.x * kSegWords + tid * kWordsPerThread;
@@ -961,6 +974,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_finalize(const float* v_in, u
 template <bool TILES>
 __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4* tile_info, uint64_t nseg, TopkState* state,
                                                     uint32_t k, uint32_t* dev_status) {
+  pdl_prologue();
   constexpr int ITEMS = TILES ? 8 : 1;  // consecutive counts per thread: one round trip to memory for all of them
   __shared__ uint2 s_warp[32];
   __shared__ uint2 s_carry;
@@ -1039,6 +1053,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
                                                         const uint2* seg_pre, uint64_t nseg, uint8_t* payload,
                                                         uint64_t payload_stride, uint64_t off_idx, uint64_t off_val,
                                                         uint32_t k, float* x, float gamma) {
+  pdl_prologue();
   __shared__ uint32_t s_warp[kThreads / 32];
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.y;
   const uint64_t widx = (uint64_t)blockIdx.x * kSegWords + tid * kWordsPerThread;
@@ -1190,7 +1205,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
 
   if (list && k) {
     TopkPred* pred = pl.pred;
-#define DSQ_P1(S) k_topk_pass1<S><<<g1, kThreads, 0, st>>>(src, io.v_inout, pred, list, cap, tile_info, pl.ntile)
+#define DSQ_P1(S) launch_pdl(k_topk_pass1<S>, g1, kThreads, st, src, io.v_inout, pred, list, cap, tile_info, pl.ntile)
     switch (srck) {
       case SRC_WORKER: DSQ_P1(SRC_WORKER); break;
       case SRC_SRV_IDENTITY: DSQ_P1(SRC_SRV_IDENTITY); break;
@@ -1204,27 +1219,27 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     // level 1 keeps a whole SM per CTA (registers), so its grid is one wave; levels 2 and 3 fit two per SM
     dim3 gl1((unsigned)(148ull / rows ? 148ull / rows : 1), rows, 1);
     dim3 gl((unsigned)(148ull * 2ull / rows ? 148ull * 2ull / rows : 1), rows, 1);
-    k_topk_lhist<1><<<gl1, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+    launch_pdl(k_topk_lhist<1>, gl1, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred);
-    k_topk_hist<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, pred, list, cap, tile_info, hist);
-    k_topk_pick1<<<rows, 1024, 0, st>>>(hist, state, k32);
-    k_topk_mark<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, list, cap, tile_info, pl.ntile);
-    k_topk_compact<<<gm, kThreads, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, state);
-    k_topk_lhist<2><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+    launch_pdl(k_topk_hist, gm, kThreads, st, io.v_inout, d, src.vec, state, pred, list, cap, tile_info, hist);
+    launch_pdl(k_topk_pick1, rows, 1024, st, hist, state, k32);
+    launch_pdl(k_topk_mark, gm, kThreads, st, io.v_inout, d, src.vec, state, list, cap, tile_info, pl.ntile);
+    launch_pdl(k_topk_compact, gm, kThreads, st, list, cap, tile_info, pl.ntile, dense, list_count, state);
+    launch_pdl(k_topk_lhist<2>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred);
-    k_topk_lhist<3><<<gl, 1024, 0, st>>>(list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+    launch_pdl(k_topk_lhist<3>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred);
     dim3 gc((unsigned)(148ull * 8ull / rows ? 148ull * 8ull / rows : 1), rows, 1);
-    k_topk_classify<<<gc, kThreads, 0, st>>>(dense, list_count, cap, state, tile_info, pl.ntile);
-    k_topk_scan<true><<<rows, 1024, 0, st>>>(seg, tile_info, pl.ntile, state, k32, io.dev_status);
+    launch_pdl(k_topk_classify, gc, kThreads, st, dense, list_count, cap, state, tile_info, pl.ntile);
+    launch_pdl(k_topk_scan<true>, rows, 1024, st, seg, tile_info, pl.ntile, state, k32, io.dev_status);
     dim3 ge((unsigned)((pl.ntile + kThreads / 32 - 1) / (kThreads / 32)), rows, 1);
-    k_topk_emit_list<<<ge, kThreads, 0, st>>>(io.v_inout, d, state, list, cap, tile_info, seg, pl.ntile,
+    launch_pdl(k_topk_emit_list, ge, kThreads, st, io.v_inout, d, state, list, cap, tile_info, seg, pl.ntile,
                                               reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x,
                                               io.gamma);
     count_launches(11);
     return cudaGetLastError();
   } else {
-#define DSQ_P1(S) k_topk_pass1_basic<S><<<g1b, kThreads, 0, st>>>(src, io.v_inout, hist, span)
+#define DSQ_P1(S) launch_pdl(k_topk_pass1_basic<S>, g1b, kThreads, st, src, io.v_inout, hist, span)
     switch (srck) {
       case SRC_WORKER: DSQ_P1(SRC_WORKER); break;
       case SRC_SRV_IDENTITY: DSQ_P1(SRC_SRV_IDENTITY); break;
@@ -1237,17 +1252,17 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     count_launches(1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (k == 0) return cudaSuccess;  // nothing kept: Q[v] = 0, delta = v, x unchanged
-    k_topk_pick_basic<<<rows, 1024, 0, st>>>(hist, state, 1, k32);
-    k_topk_mark_basic<<<gm, kThreads, 0, st>>>(io.v_inout, d, src.vec, state, bm_gt, bm_eq, pl.bm_stride, padded);
-    k_topk_refine<2><<<gs, kThreads, 0, st>>>(io.v_inout, d, state, bm_eq, pl.bm_stride, hist);
-    k_topk_pick_basic<<<rows, 1024, 0, st>>>(hist, state, 2, k32);
-    k_topk_refine<3><<<gs, kThreads, 0, st>>>(io.v_inout, d, state, bm_eq, pl.bm_stride, hist);
-    k_topk_pick_basic<<<rows, 1024, 0, st>>>(hist, state, 3, k32);
-    k_topk_finalize<<<gs, kThreads, 0, st>>>(io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
+    launch_pdl(k_topk_pick_basic, rows, 1024, st, hist, state, 1, k32);
+    launch_pdl(k_topk_mark_basic, gm, kThreads, st, io.v_inout, d, src.vec, state, bm_gt, bm_eq, pl.bm_stride, padded);
+    launch_pdl(k_topk_refine<2>, gs, kThreads, st, io.v_inout, d, state, bm_eq, pl.bm_stride, hist);
+    launch_pdl(k_topk_pick_basic, rows, 1024, st, hist, state, 2, k32);
+    launch_pdl(k_topk_refine<3>, gs, kThreads, st, io.v_inout, d, state, bm_eq, pl.bm_stride, hist);
+    launch_pdl(k_topk_pick_basic, rows, 1024, st, hist, state, 3, k32);
+    launch_pdl(k_topk_finalize, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
     count_launches(7);
   }
-  k_topk_scan<false><<<rows, 1024, 0, st>>>(seg, nullptr, pl.nseg, state, k32, io.dev_status);
-  k_topk_emit<<<gs, kThreads, 0, st>>>(io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg,
+  launch_pdl(k_topk_scan<false>, rows, 1024, st, seg, nullptr, pl.nseg, state, k32, io.dev_status);
+  launch_pdl(k_topk_emit, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg,
                                        reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x, io.gamma);
   count_launches(2);
   return cudaGetLastError();
