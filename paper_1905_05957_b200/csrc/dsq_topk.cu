@@ -975,32 +975,40 @@ template <bool TILES>
 __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4* tile_info, uint64_t nseg, TopkState* state,
                                                     uint32_t k, uint32_t* dev_status) {
   pdl_prologue();
-  constexpr int ITEMS = TILES ? 8 : 1;  // consecutive counts per thread: one round trip to memory for all of them
+  // A round takes 4096 counts: loaded and stored with neighbouring threads on neighbouring counts,
+  // scanned with four consecutive counts per thread; shared memory turns one order into the other.
+  constexpr int ITEMS = 4;
+  __shared__ uint2 s_item[1024 * ITEMS];
   __shared__ uint2 s_warp[32];
   __shared__ uint2 s_carry;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.x;
   uint2* c = seg_cnt + (uint64_t)row * nseg;
   if (tid == 0) s_carry = make_uint2(0, 0);
-  __syncthreads();
   for (uint64_t base = 0; base < nseg; base += 1024 * ITEMS) {
-    uint2 item[ITEMS];
-    uint2 mine = make_uint2(0, 0);
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) {
-      const uint64_t i = base + (uint64_t)tid * ITEMS + u;
-      item[u] = make_uint2(0, 0);
+      const uint64_t i = base + (uint64_t)u * 1024 + tid;
+      uint2 item = make_uint2(0, 0);
       if (i < nseg) {
         if (TILES) {
           const uint4 t = tile_info[(uint64_t)row * nseg + i];
-          item[u] = make_uint2(t.y + t.z, t.w);  // above the band + candidates above tau; candidates equal to tau
+          item = make_uint2(t.y + t.z, t.w);  // above the band + candidates above tau; candidates equal to tau
         } else {
-          item[u] = c[i];
+          item = c[i];
         }
       }
-      mine.x += item[u].x;
-      mine.y += item[u].y;
+      s_item[u * 1024 + tid] = item;
     }
-    uint2 incl = mine;
+    __syncthreads();
+    uint2 mine[ITEMS];
+    uint2 sum = make_uint2(0, 0);
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      mine[u] = s_item[tid * ITEMS + u];
+      sum.x += mine[u].x;
+      sum.y += mine[u].y;
+    }
+    uint2 incl = sum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const uint32_t yx = __shfl_up_sync(0xffffffffu, incl.x, o), yy = __shfl_up_sync(0xffffffffu, incl.y, o);
@@ -1020,18 +1028,23 @@ __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4*
     }
     __syncthreads();
     const uint2 carry = s_carry;
-    uint2 excl = make_uint2(carry.x + s_warp[wrp].x + incl.x - mine.x, carry.y + s_warp[wrp].y + incl.y - mine.y);
+    uint2 excl = make_uint2(carry.x + s_warp[wrp].x + incl.x - sum.x, carry.y + s_warp[wrp].y + incl.y - sum.y);
 #pragma unroll
     for (int u = 0; u < ITEMS; ++u) {
-      const uint64_t i = base + (uint64_t)tid * ITEMS + u;
-      if (i < nseg) c[i] = excl;
-      excl.x += item[u].x;
-      excl.y += item[u].y;
+      s_item[tid * ITEMS + u] = excl;
+      excl.x += mine[u].x;
+      excl.y += mine[u].y;
     }
     __syncthreads();
-    if (tid == 1023) s_carry = excl;  // the prefix after this round's last item
+    if (tid == 1023) s_carry = excl;  // the prefix after this round's last count
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      const uint64_t i = base + (uint64_t)u * 1024 + tid;
+      if (i < nseg) c[i] = s_item[u * 1024 + tid];
+    }
     __syncthreads();
   }
+  __syncthreads();
   if (tid == 0) {
     const uint2 tot = s_carry;
     const uint32_t r = state[row].r;
