@@ -187,7 +187,7 @@ def run_reference(args, wl):
 def workload_config(wl) -> dict:
     def q(s):
         return {"op": s.op, **({"chunk": s.chunk} if s.chunk else {}), **({"k": s.k} if s.op == "topk" else {}),
-                **({"levels": s.levels} if s.levels else {})}
+                **({"levels": s.levels} if s.levels else {}), **({"norm": "l2"} if s.op == "sign1" and s.norm == 2 else {})}
     return {"workload": wl.name, "n_workers": wl.n, "d": wl.d, "gradient_dist": wl.dist, "worker_q": q(wl.worker_q),
             "server_q": q(wl.server_q), "gamma": wl.gamma,
             "l2": "inputs larger than L2: g and delta_w are streamed once per step and exceed 126 MB"
@@ -361,7 +361,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", type=int, default=2, help="1..5; 2 = ResNet-18-sized 1-bit (the default)")
+    ap.add_argument("--workload", type=int, default=2, help="1..5 = the five listed configurations, 2 = ResNet-18-sized 1-bit (the default); "
+                         "6 = shape of 2 with the l2-magnitude 1-bit scale")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-steps", type=int, default=3)

@@ -67,6 +67,8 @@ typedef enum {
  *                factor is the mean absolute value of each chunk of `chunk` consecutive entries
  *                of the flat vector (the last chunk may be short; its true length divides).
  *                bit = (v >= 0);  Q[v]_j = bit ? +s_c : -s_c.
+ *                With norm = DS_NORM_L2 the magnitudes of Section 5.1's ratio are l2 norms (the
+ *                norm Section 3.2 prints): s_c = ||v_c||_2 / sqrt(len_c).  Same payload format.
  *
  * DS_Q_TOPK      "Top-k compression" of Section 5.1 (Section 3.2 "Top-k sparsification"): the k
  *                entries of largest absolute value over the whole d-vector keep their value, all
@@ -86,12 +88,16 @@ typedef enum {
  */
 typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3 } ds_op;
 
+/* ds_qspec.norm for DS_Q_SIGN1 */
+#define DS_NORM_L1 0u /* s_c = ||v_c||_1 / len_c (also selected by 1) */
+#define DS_NORM_L2 2u /* s_c = ||v_c||_2 / sqrt(len_c) */
+
 typedef struct {
   int32_t op;        /* ds_op */
   uint32_t chunk;    /* SIGN1, QSGD: a power of two in [128, 8192]; else ignored */
   uint64_t k;        /* TOPK: 0 <= k <= d; else ignored */
   uint32_t levels;   /* QSGD: 1 <= levels <= 255; else ignored */
-  uint32_t reserved; /* must be 0 */
+  uint32_t norm;     /* SIGN1: DS_NORM_L1 (0 or 1) or DS_NORM_L2 (2); else must be 0 */
 } ds_qspec;
 
 typedef struct {

@@ -38,7 +38,7 @@ def load(path: str):
     L.orc_apply_update.restype = None
     L.orc_apply_update.argtypes = [f32p, f32p, C.c_float, u64]
     L.orc_q_identity.argtypes = [f32p, u64, f32p]
-    L.orc_q_sign1.argtypes = [f32p, u64, u32, u32p, f32p, f32p]
+    L.orc_q_sign1.argtypes = [f32p, u64, u32, u32, u32p, f32p, f32p]
     L.orc_decode_sign1.argtypes = [u32p, f32p, u64, u32, f32p]
     L.orc_q_topk.argtypes = [f32p, u64, u64, u32p, f32p, f32p]
     L.orc_decode_topk.argtypes = [u32p, f32p, u64, u64, f32p]
@@ -122,6 +122,7 @@ def apply_update(x, Cv, gamma) -> np.ndarray:
 class QSpec:
     op: str = IDENTITY
     chunk: int = 0      # sign1 / qsgd: chunk length L (power of two)
+    norm: int = 1       # sign1: the scale is the ratio of l1 (1) or l2 (2) magnitudes
     k: int = 0          # topk
     levels: int = 0     # qsgd: s
 
@@ -133,13 +134,13 @@ def q_identity(v):
     return Cv, {"c": Cv.copy()}
 
 
-def q_sign1(v, L):
+def q_sign1(v, L, norm=1):
     v = _f32(v)
     d = v.size
     bits = np.zeros((d + 31) // 32, dtype=np.uint32)
     scale = np.zeros((d + L - 1) // L, dtype=np.float32)
     Cv = np.empty_like(v)
-    _check(lib().orc_q_sign1(_p(v, C.c_float), d, L, _p(bits, C.c_uint32), _p(scale, C.c_float),
+    _check(lib().orc_q_sign1(_p(v, C.c_float), d, L, norm, _p(bits, C.c_uint32), _p(scale, C.c_float),
                              _p(Cv, C.c_float)), "sign1")
     return Cv, {"bits": bits, "scale": scale}
 
@@ -202,7 +203,7 @@ def compress(q: QSpec, v, seed=0, step=0, wid=0):
     if q.op == IDENTITY:
         return q_identity(v)
     if q.op == SIGN1:
-        return q_sign1(v, q.chunk)
+        return q_sign1(v, q.chunk, q.norm)
     if q.op == TOPK:
         return q_topk(v, q.k)
     if q.op == QSGD:

@@ -22,7 +22,7 @@
  *
  * Parity pins (tests/test_oracle_*.py): identity => parallel SGD bitwise;
  * C + delta_new == g + delta_old; the telescoping identity of Section 3.3
- * (Eq. 5-6); sign scale == ||v||_1/len and its closed-form residual energy;
+ * (Eq. 5-6); sign scale == ||v||_1/len (or ||v||_2/sqrt(len)) and its closed-form residual energy;
  * top-k against a brute-force stable sort; QSGD unbiasedness and variance by
  * Monte Carlo plus its deterministic special cases; Philox4x32-10 against an
  * independent library implementation; pairwise summation against hand-derived
@@ -153,28 +153,43 @@ int orc_q_identity(const float* v, uint64_t d, float* C) {
 /* ------------------------------------------------------------------------ */
 /* Q = 1-bit quantisation with a scaling factor (Section 3.2 "1-Bit          */
 /* Quantization"; Section 5.1 "1-bit compression": the factor is magnitude   */
-/* of the compensated gradient over magnitude of the sign vector).  Reading: */
-/* magnitude = l1 norm, taken per chunk of L consecutive elements of the     */
-/* flat vector, so the factor of chunk c is ||v_c||_1 / len_c with len_c the */
-/* true length of the (possibly short, last) chunk.  A zero has no sign to   */
-/* send, so bit = (v >= 0).                                                  */
+/* of the compensated gradient over magnitude of the sign vector).  The      */
+/* factor is taken per chunk of L consecutive elements of the flat vector,   */
+/* len_c being the true length of the (possibly short, last) chunk.          */
+/*   norm = 1: magnitude = l1 norm, factor = ||v_c||_1 / len_c               */
+/*   norm = 2: magnitude = l2 norm (the norm Section 3.2 prints),            */
+/*             factor = ||v_c||_2 / sqrt(len_c)                              */
+/* A zero has no sign to send, so bit = (v >= 0).                            */
 /*   bits : ceil(d/32) words, element j -> bit (j%32) of word j/32, pad 0    */
 /*   scale: ceil(d/L) floats                                                 */
 /*   C    : d floats (may be NULL)                                           */
 /* ------------------------------------------------------------------------ */
 
-int orc_q_sign1(const float* v, uint64_t d, uint32_t L, uint32_t* bits, float* scale, float* C) {
-  if (!is_pow2_u32(L)) return ORC_ERR_ARG;
+int orc_q_sign1(const float* v, uint64_t d, uint32_t L, uint32_t norm, uint32_t* bits, float* scale, float* C) {
+  if (!is_pow2_u32(L) || (norm != 1 && norm != 2)) return ORC_ERR_ARG;
   uint64_t nw = (d + 31) / 32, nc = (d + L - 1) / L;
-  float* absv = (float*)malloc(sizeof(float) * L);
-  if (!absv) return ORC_ERR_NOMEM;
+  float* term = (float*)malloc(sizeof(float) * L);
+  if (!term) return ORC_ERR_NOMEM;
   memset(bits, 0, sizeof(uint32_t) * nw);
   for (uint64_t c = 0; c < nc; ++c) {
     uint64_t lo = c * L, hi = lo + L < d ? lo + L : d;
     uint32_t len = (uint32_t)(hi - lo);
-    for (uint32_t t = 0; t < L; ++t) absv[t] = t < len ? fabsf(v[lo + t]) : 0.0f;
-    float l1 = pairwise_sum(absv, L);
-    float s = l1 / (float)len;
+    float s;
+    if (norm == 1) {
+      for (uint32_t t = 0; t < L; ++t) term[t] = t < len ? fabsf(v[lo + t]) : 0.0f;
+      float l1 = pairwise_sum(term, L);
+      s = l1 / (float)len;
+    } else {
+      for (uint32_t t = 0; t < L; ++t) {
+        float e = t < len ? v[lo + t] : 0.0f;
+        float e2 = e * e;
+        term[t] = e2;
+      }
+      float ss = pairwise_sum(term, L);
+      float l2 = sqrtf(ss);
+      float root_len = sqrtf((float)len);
+      s = l2 / root_len;
+    }
     scale[c] = s;
     for (uint64_t j = lo; j < hi; ++j) {
       int nonneg = v[j] >= 0.0f;
@@ -182,7 +197,7 @@ int orc_q_sign1(const float* v, uint64_t d, uint32_t L, uint32_t* bits, float* s
       if (C) C[j] = nonneg ? s : -s;
     }
   }
-  free(absv);
+  free(term);
   return ORC_OK;
 }
 

@@ -28,7 +28,7 @@ EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggreg
 
 class ds_qspec(C.Structure):
     _fields_ = [("op", C.c_int32), ("chunk", C.c_uint32), ("k", C.c_uint64), ("levels", C.c_uint32),
-                ("reserved", C.c_uint32)]
+                ("norm", C.c_uint32)]
 
 
 class ds_config(C.Structure):
@@ -85,7 +85,7 @@ def load_library() -> C.CDLL:
 
 
 def _qspec(q: Q) -> ds_qspec:
-    return ds_qspec(OPS[q.op], q.chunk, q.k, q.levels, 0)
+    return ds_qspec(OPS[q.op], q.chunk, q.k, q.levels, q.norm if q.op == "sign1" else 0)
 
 
 def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int) -> ds_config:

@@ -28,7 +28,7 @@ inline uint32_t log2u(uint32_t x) { uint32_t l = 0; while ((1u << l) < x) ++l; r
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 bool qspec_ok(const ds_qspec& q, uint64_t d) {
-  if (q.reserved != 0) return false;
+  if (q.op == DS_Q_SIGN1 ? (q.norm != DS_NORM_L1 && q.norm != 1u && q.norm != DS_NORM_L2) : q.norm != 0) return false;
   switch (q.op) {
     case DS_Q_IDENTITY: return true;
     case DS_Q_SIGN1: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192;
@@ -182,6 +182,7 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       p.gamma = c->cfg.gamma;
       p.levels_f = (float)q.levels;
       p.levels_u = q.levels;
+      p.sign_l2 = (q.op == DS_Q_SIGN1 && q.norm == DS_NORM_L2) ? 1u : 0u;
       p.keys = philox_key_schedule((uint32_t)(c->cfg.seed & 0xFFFFFFFFu), (uint32_t)(c->cfg.seed >> 32));
       p.step = step;
       p.server_pass = server ? 1u : 0u;

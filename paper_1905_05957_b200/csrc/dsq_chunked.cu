@@ -113,7 +113,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
       e[j] = base + (uint64_t)(j * G + t) * 4u;
       cnt[j] = FULL ? 4u : (e[j] < d ? (uint32_t)min((uint64_t)4, d - e[j]) : 0u);
     }
-    src_load_tile<SRC, V>(src, row, e, cnt, v);
+    src_load_tile<SRC, V, (int)G * 4>(src, row, e, cnt, v);
   }
 
   // fused model update (server pass): fetch x now so that its latency hides behind the reduction
@@ -125,12 +125,12 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
       xv[kServer ? j : 0] = cnt[j] ? load_row4(p.x, base + (uint64_t)(j * G + t) * 4u, cnt[j], 1) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
 
-  // ---- chunk reduction: sum |v| (SIGN1) or sum v*v (QSGD), pairwise in index order
+  // ---- chunk reduction: sum |v| (SIGN1) or sum v*v (SIGN1 with l2 magnitudes, QSGD), pairwise in index order
   float part[V];
 #pragma unroll
   for (int j = 0; j < V; ++j) {
     float m0, m1, m2, m3;
-    if constexpr (OP == DS_Q_SIGN1) {
+    if (OP == DS_Q_SIGN1 && !p.sign_l2) {
       m0 = fabsf(v[j].x); m1 = fabsf(v[j].y); m2 = fabsf(v[j].z); m3 = fabsf(v[j].w);
     } else {
       const float4 sq = mul4_rn(v[j], v[j]);
@@ -160,7 +160,9 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
   const uint32_t len = FULL ? L : (chunk_live ? (uint32_t)min((uint64_t)L, d - base) : 1u);
   float s_or_q, inv_q = 0.f;
   if constexpr (OP == DS_Q_SIGN1) {
-    s_or_q = __fdiv_rn(total, (float)len);  // mean |v| over the true chunk length
+    // ratio of the magnitudes of v_c and sign(v_c) over the true chunk length: mean |v|, or with
+    // l2 magnitudes ||v_c||_2 / sqrt(len)
+    s_or_q = p.sign_l2 ? __fdiv_rn(__fsqrt_rn(total), __fsqrt_rn((float)len)) : __fdiv_rn(total, (float)len);
     if (chunk_live && t == 0) p.out_scale[(uint64_t)row * p.scale_stride + c] = s_or_q;
   } else {
     // square root and the two divisions once per chunk (its first warp), not once per thread
@@ -269,7 +271,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
 }
 
 template <int OP, int SRC, int V, int LOG2G>
-__global__ void __launch_bounds__(kThreads) k_chunked(const SrcParams src, const ChunkParams p) {
+__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : kServerCtasPerSm) k_chunked(const SrcParams src, const ChunkParams p) {
   pdl_prologue();
   __shared__ float s_red[64];
   __shared__ float s_scal[16];

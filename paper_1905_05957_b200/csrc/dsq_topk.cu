@@ -204,7 +204,7 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
       ee[j] = base + (uint64_t)(j * kThreads + tid) * 4u;
       cnt[j] = FULL ? 4u : (ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u);
     }
-    src_load_tile<SRC, 4>(src, row, ee, cnt, v);
+    src_load_tile<SRC, 4, kThreads * 4>(src, row, ee, cnt, v);
   }
   if constexpr (FULL) {
     float4* op = reinterpret_cast<float4*>(out_row + base) + tid;
@@ -229,7 +229,7 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
 }
 
 template <int SRC>
-__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER || SRC == SRC_SRV_TOPK ? 5 : 1) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred, uint2* list,
+__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER || SRC == SRC_SRV_TOPK ? 5 : kServerCtasPerSm) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred, uint2* list,
                                                          uint64_t cap, uint4* tile_info, uint64_t ntile) {
   pdl_prologue();
   __shared__ uint4 s_tot[kThreads / 32];
@@ -701,12 +701,14 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit_list(float* v_io, uint64
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   const uint64_t tile = (uint64_t)blockIdx.x * (kThreads / 32) + (tid >> 5);
   if (tile >= ntile) return;
+  // the first 64 slots of the region are fetched together with the tile's counts (a region always
+  // has kTile slots; those past the count are never looked at), so one memory round trip serves both
+  const uint2* region = list + (uint64_t)row * cap + tile * kTile;
+  uint4 q = reinterpret_cast<const uint4*>(region)[lane];  // 64 entries per trip, two neighbours per lane
   const uint4 info = tile_info[(uint64_t)row * ntile + tile];
+  const uint2 pre = tile_pre[(uint64_t)row * ntile + tile];
   const uint32_t n = min(info.x, (uint32_t)kTile);
   if (n == 0) return;
-  const uint2* region = list + (uint64_t)row * cap + tile * kTile;
-  uint4 q = region_batch(region, 0, n, lane);  // 64 entries per trip, two neighbours per lane
-  const uint2 pre = tile_pre[(uint64_t)row * ntile + tile];
   const uint32_t tau = state[row].tau, r = state[row].r, zeroed_above = state[row].zeroed_above;
   const bool ties = info.w != 0;  // the tile holds an entry equal to tau
   const uint32_t lt = (1u << lane) - 1u;
@@ -779,7 +781,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_pass1_basic(const SrcParams s
       ee[j] = base + (uint64_t)(j * kThreads + tid) * 4u;
       cnt[j] = ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u;
     }
-    src_load_tile<SRC, 4>(src, row, ee, cnt, v);
+    src_load_tile<SRC, 4, kThreads * 4>(src, row, ee, cnt, v);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (!cnt[j]) continue;

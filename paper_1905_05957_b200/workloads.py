@@ -42,6 +42,7 @@ class Q:
     chunk: int = 0
     k: int = 0
     levels: int = 0
+    norm: int = 1            # sign1: scale from l1 (1) or l2 (2) magnitudes
 
 
 @dataclass(frozen=True)
@@ -77,6 +78,10 @@ def _wl() -> dict[int, Workload]:
                     Q("topk", k=d3 // 100), Q("topk", k=d3 // 100)),
         4: Workload(4, "qsgd255_n8_gpt2small", 8, 124_439_808, 10, "student_t", q2048, q2048),
         5: Workload(5, "sign1_topk_n32_d60m", 32, d5, 50, "hetero", s4096, Q("topk", k=d5 // 200)),
+        # beyond the five listed configurations: the shape of workload 2 with the 1-bit scale taken
+        # from l2 magnitudes (the norm Section 3.2 prints)
+        6: Workload(6, "sign1l2_n8_resnet18", 8, 11_689_512, 20, "layered",
+                    Q("sign1", chunk=4096, norm=2), Q("sign1", chunk=4096, norm=2)),
     }
 
 

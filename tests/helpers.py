@@ -10,7 +10,7 @@ REL_TOL = 1e-5   # bar for fp32 values, scales and delta (reduction order may di
 
 
 def to_oracle_q(q: Q) -> oracle.QSpec:
-    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels)
+    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels, norm=q.norm)
 
 
 def u32(t) -> np.ndarray:

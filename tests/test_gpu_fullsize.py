@@ -1,4 +1,4 @@
-"""The five workloads at full size, in the launch configuration the benchmark times: one step from
+"""The benchmark workloads at full size, in the launch configuration the benchmark times: one step from
 a seeded random state (non-zero errors and model), compared with the oracle element by element."""
 import numpy as np
 import psutil
@@ -12,7 +12,7 @@ from tests.helpers import compare_state, to_oracle_q
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6])
 def test_full_size_step_matches_oracle(wid):
     wl = WORKLOADS[wid]
     need = 4 * wl.n * wl.d * 4 + (2 << 30)

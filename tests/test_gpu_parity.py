@@ -10,6 +10,7 @@ from tests.helpers import compare_state, to_oracle_q
 pytestmark = pytest.mark.gpu
 
 SIGN = lambda L=4096: Q("sign1", chunk=L)
+SIGN_L2 = lambda L=4096: Q("sign1", chunk=L, norm=2)
 QSGD = lambda L=2048, s=255: Q("qsgd", chunk=L, levels=s)
 TOPK = lambda k: Q("topk", k=k)
 IDENT = Q("identity")
@@ -50,6 +51,20 @@ def randn_steps(n, d, T, seed=0, scale=1.0):
 @pytest.mark.parametrize("L", [128, 1024, 4096, 8192])
 def test_sign1_both_passes(d, L):
     run_lockstep(3, d, SIGN(L), SIGN(L), randn_steps(3, d, 3, seed=d + L))
+
+
+@pytest.mark.parametrize("d", [4096, 10_000, 65_536 + 4 * 37, 33, 1])
+@pytest.mark.parametrize("L", [128, 2048, 4096, 8192])
+def test_sign1_l2_magnitudes_both_passes(d, L):
+    run_lockstep(3, d, SIGN_L2(L), SIGN_L2(L), randn_steps(3, d, 3, seed=d + L + 1))
+
+
+def test_sign1_l2_mixed_with_other_operators_and_unaligned_rows():
+    d = 50_000 + 13
+    for wq, sq in [(SIGN_L2(4096), TOPK(500)), (SIGN_L2(512), SIGN(2048)), (QSGD(1024, 31), SIGN_L2(4096)),
+                   (TOPK(700), SIGN_L2(1024)), (IDENT, SIGN_L2(128))]:
+        run_lockstep(4, d, wq, sq, randn_steps(4, d, 2, seed=41))
+    run_lockstep(3, 30_000, SIGN_L2(4096), SIGN_L2(4096), randn_steps(3, 30_000, 3, seed=42), fuse=False)
 
 
 @pytest.mark.parametrize("d", [2048, 10_000, 40_000 + 4, 5])
@@ -117,7 +132,7 @@ def test_zero_signed_zero_subnormal_and_zero_chunks():
     g[:, 5000:5100] = 1e-41      # subnormals
     g[:, 5100:5200] = -1e-41
     g[0, 8192:] = 1e-30          # squares underflow: a quantisation chunk of norm ~0
-    for wq in (SIGN(4096), QSGD(2048), TOPK(100), SIGN(128), QSGD(128, 5)):
+    for wq in (SIGN(4096), QSGD(2048), TOPK(100), SIGN(128), QSGD(128, 5), SIGN_L2(4096), SIGN_L2(128)):
         run_lockstep(n, d, wq, wq, [g, g.clone(), -g])
 
 
@@ -154,7 +169,7 @@ def test_many_workers_and_one_worker():
 
 # ------------------------------------------------------------------ the five workloads, scaled down
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6])
 def test_workload_recipes_scaled(wid):
     wl = WORKLOADS[wid]
     wl = wl if wid == 1 else wl.scaled(d=200_000 + 40, n=min(wl.n, 8), steps=4)

@@ -8,11 +8,12 @@ from oracle import QSpec
 QS = {
     "identity": QSpec(oracle.IDENTITY),
     "sign1": QSpec(oracle.SIGN1, chunk=128),
+    "sign1_l2": QSpec(oracle.SIGN1, chunk=128, norm=2),
     "topk": QSpec(oracle.TOPK, k=37),
     "qsgd": QSpec(oracle.QSGD, chunk=128, levels=15),
 }
 PAIRS = [("identity", "identity"), ("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"),
-         ("sign1", "topk"), ("topk", "identity"), ("qsgd", "sign1")]
+         ("sign1", "topk"), ("topk", "identity"), ("qsgd", "sign1"), ("sign1_l2", "sign1_l2"), ("sign1_l2", "sign1")]
 
 
 def _grads(n, d, T, seed=0):
@@ -73,7 +74,7 @@ def test_telescoping_identity_of_the_global_update_rule(wq, sq):
     assert np.max(np.abs(lhs - rhs)) <= 40 * T * 2.0**-24 * scale
 
 
-@pytest.mark.parametrize("wq,sq", [("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd")])
+@pytest.mark.parametrize("wq,sq", [("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"), ("sign1_l2", "sign1_l2")])
 def test_error_stays_bounded_on_stationary_gradients(wq, sq):
     """Section 4: a contracting Q keeps ||delta_t|| bounded; a broken residual makes it grow."""
     n, d, T = 2, 512, 120

@@ -19,8 +19,14 @@ MUTANTS = [
      "  float s = 0.0f; for (size_t i = 0; i < len; ++i) s = s + a[i];\n  return s;",
      lambda: [t_prim.test_pairwise_sum_hand_derived(e, i) for e, i in t_prim._cases()]),
     ("sign scale divides by the nominal chunk length",
-     "float s = l1 / (float)len;", "float s = l1 / (float)L;",
+     "s = l1 / (float)len;", "s = l1 / (float)L;",
      t_ops.test_sign1_short_last_chunk_divides_by_true_length),
+    ("l2 sign scale divides by the length instead of its root",
+     "s = l2 / root_len;", "s = l2 / (float)len;",
+     lambda: t_ops.test_sign1_l2_scale_is_rms_and_keeps_the_l2_magnitude(10000, 4096)),
+    ("l2 sign scale sums |v| instead of v*v",
+     "float e2 = e * e;\n        term[t] = e2;", "float e2 = fabsf(e);\n        term[t] = e2;",
+     lambda: t_ops.test_sign1_l2_scale_is_rms_and_keeps_the_l2_magnitude(10000, 4096)),
     ("sign bit is v > 0",
      "int nonneg = v[j] >= 0.0f;\n      if (nonneg) bits[j / 32]", "int nonneg = v[j] > 0.0f;\n      if (nonneg) bits[j / 32]",
      lambda: t_ops.test_sign1_scale_is_l1_mean_per_chunk_and_bits_are_signs(10000, 4096)),

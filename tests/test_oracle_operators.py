@@ -60,6 +60,54 @@ def test_sign1_short_last_chunk_divides_by_true_length():
     assert p["scale"].tolist() == [2.0, 2.0]   # a divide by L would give 6/128
 
 
+@pytest.mark.parametrize("d,L", [(4096, 4096), (10000, 4096), (777, 128), (33, 4096), (1, 128)])
+def test_sign1_l2_scale_is_rms_and_keeps_the_l2_magnitude(d, L):
+    """With l2 magnitudes (the norm Section 3.2 prints) the factor of Section 5.1 is
+    ||v_c||_2 / ||sign(v_c)||_2 = ||v_c||_2 / sqrt(len_c), and the recovered chunk has the l2
+    magnitude of the compensated one."""
+    v = _rng(3 * d + 1).standard_normal(d).astype(np.float32)
+    v[::5] = 0.0
+    C, p = oracle.q_sign1(v, L, norm=2)
+    C1, p1 = oracle.q_sign1(v, L, norm=1)
+    nc = (d + L - 1) // L
+    for c in range(nc):
+        seg = v[c * L:(c + 1) * L].astype(np.float64)
+        rms = math.sqrt((seg**2).sum() / len(seg))
+        assert abs(float(p["scale"][c]) - rms) <= 1e-6 * rms + 1e-30
+        got = math.sqrt((C[c * L:(c + 1) * L].astype(np.float64) ** 2).sum())
+        assert abs(got - math.sqrt((seg**2).sum())) <= 2e-6 * math.sqrt((seg**2).sum()) + 1e-30
+        # root mean square >= mean absolute value (Cauchy-Schwarz), equal only for constant |v|
+        assert float(p["scale"][c]) >= float(p1["scale"][c]) * (1 - 1e-6)
+    assert np.array_equal(p["bits"], p1["bits"])           # the signs do not depend on the norm
+    assert np.array_equal(oracle.decode_sign1(p["bits"], p["scale"], d, L), C)
+
+
+def test_sign1_l2_constant_chunk_short_chunk_and_residual_energy():
+    L = 4096
+    # constant magnitude: l2 and l1 factors coincide and the chunk is represented exactly
+    w = np.where(_rng(13).random(L) < 0.5, np.float32(0.375), np.float32(-0.375)).astype(np.float32)
+    C, p = oracle.q_sign1(w, L, norm=2)
+    assert float(p["scale"][0]) == 0.375 and np.array_equal(C, w)
+    # short last chunk: the root of the TRUE length divides (sqrt(4 * 9) / sqrt(4) = 3)
+    v = np.full(128 + 4, 3.0, dtype=np.float32)
+    _, p = oracle.q_sign1(v, 128, norm=2)
+    assert p["scale"].tolist() == [3.0, 3.0]
+    # residual energy: ||v - s sign(v)||^2 = 2 ||v||_2^2 - 2 s ||v||_1 with s = ||v||_2 / sqrt(len)
+    v = _rng(14).standard_normal(2 * L).astype(np.float32)
+    C, p = oracle.q_sign1(v, L, norm=2)
+    delta = oracle.residual(v, C).astype(np.float64)
+    for c in range(2):
+        seg = v[c * L:(c + 1) * L].astype(np.float64)
+        s = math.sqrt((seg**2).sum() / L)
+        closed = 2 * (seg**2).sum() - 2 * s * np.abs(seg).sum()
+        assert abs((delta[c * L:(c + 1) * L] ** 2).sum() - closed) <= 1e-5 * (seg**2).sum()
+
+
+def test_sign1_rejects_unknown_norm():
+    with pytest.raises(ValueError):
+        oracle.q_sign1(np.ones(8, np.float32), 128, norm=3)
+
+
 # ------------------------------------------------------------------ top-k
 
 def _brute_topk(v, k):
