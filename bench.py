@@ -35,8 +35,8 @@ NCU_TRAFFIC = {
     2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748234752 + 335448320, "cb37fb5109354746"),
 }
 KERNEL_SOURCES = {  # files whose change invalidates the captured counters
-    "sign1": ("dsq_chunked.cu", "dsq_common.cuh", "dsq_internal.h"),
-    "qsgd": ("dsq_chunked.cu", "dsq_common.cuh", "dsq_internal.h"),
+    "sign1": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
+    "qsgd": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
     "topk": ("dsq_topk.cu", "dsq_common.cuh", "dsq_internal.h"),
     "identity": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
 }

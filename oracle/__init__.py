@@ -14,7 +14,7 @@ import numpy as np
 
 from . import build as _build
 
-IDENTITY, SIGN1, TOPK, QSGD = "identity", "sign1", "topk", "qsgd"
+IDENTITY, SIGN1, TOPK, QSGD, CLIP = "identity", "sign1", "topk", "qsgd", "clip"
 SERVER_WID = 0xFFFFFFFF
 
 _lib = None
@@ -44,6 +44,8 @@ def load(path: str):
     L.orc_decode_topk.argtypes = [u32p, f32p, u64, u64, f32p]
     L.orc_q_qsgd.argtypes = [f32p, u64, u32, u32, u64, u32, u32, u8p, u32p, f32p, f32p, f32p]
     L.orc_decode_qsgd.argtypes = [u8p, u32p, f32p, u64, u32, f32p]
+    L.orc_q_clip.argtypes = [f32p, u64, u32, u8p, f32p]
+    L.orc_decode_clip.argtypes = [u8p, u64, u32, f32p]
     return L
 
 
@@ -125,6 +127,7 @@ class QSpec:
     norm: int = 1       # sign1: the scale is the ratio of l1 (1) or l2 (2) magnitudes
     k: int = 0          # topk
     levels: int = 0     # qsgd: s
+    bits: int = 0       # clip: how many low bits of each binary32 number are set to zero (16 or 24)
 
 
 def q_identity(v):
@@ -198,6 +201,22 @@ def decode_qsgd(lvl, sgn, qstep, d, L):
     return Cv
 
 
+def q_clip(v, b):
+    v = _f32(v)
+    d = v.size
+    hi = np.zeros(d * ((32 - b) // 8 if b in (16, 24) else 1), dtype=np.uint8)
+    Cv = np.empty_like(v)
+    _check(lib().orc_q_clip(_p(v, C.c_float), d, b, _p(hi, C.c_uint8), _p(Cv, C.c_float)), "clip")
+    return Cv, {"hi": hi.view(np.uint16) if b == 16 else hi}
+
+
+def decode_clip(hi, d, b):
+    hi = np.ascontiguousarray(hi).view(np.uint8)
+    Cv = np.empty(d, dtype=np.float32)
+    _check(lib().orc_decode_clip(_p(hi, C.c_uint8), d, b, _p(Cv, C.c_float)), "decode_clip")
+    return Cv
+
+
 def compress(q: QSpec, v, seed=0, step=0, wid=0):
     """Q_omega[v] for the operator ``q``; omega = (seed, step, wid) where Q is random."""
     if q.op == IDENTITY:
@@ -208,6 +227,8 @@ def compress(q: QSpec, v, seed=0, step=0, wid=0):
         return q_topk(v, q.k)
     if q.op == QSGD:
         return q_qsgd(v, q.chunk, q.levels, seed, step, wid)
+    if q.op == CLIP:
+        return q_clip(v, q.bits)
     raise ValueError(q.op)
 
 

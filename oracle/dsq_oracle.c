@@ -24,7 +24,8 @@
  * C + delta_new == g + delta_old; the telescoping identity of Section 3.3
  * (Eq. 5-6); sign scale == ||v||_1/len (or ||v||_2/sqrt(len)) and its closed-form residual energy;
  * top-k against a brute-force stable sort; QSGD unbiasedness and variance by
- * Monte Carlo plus its deterministic special cases; Philox4x32-10 against an
+ * Monte Carlo plus its deterministic special cases; clipping against worked
+ * binary cases, its error bound and idempotence; Philox4x32-10 against an
  * independent library implementation; pairwise summation against hand-derived
  * rounding cases.  No function here is "parity unpinned".
  */
@@ -207,6 +208,42 @@ int orc_decode_sign1(const uint32_t* bits, const float* scale, uint64_t d, uint3
     float s = scale[j / L];
     int nonneg = (bits[j / 32] >> (j % 32)) & 1u;
     C[j] = nonneg ? s : -s;
+  }
+  return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Q = clipping (Section 3.2 "Clipping": set the lower bits of every number  */
+/* to zero; deterministic and biased).  Reading: the number is its binary32  */
+/* representation and its low b bits are cleared, which keeps the sign, the  */
+/* exponent and the leading 23 - b fraction bits (b <= 23), i.e. truncates   */
+/* the magnitude toward zero.  What is sent per entry is the surviving high  */
+/* 32 - b bits; b is 16 or 24 so that an entry is a 16- or an 8-bit word.    */
+/*   hi : d words of (32 - b) bits, little-endian bytes                      */
+/*   C  : d floats (may be NULL)                                             */
+/* ------------------------------------------------------------------------ */
+
+int orc_q_clip(const float* v, uint64_t d, uint32_t b, uint8_t* hi, float* C) {
+  if (b != 16 && b != 24) return ORC_ERR_ARG;
+  uint32_t bytes = (32 - b) / 8;
+  for (uint64_t j = 0; j < d; ++j) {
+    uint32_t u = f32_bits(v[j]);
+    uint32_t kept = u >> b;       /* the high 32 - b bits */
+    uint32_t cleared = kept << b; /* the number with its low b bits set to zero */
+    for (uint32_t t = 0; t < bytes; ++t) hi[j * bytes + t] = (uint8_t)(kept >> (8 * t));
+    if (C) memcpy(&C[j], &cleared, sizeof cleared);
+  }
+  return ORC_OK;
+}
+
+int orc_decode_clip(const uint8_t* hi, uint64_t d, uint32_t b, float* C) {
+  if (b != 16 && b != 24) return ORC_ERR_ARG;
+  uint32_t bytes = (32 - b) / 8;
+  for (uint64_t j = 0; j < d; ++j) {
+    uint32_t kept = 0;
+    for (uint32_t t = 0; t < bytes; ++t) kept |= (uint32_t)hi[j * bytes + t] << (8 * t);
+    uint32_t u = kept << b;
+    memcpy(&C[j], &u, sizeof u);
   }
   return ORC_OK;
 }

@@ -1,18 +1,23 @@
-"""Compile the CUDA library in-tree: paper_1905_05957_b200/csrc/libdsq.so (sm_100a only)."""
+"""Compile the CUDA library in-tree: paper_1905_05957_b200/csrc/libdsq.so (sm_100a only).
+
+Every translation unit is compiled to an object file on its own (side by side), then linked."""
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(CSRC, "libdsq.so")
-SOURCES = ["dsq_api.cu", "dsq_chunked.cu", "dsq_elementwise.cu", "dsq_topk.cu", "dsq_static.cu"]
-HEADERS = ["dsq_common.cuh", "dsq_internal.h", os.path.join("..", "..", "include", "dsq.h")]
+SOURCES = ["dsq_api.cu", "dsq_chunked.cu", "dsq_chunked_sign.cu", "dsq_chunked_sign_l2.cu", "dsq_chunked_qsgd.cu",
+           "dsq_elementwise.cu", "dsq_topk.cu", "dsq_static.cu"]
+HEADERS = ["dsq_common.cuh", "dsq_chunked.cuh", "dsq_internal.h", os.path.join("..", "..", "include", "dsq.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-fmad=false",                      # every multiply and add rounds separately
-    "-Xcompiler", "-fPIC", "-shared",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -27,9 +32,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-          ["-o", LIB + ".tmp"] + [os.path.join(CSRC, f) for f in SOURCES]
-    subprocess.run(cmd, check=True)
+    os.makedirs(OBJ, exist_ok=True)
+    extra = ["-Xptxas", "-v"] if verbose else []
+
+    def compile_one(src: str) -> str:
+        obj = os.path.join(OBJ, src[:-3] + ".o")
+        subprocess.run([nvcc] + NVCC_FLAGS + extra + ["-c", os.path.join(CSRC, src), "-o", obj], check=True)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(compile_one, SOURCES))
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB + ".tmp"] + objs, check=True)
     os.replace(LIB + ".tmp", LIB)
     return LIB
 

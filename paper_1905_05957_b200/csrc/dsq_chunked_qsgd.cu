@@ -1,0 +1,9 @@
+// Randomised s-level quantisation: instantiations of the chunk kernel.
+#include "dsq_chunked.cuh"
+
+namespace dsq {
+cudaError_t launch_chunked_qsgd(int srck, const SrcParams& src, const ChunkParams& p, uint32_t rows, uint32_t chunk,
+                                cudaStream_t st) {
+  return launch_src<DS_Q_QSGD>(srck, src, p, rows, chunk, st);
+}
+}  // namespace dsq

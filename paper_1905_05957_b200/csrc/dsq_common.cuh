@@ -10,8 +10,8 @@ namespace dsq {
 constexpr int kThreads = 256;  // every streaming kernel uses 256-thread CTAs
 
 // Kernels that decode worker payloads (server passes) are compiled for this many CTAs per SM: they
-// are bound by instruction issue, and four resident CTAs hide the latency of the payload loads
-// better than a larger register budget does (measured).
+// are bound by instruction issue and by the latency of the payload loads, and four resident CTAs
+// serve both better than a larger register budget does (measured on all server kernels).
 constexpr int kServerCtasPerSm = 4;
 
 // Kernels are launched with programmatic stream serialization: once every CTA of a kernel has
@@ -118,118 +118,14 @@ __device__ __forceinline__ float signed_by_bit(float m, uint32_t w, int k) {
 // Exact float value of byte `k` of `x` (one conversion instruction with a byte selector).
 __device__ __forceinline__ float byte_to_float(uint32_t x, int k) { return __uint2float_rn((x >> (8 * k)) & 0xFFu); }
 
-// +m or -m according to the sign bit of entry k inside `byte` (a byte of a sign word; 1 = non-negative).
-// pw_k = 2^(31 - position of the bit): the product moves that bit to bit 31 (the multiply runs on
-// the multiply-add pipe, which the adds leave half idle; a shift would queue up with the logic
-// instruction that follows it).
-__device__ __forceinline__ float signed_by_byte(float m, uint32_t byte, uint32_t pw_k) {
-  return __uint_as_float(__float_as_uint(m) ^ (~(byte * pw_k) & 0x80000000u));
-}
-
-// Adds the decoded payloads of B consecutive workers to acc, in worker order.  Every lane fetches
-// the byte that holds the four sign bits of its row itself (neighbouring lanes share bytes, a warp
-// reads 16 consecutive bytes: one L1 access) and the scale of the row's chunk (one address for the
-// whole warp row).  sgn / scl / lvl point at this thread's first row in the first of the B
-// payloads; row j starts RS entries after row j-1, so every load is a per-worker address plus a
-// constant.  SAME: all rows of the thread lie in one chunk and one scale load per worker serves
-// them all.  ALL: B workers exist and every row is inside the vector, nothing is predicated.
-template <int SRC, int V, int RS, bool SAME, bool ALL, int B>
-__device__ __forceinline__ void add_decoded(const SrcParams& p, uint32_t left, const uint8_t* sgn, const float* scl,
-                                            const uint8_t* lvl, const uint32_t (&cstep)[V], const uint32_t (&cnt)[V],
-                                            const uint32_t (&pw)[4], float4 (&acc)[V]) {
-  constexpr int NS = SAME ? 1 : V;
-  uint32_t sb[V][B];
-  float sc[NS][B];
-  uint32_t lv[SRC == SRC_SRV_QSGD ? V : 1][SRC == SRC_SRV_QSGD ? B : 1];
-#pragma unroll
-  for (int u = 0; u < B; ++u) {
-    const bool on = ALL || (uint32_t)u < left;
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-      if (ALL) {
-        sb[j][u] = __ldg(sgn + j * (RS / 8));
-        if (j < NS) sc[j][u] = __ldg(scl + cstep[j]);
-        if constexpr (SRC == SRC_SRV_QSGD) lv[j][u] = __ldcs(reinterpret_cast<const uint32_t*>(lvl + j * RS));
-      } else {
-        sb[j][u] = 0;
-        if (on && cnt[j]) sb[j][u] = __ldg(sgn + j * (RS / 8));
-        if (j < NS) {
-          sc[j][u] = 0.f;
-          if (on && cnt[j]) sc[j][u] = __ldg(scl + cstep[j]);
-        }
-        if constexpr (SRC == SRC_SRV_QSGD) {
-          lv[j][u] = 0;
-          if (on && cnt[j]) lv[j][u] = __ldcs(reinterpret_cast<const uint32_t*>(lvl + j * RS));
-        }
-      }
-    }
-    sgn += p.wp_stride;
-    scl = reinterpret_cast<const float*>(reinterpret_cast<const uint8_t*>(scl) + p.wp_stride);
-    if constexpr (SRC == SRC_SRV_QSGD) lvl += p.wp_stride;
-  }
-#pragma unroll
-  for (int u = 0; u < B; ++u) {
-    if (ALL || (uint32_t)u < left) {
-#pragma unroll
-      for (int j = 0; j < V; ++j) {
-        const float s = sc[SAME ? 0 : j][u];
-        const uint32_t b = sb[j][u];
-        if constexpr (SRC == SRC_SRV_SIGN1) {
-          acc[j] = add4_rn(acc[j], make_float4(signed_by_byte(s, b, pw[0]), signed_by_byte(s, b, pw[1]),
-                                               signed_by_byte(s, b, pw[2]), signed_by_byte(s, b, pw[3])));
-        } else {
-          const uint32_t l4 = lv[j][u];
-          const float4 mag = mul4_rn(make_float4(byte_to_float(l4, 0), byte_to_float(l4, 1), byte_to_float(l4, 2),
-                                                 byte_to_float(l4, 3)),
-                                     make_float4(s, s, s, s));
-          acc[j] = add4_rn(acc[j], make_float4(signed_by_byte(mag.x, b, pw[0]), signed_by_byte(mag.y, b, pw[1]),
-                                               signed_by_byte(mag.z, b, pw[2]), signed_by_byte(mag.w, b, pw[3])));
-        }
-      }
-    }
-  }
-}
-
-// All n workers through add_decoded, B at a time.
-template <int SRC, int V, int RS, bool SAME, int B>
-__device__ __forceinline__ void add_decoded_all(const SrcParams& p, uint64_t e0, const uint32_t (&cnt)[V],
-                                                const uint32_t (&pw)[4], float4 (&acc)[V]) {
-  constexpr int kSgn = SRC == SRC_SRV_SIGN1 ? 0 : 1;    // payload sub-array of the sign words
-  constexpr int kScl = SRC == SRC_SRV_SIGN1 ? 1 : 2;    // ... of the per-chunk scale / grid step
-  const uint8_t* sgn = p.wp + p.wp_off[kSgn] + (e0 >> 3);
-  const float* scl = reinterpret_cast<const float*>(p.wp + p.wp_off[kScl]) + (e0 >> p.w_log2_chunk);
-  const uint8_t* lvl = p.wp + p.wp_off[0] + e0;
-  uint32_t cstep[V];  // chunk of row j minus chunk of row 0
-  bool all = true;
-#pragma unroll
-  for (int j = 0; j < V; ++j) {
-    cstep[j] = (uint32_t)(((e0 + (uint64_t)j * RS) >> p.w_log2_chunk) - (e0 >> p.w_log2_chunk));
-    all = all && cnt[j] != 0;
-  }
-  const uint64_t batch = (uint64_t)B * p.wp_stride;
-  uint32_t i0 = 0;
-  if (all) {
-    for (; i0 + B <= p.n; i0 += B) {
-      add_decoded<SRC, V, RS, SAME, true, B>(p, B, sgn, scl, lvl, cstep, cnt, pw, acc);
-      sgn += batch;
-      scl = reinterpret_cast<const float*>(reinterpret_cast<const uint8_t*>(scl) + batch);
-      lvl += batch;
-    }
-  }
-  for (; i0 < p.n; i0 += B) {
-    add_decoded<SRC, V, RS, SAME, false, B>(p, p.n - i0, sgn, scl, lvl, cstep, cnt, pw, acc);
-    sgn += batch;
-    scl = reinterpret_cast<const float*>(reinterpret_cast<const uint8_t*>(scl) + batch);
-    lvl += batch;
-  }
-}
-
 // The vector to compress, for a tile of V rows: row j of the calling thread is the float4 at entry
 // e[j] of vector `row`; cnt[j] in [0, 4] says how many of its entries exist (the others, and whole
-// rows with cnt 0, are returned as +0).  The e[j] are multiples of 4 and RS entries apart
-// (e[j] = e[0] + j * RS, RS a multiple of 128).  Workers are accumulated in order 0..n-1, the order
-// in which Eq. 4 is summed.
-template <int SRC, int V, int RS>
+// rows with cnt 0, are returned as +0).  Must be called by all 32 lanes of a warp together, the
+// lanes holding consecutive float4 of each row (e[j] = 128-aligned warp base + 4 * lane): server
+// sources load the sign words and scales of eight workers with one instruction per row (lane l
+// fetches word l%4 of worker l/4) and hand them round with shuffles.  Workers are accumulated in
+// order 0..n-1, the order in which Eq. 4 is summed.
+template <int SRC, int V>
 __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, const uint64_t (&e)[V],
                                               const uint32_t (&cnt)[V], float4 (&v)[V]) {
   if constexpr (SRC == SRC_WORKER) {
@@ -243,6 +139,7 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
     for (int j = 0; j < V; ++j)
       v[j] = add4_rn(a[j], b[j]);
   } else {
+    const uint32_t lane = threadIdx.x & 31u;
     float4 acc[V], ds[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) {
@@ -261,23 +158,57 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
         }
       }
     } else if constexpr (SRC == SRC_SRV_SIGN1 || SRC == SRC_SRV_QSGD) {
-      // the sign bits of the row's entries k = 0..3 sit at bits sh + k of their byte
-      const uint32_t sh = (uint32_t)e[0] & 4u;
-      uint32_t pw[4];
+      constexpr int kSgn = SRC == SRC_SRV_SIGN1 ? 0 : 1;    // payload sub-array of the sign words
+      constexpr int kScl = SRC == SRC_SRV_SIGN1 ? 1 : 2;    // ... of the per-chunk scale / grid step
+      const uint64_t nw = (p.d + 31) >> 5;
+      const uint32_t sh = (lane & 7u) * 4u;                 // this lane's nibble inside its word
+      for (uint32_t i0 = 0; i0 < p.n; i0 += 8) {
+        uint32_t wreg[V];
+        float sreg[V];
+        uint32_t lv[SRC == SRC_SRV_QSGD ? V : 1][SRC == SRC_SRV_QSGD ? 8 : 1];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        pw[k] = 1u << (31 - k - sh);
-        asm volatile("" : "+r"(pw[k]));  // stays a multiplier: not to be folded back into a shift
-      }
-      constexpr int kB = 4;  // workers fetched at once (their loads are in flight together)
-      bool same = true;
+        for (int j = 0; j < V; ++j) {
+          // warp base of this row: entry of lane 0 (valid arithmetic even where the row is past the end)
+          const uint64_t e0 = e[j] - 4u * lane;
+          const uint64_t word = (e0 >> 5) + (lane & 3u);
+          const uint32_t wi = i0 + (lane >> 2);
+          wreg[j] = 0;
+          sreg[j] = 0.f;
+          if (wi < p.n && word < nw)
+            wreg[j] = __ldg(reinterpret_cast<const uint32_t*>(p.wp + wi * p.wp_stride + p.wp_off[kSgn]) + word);
+          if (lane < 8 && i0 + lane < p.n && e0 < p.d)
+            sreg[j] = __ldg(reinterpret_cast<const float*>(p.wp + (i0 + lane) * p.wp_stride + p.wp_off[kScl]) +
+                            (e0 >> p.w_log2_chunk));
+          if constexpr (SRC == SRC_SRV_QSGD) {
 #pragma unroll
-      for (int j = 1; j < V; ++j)
-        if (cnt[j] && (e[j] >> p.w_log2_chunk) != (e[0] >> p.w_log2_chunk)) same = false;
-      if (same) {
-        add_decoded_all<SRC, V, RS, true, kB>(p, e[0], cnt, pw, acc);
-      } else {
-        add_decoded_all<SRC, V, RS, false, kB>(p, e[0], cnt, pw, acc);
+            for (int u = 0; u < 8; ++u) {
+              lv[j][u] = 0;
+              if (i0 + u < p.n && cnt[j])
+                lv[j][u] = __ldcs(reinterpret_cast<const uint32_t*>(p.wp + (i0 + u) * p.wp_stride + p.wp_off[0] + e[j]));
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const uint32_t ww = __shfl_sync(0xffffffffu, wreg[j], u * 4 + (lane >> 3)) >> sh;
+            const float sc = __shfl_sync(0xffffffffu, sreg[j], u);
+            if (i0 + u < p.n) {
+              if constexpr (SRC == SRC_SRV_SIGN1) {
+                acc[j] = add4_rn(acc[j], make_float4(signed_by_bit(sc, ww, 0), signed_by_bit(sc, ww, 1),
+                                                     signed_by_bit(sc, ww, 2), signed_by_bit(sc, ww, 3)));
+              } else {
+                const uint32_t l4 = lv[j][u];
+                const float4 mag = mul4_rn(make_float4(byte_to_float(l4, 0), byte_to_float(l4, 1), byte_to_float(l4, 2),
+                                                       byte_to_float(l4, 3)),
+                                           make_float4(sc, sc, sc, sc));
+                acc[j] = add4_rn(acc[j], make_float4(signed_by_bit(mag.x, ww, 0), signed_by_bit(mag.y, ww, 1),
+                                                     signed_by_bit(mag.z, ww, 2), signed_by_bit(mag.w, ww, 3)));
+              }
+            }
+          }
+        }
       }
     } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc (cleared before every use)
 #pragma unroll

@@ -20,7 +20,7 @@ __global__ void __launch_bounds__(kThreads) k_identity(const SrcParams src, floa
     const uint32_t cc[1] = {e < src.d ? (uint32_t)min((uint64_t)4, src.d - e) : 0u};
     const uint32_t cnt = cc[0];
     float4 vv[1];
-    src_load_tile<SRC, 1, 0>(src, row, ee, cc, vv);
+    src_load_tile<SRC, 1>(src, row, ee, cc, vv);
     const float4 v = vv[0];
     if (!cnt) continue;
     store_row4(out_c + (uint64_t)row * c_row_stride, e, cnt, 1, v);  // Q[v] = v

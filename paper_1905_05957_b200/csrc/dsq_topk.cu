@@ -204,7 +204,7 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
       ee[j] = base + (uint64_t)(j * kThreads + tid) * 4u;
       cnt[j] = FULL ? 4u : (ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u);
     }
-    src_load_tile<SRC, 4, kThreads * 4>(src, row, ee, cnt, v);
+    src_load_tile<SRC, 4>(src, row, ee, cnt, v);
   }
   if constexpr (FULL) {
     float4* op = reinterpret_cast<float4*>(out_row + base) + tid;
@@ -781,7 +781,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_pass1_basic(const SrcParams s
       ee[j] = base + (uint64_t)(j * kThreads + tid) * 4u;
       cnt[j] = ee[j] < d ? (uint32_t)min((uint64_t)4, d - ee[j]) : 0u;
     }
-    src_load_tile<SRC, 4, kThreads * 4>(src, row, ee, cnt, v);
+    src_load_tile<SRC, 4>(src, row, ee, cnt, v);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       if (!cnt[j]) continue;

@@ -11,9 +11,11 @@ QS = {
     "sign1_l2": QSpec(oracle.SIGN1, chunk=128, norm=2),
     "topk": QSpec(oracle.TOPK, k=37),
     "qsgd": QSpec(oracle.QSGD, chunk=128, levels=15),
+    "clip": QSpec(oracle.CLIP, bits=16),
 }
 PAIRS = [("identity", "identity"), ("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"),
-         ("sign1", "topk"), ("topk", "identity"), ("qsgd", "sign1"), ("sign1_l2", "sign1_l2"), ("sign1_l2", "sign1")]
+         ("sign1", "topk"), ("topk", "identity"), ("qsgd", "sign1"), ("sign1_l2", "sign1_l2"), ("sign1_l2", "sign1"),
+         ("clip", "clip"), ("clip", "topk"), ("sign1", "clip")]
 
 
 def _grads(n, d, T, seed=0):
@@ -48,7 +50,7 @@ def test_residual_reconstructs_compensated_gradient(wq, sq):
         v_w = g + old_w
         tol = 2.0**-23 * np.maximum(np.abs(v_w), np.abs(C_all))
         assert np.all(np.abs((C_all.astype(np.float64) + st.delta_w) - v_w) <= tol)
-        if wq in ("identity", "topk"):
+        if wq in ("identity", "topk", "clip"):
             assert np.array_equal(C_all + st.delta_w, v_w)
         Cv = oracle.server_pass(st, C_all, QS[sq], 1, t)
         v_s = oracle.server_mean_add(C_all, old_s)

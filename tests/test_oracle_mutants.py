@@ -27,6 +27,12 @@ MUTANTS = [
     ("l2 sign scale sums |v| instead of v*v",
      "float e2 = e * e;\n        term[t] = e2;", "float e2 = fabsf(e);\n        term[t] = e2;",
      lambda: t_ops.test_sign1_l2_scale_is_rms_and_keeps_the_l2_magnitude(10000, 4096)),
+    ("clipping keeps one bit too many",
+     "uint32_t kept = u >> b;       /* the high 32 - b bits */", "uint32_t kept = (u >> (b - 1)) << 1 >> 1;",
+     t_ops.test_clip_worked_binary_cases),
+    ("clipping rounds to nearest instead of clearing bits",
+     "uint32_t kept = u >> b;       /* the high 32 - b bits */", "uint32_t kept = (u + (1u << (b - 1))) >> b;",
+     t_ops.test_clip_worked_binary_cases),
     ("sign bit is v > 0",
      "int nonneg = v[j] >= 0.0f;\n      if (nonneg) bits[j / 32]", "int nonneg = v[j] > 0.0f;\n      if (nonneg) bits[j / 32]",
      lambda: t_ops.test_sign1_scale_is_l1_mean_per_chunk_and_bits_are_signs(10000, 4096)),

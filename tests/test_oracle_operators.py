@@ -243,3 +243,57 @@ def test_qsgd_levels_bracket_the_value_and_decode_roundtrip():
     r = np.float32(abs(v[j])) * inv_q
     want = int(np.floor(r)) + (1 if u < float(r - np.floor(r)) else 0)
     assert p["lvl"][j] == want
+
+
+# ------------------------------------------------------------------ clipping
+
+def test_clip_worked_binary_cases():
+    """Section 3.2 "Clipping" clears low bits of the number (its example drops low decimal digits of
+    1.23456); for binary32 with b = 16 the sign, the exponent and 7 fraction bits survive."""
+    one = np.float32(1.0)
+    cases16 = [
+        (1.0, 1.0), (-2.0, -2.0), (1.5, 1.5), (0.0, 0.0),
+        (1.0 + 2.0**-7, 1.0 + 2.0**-7),          # the last surviving fraction bit
+        (1.0 + 2.0**-8, 1.0),                    # the first cleared one
+        (1.0 + 2.0**-7 + 2.0**-9, 1.0 + 2.0**-7),
+        (-(3.0 + 2.0**-10), -3.0),               # truncation is toward zero for negatives too
+        (1.9999999, 1.9921875),                  # 1 + 127/128: never rounds up to 2
+        (float(np.float32(3.14159265)), 3.140625),
+    ]
+    v = np.array([c[0] for c in cases16], dtype=np.float32)
+    want = np.array([c[1] for c in cases16], dtype=np.float32)
+    C, p = oracle.q_clip(v, 16)
+    assert np.array_equal(C, want)
+    assert p["hi"].dtype == np.uint16 and int(p["hi"][0]) == 0x3F80 and int(p["hi"][1]) == 0xC000
+    # b = 24 keeps the sign and the seven high bits of the biased exponent: 1.0 = 0x3F800000 has
+    # exponent field 127 = 0b01111111, whose low bit goes, leaving 126, i.e. 0.5; 3.0 = 0x40400000
+    # keeps field 128, i.e. 2.0; 2^-126 (field 1) falls to 0; 1e30 = 0x7149F2CA -> 0x71000000 = 2^99
+    C, p = oracle.q_clip(np.array([1.0, -1.0, 3.0, 0.75, 2.0**-126, 1e30], dtype=np.float32), 24)
+    assert C.tolist() == [0.5, -0.5, 2.0, 0.5, 0.0, float(2.0**99)]
+    assert p["hi"].dtype == np.uint8 and p["hi"].tolist() == [0x3F, 0xBF, 0x40, 0x3F, 0x00, 0x71] and one == 1.0
+    with pytest.raises(ValueError):
+        oracle.q_clip(v, 12)
+
+
+@pytest.mark.parametrize("b", [16, 24])
+def test_clip_error_bound_idempotence_exact_residual_and_decode(b):
+    r = _rng(50 + b)
+    v = (r.standard_normal(20000) * 10.0 ** r.uniform(-6, 6, 20000)).astype(np.float32)
+    v[:4] = [0.0, -0.0, 1e-41, -1e-41]
+    C, p = oracle.q_clip(v, b)
+    # never grows, never changes sign, and equals the value with its low b bits cleared
+    assert np.all(np.abs(C) <= np.abs(v)) and np.array_equal(np.signbit(C), np.signbit(v))
+    mask = np.uint32((0xFFFFFFFF << b) & 0xFFFFFFFF)
+    assert np.array_equal(C.view(np.uint32), v.view(np.uint32) & mask)
+    if b == 16:   # truncating 16 of the 23 fraction bits: relative error below 2^-7 on normal numbers
+        normal = np.abs(v) >= 2.0**-126
+        assert np.all(np.abs(v[normal].astype(np.float64) - C[normal]) < 2.0**-7 * np.abs(v[normal]))
+    # clipping what is already clipped changes nothing
+    C2, p2 = oracle.q_clip(C, b)
+    assert np.array_equal(C2.view(np.uint32), C.view(np.uint32)) and np.array_equal(p2["hi"], p["hi"])
+    # the residual is exact: Q[v] + (v - Q[v]) gives v back bit for bit
+    delta = oracle.residual(v, C)
+    assert np.array_equal(C.astype(np.float64) + delta.astype(np.float64), v.astype(np.float64))
+    assert np.array_equal(oracle.decode_clip(p["hi"], v.size, b).view(np.uint32), C.view(np.uint32))
+    # a contraction (Section 4 needs ||v - Q[v]|| <= alpha ||v|| with alpha < 1 on what it is applied to)
+    assert np.linalg.norm(delta.astype(np.float64)) < np.linalg.norm(v.astype(np.float64))
