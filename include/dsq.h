@@ -83,10 +83,16 @@ typedef enum {
  *                index or 0xFFFFFFFF on the server pass, step); entry uses output word
  *                offset_in_chunk%4, top 24 bits, as a uniform in [0,1).
  *
+ * DS_Q_CLIP      "Clipping" of Section 3.2: the low `levels` bits (16 or 24) of every binary32 number
+ *                are set to zero, which keeps the sign, the exponent and the leading fraction
+ *                bits (truncation toward zero); deterministic and biased.  The payload carries
+ *                the surviving high 32 - levels bits of every entry.  The residual v - Q[v] is
+ *                exact.
+ *
  * Chunk reductions (sum of |v| or of v*v) are pairwise sums in index order over the chunk padded
  * with zeros to `chunk` entries, so results do not depend on launch geometry.
  */
-typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3 } ds_op;
+typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3, DS_Q_CLIP = 4 } ds_op;
 
 /* ds_qspec.norm for DS_Q_SIGN1 */
 #define DS_NORM_L1 0u /* s_c = ||v_c||_1 / len_c (also selected by 1) */
@@ -96,7 +102,7 @@ typedef struct {
   int32_t op;        /* ds_op */
   uint32_t chunk;    /* SIGN1, QSGD: a power of two in [128, 8192]; else ignored */
   uint64_t k;        /* TOPK: 0 <= k <= d; else ignored */
-  uint32_t levels;   /* QSGD: 1 <= levels <= 255; else ignored */
+  uint32_t levels;   /* QSGD: 1 <= levels <= 255; CLIP: bits set to zero, 16 or 24; else ignored */
   uint32_t norm;     /* SIGN1: DS_NORM_L1 (0 or 1) or DS_NORM_L2 (2); else must be 0 */
 } ds_qspec;
 
@@ -147,6 +153,7 @@ typedef struct {
  *   QSGD      [0] uint8  lvl[d]            [1] uint32 sgn[ceil(d/32)] (bit = v >= 0)
  *             [2] float  step[ceil(d/chunk)] (the grid step q = N_c / levels that multiplies the
  *                 levels; 0 for a chunk sent as all zeros)
+ *   CLIP      [0] uint16 hi[d] (levels = 16) or uint8 hi[d] (levels = 24): bits(v) >> levels
  */
 typedef struct {
   uint64_t stride;

@@ -20,7 +20,7 @@ DS_ERR_INVALID_ARG, DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL = -1, -2, -3
 DS_ERR_STATE, DS_ERR_CUDA, DS_ERR_UNSUPPORTED = -4, -5, -6
 DS_FUSE_APPLY = 1
 DS_DEV_TOPK_INCONSISTENT = 1
-OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3}
+OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4}
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
            "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
            "ds_kernel_launches", "ds_topk_worker_static")
@@ -85,7 +85,7 @@ def load_library() -> C.CDLL:
 
 
 def _qspec(q: Q) -> ds_qspec:
-    return ds_qspec(OPS[q.op], q.chunk, q.k, q.levels, q.norm if q.op == "sign1" else 0)
+    return ds_qspec(OPS[q.op], q.chunk, q.k, q.bits if q.op == "clip" else q.levels, q.norm if q.op == "sign1" else 0)
 
 
 def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int) -> ds_config:
@@ -105,17 +105,21 @@ _VIEW_DTYPES = {
     "sign1": (("bits", torch.int32), ("scale", torch.float32)),
     "topk": (("idx", torch.int32), ("val", torch.float32)),
     "qsgd": (("lvl", torch.uint8), ("sgn", torch.int32), ("step", torch.float32)),
+    "clip": (("hi", torch.int16),),      # 8-bit entries when 24 bits are cleared, see payload_views
 }
 
 
-def payload_views(buf: torch.Tensor, layout: ds_payload_layout, op: str, rows: int) -> list[dict]:
+def payload_views(buf: torch.Tensor, layout: ds_payload_layout, q: Q, rows: int) -> list[dict]:
     """Typed views of the sub-arrays of each payload inside the raw byte buffer (no copies).
-    uint32 fields are exposed as int32 tensors with the same bits."""
+    uint32 / uint16 fields are exposed as int32 / int16 tensors with the same bits."""
     out = []
+    fields = _VIEW_DTYPES[q.op]
+    if q.op == "clip" and q.bits == 24:
+        fields = (("hi", torch.uint8),)
     for i in range(rows):
         base = i * layout.stride
         views = {}
-        for j, (name, dt) in enumerate(_VIEW_DTYPES[op]):
+        for j, (name, dt) in enumerate(fields):
             nbytes = layout.count[j] * torch.empty(0, dtype=dt).element_size()
             views[name] = buf[base + layout.off[j]: base + layout.off[j] + nbytes].view(dt)
         out.append(views)
@@ -218,10 +222,10 @@ class DoubleSqueeze:
 
     # -- views ----------------------------------------------------------------------------------
     def worker_views(self) -> list[dict]:
-        return payload_views(self.worker_payload, self.worker_layout, self.worker_q.op, self.n)
+        return payload_views(self.worker_payload, self.worker_layout, self.worker_q, self.n)
 
     def server_views(self) -> dict:
-        return payload_views(self.server_payload, self.server_layout, self.server_q.op, 1)[0]
+        return payload_views(self.server_payload, self.server_layout, self.server_q, 1)[0]
 
     def device_status(self) -> int:
         return int(self.dev_status[0].item())

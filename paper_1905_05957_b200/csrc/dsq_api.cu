@@ -34,6 +34,7 @@ bool qspec_ok(const ds_qspec& q, uint64_t d) {
     case DS_Q_SIGN1: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192;
     case DS_Q_QSGD: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192 && q.levels >= 1 && q.levels <= 255;
     case DS_Q_TOPK: return q.k <= d;
+    case DS_Q_CLIP: return q.levels == 16 || q.levels == 24;
     default: return false;
   }
 }
@@ -60,6 +61,7 @@ void layout_of(const ds_qspec& q, uint64_t d, ds_payload_layout* L) {
     case DS_Q_SIGN1: put(0, nw, 4); put(1, (d + q.chunk - 1) / q.chunk, 4); break;
     case DS_Q_TOPK: put(0, q.k, 4); put(1, q.k, 4); break;
     case DS_Q_QSGD: put(0, d, 1); put(1, nw, 4); put(2, (d + q.chunk - 1) / q.chunk, 4); break;
+    case DS_Q_CLIP: put(0, d, (32 - q.levels) / 8); break;
   }
   L->stride = pos ? pos : 16;
 }
@@ -139,12 +141,14 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
   for (int i = 0; i < 3; ++i) s.wp_off[i] = c->wl.off[i];
   s.w_log2_chunk = (wq.op == DS_Q_SIGN1 || wq.op == DS_Q_QSGD) ? log2u(wq.chunk) : 0;
   s.w_levels = (float)wq.levels;
+  s.w_clip_bits = wq.op == DS_Q_CLIP ? wq.levels : 0;
   s.acc = c->acc;
   s.vec = 1;
   switch (wq.op) {
     case DS_Q_IDENTITY: *kind = SRC_SRV_IDENTITY; break;
     case DS_Q_SIGN1: *kind = SRC_SRV_SIGN1; break;
     case DS_Q_TOPK: *kind = SRC_SRV_TOPK; break;
+    case DS_Q_CLIP: *kind = SRC_SRV_CLIP; break;
     default: *kind = SRC_SRV_QSGD; break;
   }
   return s;
@@ -201,6 +205,9 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       e = launch_topk(src_kind, src, server ? c->splan : c->wplan, c->buf.workspace, io, rows, q.k, st);
       break;
     }
+    case DS_Q_CLIP:
+      e = launch_clip(src_kind, src, q.levels, payload + L.off[0], L.stride, delta, d, x_fused, c->cfg.gamma, rows, st);
+      break;
     default: return DS_ERR_UNSUPPORTED;
   }
   return e == cudaSuccess ? DS_OK : cuda_fail(e, "kernel launch");
@@ -304,6 +311,7 @@ int ds_apply_update(ds_handle h, void* cuda_stream) {
   for (int i = 0; i < 3; ++i) pv.off[i] = h->sl.off[i];
   pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD) ? log2u(q.chunk) : 0;
   pv.levels_f = (float)q.levels;
+  pv.clip_bits = q.op == DS_Q_CLIP ? q.levels : 0;
   pv.k = q.k;
   const cudaError_t e = launch_apply(pv, h->buf.x, h->cfg.d, h->cfg.gamma, static_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return cuda_fail(e, "apply update");

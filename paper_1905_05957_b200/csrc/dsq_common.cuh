@@ -29,6 +29,7 @@ enum Src : int {
   SRC_SRV_SIGN1 = 2,
   SRC_SRV_TOPK = 3,      // the sparse payloads were summed into a dense accumulator beforehand
   SRC_SRV_QSGD = 4,
+  SRC_SRV_CLIP = 5,      // payload = the high bits of every entry
 };
 
 // Where v comes from.  Worker payload sub-arrays follow the documented payload layout.
@@ -43,6 +44,7 @@ struct SrcParams {
   uint64_t wp_off[3];      // sub-array offsets inside a payload
   uint32_t w_log2_chunk;   // worker chunk length (SIGN1, QSGD)
   float w_levels;          // worker QSGD level count as a float
+  uint32_t w_clip_bits;    // worker CLIP: low bits that were set to zero (16 or 24)
   const float* acc;        // SRC_SRV_TOPK: dense accumulator [d] holding the sum of the sparse payloads
   int vec;                 // 1 if every row starts 16-byte aligned (d % 4 == 0)
 };
@@ -206,6 +208,52 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
                 acc[j] = add4_rn(acc[j], make_float4(signed_by_bit(mag.x, ww, 0), signed_by_bit(mag.y, ww, 1),
                                                      signed_by_bit(mag.z, ww, 2), signed_by_bit(mag.w, ww, 3)));
               }
+            }
+          }
+        }
+      }
+    } else if constexpr (SRC == SRC_SRV_CLIP) {
+      // Q[v_i] = hi << bits; four workers' rows are fetched before they are added (in worker order)
+      const bool wide = p.w_clip_bits == 16;  // 16-bit entries, else 8-bit
+      for (uint32_t i0 = 0; i0 < p.n; i0 += 4) {
+        uint2 raw[V][4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint8_t* hp = p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[0];
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            raw[j][u] = make_uint2(0u, 0u);
+            if (i0 + u >= p.n || !cnt[j]) continue;
+            if (cnt[j] == 4) {
+              if (wide) raw[j][u] = __ldcs(reinterpret_cast<const uint2*>(hp + 2 * e[j]));
+              else raw[j][u].x = __ldcs(reinterpret_cast<const uint32_t*>(hp + e[j]));
+            } else {
+              // a ragged last row: entry by entry, packed as a full row would be
+              uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                if ((uint32_t)k < cnt[j])
+                  w[k] = wide ? (uint32_t)__ldcs(reinterpret_cast<const uint16_t*>(hp + 2 * e[j]) + k) : (uint32_t)__ldcs(hp + e[j] + k);
+              raw[j][u] = wide ? make_uint2(w[0] | w[1] << 16, w[2] | w[3] << 16)
+                               : make_uint2(w[0] | w[1] << 8 | w[2] << 16 | w[3] << 24, 0u);
+            }
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (i0 + u < p.n) {
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+              const uint2 r = raw[j][u];
+              float4 c;
+              if (wide) {
+                c = make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u),
+                                __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xFFFF0000u));
+              } else {
+                c = make_float4(__uint_as_float(r.x << 24), __uint_as_float((r.x << 16) & 0xFF000000u),
+                                __uint_as_float((r.x << 8) & 0xFF000000u), __uint_as_float(r.x & 0xFF000000u));
+              }
+              acc[j] = add4_rn(acc[j], c);
             }
           }
         }

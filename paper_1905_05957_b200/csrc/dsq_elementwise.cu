@@ -50,11 +50,88 @@ cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64
     case SRC_SRV_SIGN1: DSQ_ID(SRC_SRV_SIGN1); break;
     case SRC_SRV_TOPK: DSQ_ID(SRC_SRV_TOPK); break;
     case SRC_SRV_QSGD: DSQ_ID(SRC_SRV_QSGD); break;
+    case SRC_SRV_CLIP: DSQ_ID(SRC_SRV_CLIP); break;
     default: return cudaErrorInvalidValue;
   }
 #undef DSQ_ID
   count_launches(1);
   return cudaGetLastError();
+}
+
+// Q = clipping (Section 3.2): the low BITS bits of every number are set to zero; the payload is what
+// is left, bits(v) >> BITS, as 16- or 8-bit entries.  The residual v - Q[v] is exact.
+template <int SRC, int BITS>
+__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : kServerCtasPerSm)
+k_clip(const SrcParams src, uint8_t* out_hi, uint64_t hi_row_stride, float* delta_out, uint64_t delta_row_stride, float* x,
+       float gamma) {
+  pdl_prologue();
+  constexpr uint32_t kMask = 0xFFFFFFFFu << BITS;
+  const uint32_t row = blockIdx.y;
+  const uint64_t nq = (src.d + 3) / 4;
+  uint8_t* hi = out_hi + (uint64_t)row * hi_row_stride;
+  // the loop bound is the same for all threads of the CTA: the source is read warp-cooperatively
+  for (uint64_t q0 = (uint64_t)blockIdx.x * kThreads; q0 < nq; q0 += (uint64_t)gridDim.x * kThreads) {
+    const uint64_t ee[1] = {(q0 + threadIdx.x) * 4};
+    const uint64_t e = ee[0];
+    const uint32_t cc[1] = {e < src.d ? (uint32_t)min((uint64_t)4, src.d - e) : 0u};
+    const uint32_t cnt = cc[0];
+    float4 vv[1];
+    src_load_tile<SRC, 1>(src, row, ee, cc, vv);
+    const float4 v = vv[0];
+    if (!cnt) continue;
+    const uint32_t u0 = __float_as_uint(v.x), u1 = __float_as_uint(v.y), u2 = __float_as_uint(v.z), u3 = __float_as_uint(v.w);
+    const float4 C = make_float4(__uint_as_float(u0 & kMask), __uint_as_float(u1 & kMask), __uint_as_float(u2 & kMask),
+                                 __uint_as_float(u3 & kMask));
+    if (cnt == 4) {
+      if (BITS == 16) {
+        __stcs(reinterpret_cast<uint2*>(hi + 2 * e), make_uint2(u0 >> 16 | (u1 & kMask), u2 >> 16 | (u3 & kMask)));
+      } else {
+        __stcs(reinterpret_cast<uint32_t*>(hi + e), u0 >> 24 | (u1 >> 24) << 8 | (u2 >> 24) << 16 | (u3 & kMask));
+      }
+    } else {
+      const uint32_t us[4] = {u0, u1, u2, u3};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if ((uint32_t)k < cnt) {
+          if (BITS == 16) reinterpret_cast<uint16_t*>(hi + 2 * e)[k] = (uint16_t)(us[k] >> 16);
+          else hi[e + k] = (uint8_t)(us[k] >> 24);
+        }
+      }
+    }
+    store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
+    if (x) {
+      float4 xv = load_row4(x, e, cnt, 1);
+      xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
+      xv.z = __fsub_rn(xv.z, __fmul_rn(gamma, C.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(gamma, C.w));
+      store_row4(x, e, cnt, 1, xv);
+    }
+  }
+}
+
+template <int BITS>
+static cudaError_t launch_clip_bits(int srck, const SrcParams& src, uint8_t* out_hi, uint64_t hi_row_stride, float* delta_out,
+                                    uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st) {
+  dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
+#define DSQ_CL(S) launch_pdl(k_clip<S, BITS>, grid, kThreads, st, src, out_hi, hi_row_stride, delta_out, delta_row_stride, x, gamma)
+  switch (srck) {
+    case SRC_WORKER: DSQ_CL(SRC_WORKER); break;
+    case SRC_SRV_IDENTITY: DSQ_CL(SRC_SRV_IDENTITY); break;
+    case SRC_SRV_SIGN1: DSQ_CL(SRC_SRV_SIGN1); break;
+    case SRC_SRV_TOPK: DSQ_CL(SRC_SRV_TOPK); break;
+    case SRC_SRV_QSGD: DSQ_CL(SRC_SRV_QSGD); break;
+    case SRC_SRV_CLIP: DSQ_CL(SRC_SRV_CLIP); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef DSQ_CL
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_clip(int srck, const SrcParams& src, uint32_t bits, uint8_t* out_hi, uint64_t hi_row_stride,
+                        float* delta_out, uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st) {
+  if (bits == 16) return launch_clip_bits<16>(srck, src, out_hi, hi_row_stride, delta_out, delta_row_stride, x, gamma, rows, st);
+  if (bits == 24) return launch_clip_bits<24>(srck, src, out_hi, hi_row_stride, delta_out, delta_row_stride, x, gamma, rows, st);
+  return cudaErrorInvalidValue;
 }
 
 // Dense decode of a server payload and update of x.
@@ -71,6 +148,14 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, 
       const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]) + (e >> 5)) >> (uint32_t)(e & 31);
       const float s = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
       C = make_float4(signed_by_bit(s, w, 0), signed_by_bit(s, w, 1), signed_by_bit(s, w, 2), signed_by_bit(s, w, 3));
+    } else if (pv.op == DS_Q_CLIP) {
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if ((uint32_t)k < cnt)
+          w[k] = pv.clip_bits == 16 ? (uint32_t)__ldcs(reinterpret_cast<const uint16_t*>(pv.base + pv.off[0]) + e + k) << 16
+                                    : (uint32_t)__ldcs(pv.base + pv.off[0] + e + k) << 24;
+      C = make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]), __uint_as_float(w[2]), __uint_as_float(w[3]));
     } else {  // DS_Q_QSGD
       const uint32_t lv = __ldcs(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0] + e));
       const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[1]) + (e >> 5)) >> (uint32_t)(e & 31);

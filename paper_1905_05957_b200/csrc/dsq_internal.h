@@ -55,6 +55,7 @@ struct PayloadView {
   uint64_t off[3];
   uint32_t log2_chunk;
   float levels_f;
+  uint32_t clip_bits;
   uint64_t k;
 };
 
@@ -109,6 +110,10 @@ cudaError_t launch_chunked(int op, int src_kind, const SrcParams& src, const Chu
 // Q = identity: payload c = v, residual +0, optional fused update.
 cudaError_t launch_identity(int src_kind, const SrcParams& src, float* out_c, uint64_t c_row_stride, float* delta_out,
                             uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);
+
+// Q = clipping: payload hi = bits(v) >> bits (16- or 8-bit entries), residual v - Q[v], optional fused update.
+cudaError_t launch_clip(int src_kind, const SrcParams& src, uint32_t bits, uint8_t* out_hi, uint64_t hi_row_stride,
+                        float* delta_out, uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);
 
 // x = x - gamma * decode(payload)
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);

@@ -1227,6 +1227,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
       case SRC_SRV_SIGN1: DSQ_P1(SRC_SRV_SIGN1); break;
       case SRC_SRV_TOPK: DSQ_P1(SRC_SRV_TOPK); break;
       case SRC_SRV_QSGD: DSQ_P1(SRC_SRV_QSGD); break;
+      case SRC_SRV_CLIP: DSQ_P1(SRC_SRV_CLIP); break;
       default: return cudaErrorInvalidValue;
     }
 #undef DSQ_P1
@@ -1261,6 +1262,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
       case SRC_SRV_SIGN1: DSQ_P1(SRC_SRV_SIGN1); break;
       case SRC_SRV_TOPK: DSQ_P1(SRC_SRV_TOPK); break;
       case SRC_SRV_QSGD: DSQ_P1(SRC_SRV_QSGD); break;
+      case SRC_SRV_CLIP: DSQ_P1(SRC_SRV_CLIP); break;
       default: return cudaErrorInvalidValue;
     }
 #undef DSQ_P1

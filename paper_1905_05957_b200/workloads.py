@@ -38,11 +38,12 @@ assert len(RESNET18_SLICES) == 62 and sum(RESNET18_SLICES) == 11_689_512
 
 @dataclass(frozen=True)
 class Q:
-    op: str = "identity"     # identity | sign1 | topk | qsgd
+    op: str = "identity"     # identity | sign1 | topk | qsgd | clip
     chunk: int = 0
     k: int = 0
     levels: int = 0
     norm: int = 1            # sign1: scale from l1 (1) or l2 (2) magnitudes
+    bits: int = 0            # clip: low bits of every number set to zero (16 or 24)
 
 
 @dataclass(frozen=True)
@@ -82,6 +83,8 @@ def _wl() -> dict[int, Workload]:
         # from l2 magnitudes (the norm Section 3.2 prints)
         6: Workload(6, "sign1l2_n8_resnet18", 8, 11_689_512, 20, "layered",
                     Q("sign1", chunk=4096, norm=2), Q("sign1", chunk=4096, norm=2)),
+        # ... and with clipping of the low 16 bits (Section 3.2) on both passes
+        7: Workload(7, "clip16_n8_resnet18", 8, 11_689_512, 20, "layered", Q("clip", bits=16), Q("clip", bits=16)),
     }
 
 

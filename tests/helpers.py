@@ -10,12 +10,14 @@ REL_TOL = 1e-5   # bar for fp32 values, scales and delta (reduction order may di
 
 
 def to_oracle_q(q: Q) -> oracle.QSpec:
-    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels, norm=q.norm)
+    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels, norm=q.norm, bits=q.bits)
 
 
 def u32(t) -> np.ndarray:
     """Device int32/uint8 tensor -> host array with unsigned bits."""
     a = t.detach().cpu().numpy()
+    if a.dtype == np.int16:
+        return a.view(np.uint16)
     return a.view(np.uint32) if a.dtype == np.int32 else a
 
 
@@ -54,6 +56,8 @@ def compare_payload(name: str, op: str, gpu_views: dict, ora: dict):
         assert_bits_match(f"{name}.lvl", u32(gpu_views["lvl"]), ora["lvl"])
         assert_bits_match(f"{name}.sgn", u32(gpu_views["sgn"]), ora["sgn"])
         assert_float_match(f"{name}.step", gpu_views["step"].cpu().numpy(), ora["step"])
+    elif op == "clip":
+        assert_bits_match(f"{name}.hi", u32(gpu_views["hi"]), ora["hi"])
     else:
         raise ValueError(op)
 

@@ -14,6 +14,7 @@ SIGN_L2 = lambda L=4096: Q("sign1", chunk=L, norm=2)
 QSGD = lambda L=2048, s=255: Q("qsgd", chunk=L, levels=s)
 TOPK = lambda k: Q("topk", k=k)
 IDENT = Q("identity")
+CLIP = lambda b=16: Q("clip", bits=b)
 
 
 def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None, scribble=False):
@@ -78,6 +79,23 @@ def test_topk_both_passes(d, k):
     run_lockstep(3, d, TOPK(k), TOPK(k), randn_steps(3, d, 3, seed=d + k))
 
 
+@pytest.mark.parametrize("d", [4096, 10_000, 65_536 + 4 * 37, 33, 5, 1])
+@pytest.mark.parametrize("b", [16, 24])
+def test_clip_both_passes(d, b):
+    run_lockstep(3, d, CLIP(b), CLIP(b), randn_steps(3, d, 3, seed=d + b))
+
+
+def test_clip_mixed_with_other_operators_unaligned_rows_and_unfused_update():
+    d = 50_000 + 13
+    for wq, sq in [(CLIP(16), TOPK(500)), (CLIP(24), SIGN(2048)), (QSGD(1024, 31), CLIP(16)), (TOPK(700), CLIP(24)),
+                   (CLIP(16), QSGD(2048)), (SIGN(4096), CLIP(16)), (IDENT, CLIP(16)), (CLIP(16), IDENT),
+                   (CLIP(16), SIGN_L2(1024))]:
+        run_lockstep(5, d, wq, sq, randn_steps(5, d, 2, seed=43))
+    run_lockstep(3, 30_000, CLIP(16), CLIP(16), randn_steps(3, 30_000, 3, seed=44), fuse=False)
+    run_lockstep(3, 30_001, CLIP(24), CLIP(24), randn_steps(3, 30_001, 2, seed=45), fuse=False)
+    run_lockstep(37, 9000, CLIP(16), CLIP(16), randn_steps(37, 9000, 2, seed=46))
+
+
 def test_identity_is_parallel_sgd():
     run_lockstep(4, 10_001, IDENT, IDENT, randn_steps(4, 10_001, 3))
 
@@ -132,7 +150,7 @@ def test_zero_signed_zero_subnormal_and_zero_chunks():
     g[:, 5000:5100] = 1e-41      # subnormals
     g[:, 5100:5200] = -1e-41
     g[0, 8192:] = 1e-30          # squares underflow: a quantisation chunk of norm ~0
-    for wq in (SIGN(4096), QSGD(2048), TOPK(100), SIGN(128), QSGD(128, 5), SIGN_L2(4096), SIGN_L2(128)):
+    for wq in (SIGN(4096), QSGD(2048), TOPK(100), SIGN(128), QSGD(128, 5), SIGN_L2(4096), SIGN_L2(128), CLIP(16), CLIP(24)):
         run_lockstep(n, d, wq, wq, [g, g.clone(), -g])
 
 
@@ -169,7 +187,7 @@ def test_many_workers_and_one_worker():
 
 # ------------------------------------------------------------------ the five workloads, scaled down
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7])
 def test_workload_recipes_scaled(wid):
     wl = WORKLOADS[wid]
     wl = wl if wid == 1 else wl.scaled(d=200_000 + 40, n=min(wl.n, 8), steps=4)
