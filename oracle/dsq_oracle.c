@@ -213,9 +213,9 @@ int orc_decode_sign1(const uint32_t* bits, const float* scale, uint64_t d, uint3
 }
 
 /* ------------------------------------------------------------------------ */
-/* Q = clipping (Section 3.2 "Clipping": set the lower bits of every number  */
-/* to zero; deterministic and biased).  Reading: the number is its binary32  */
-/* representation and its low b bits are cleared, which keeps the sign, the  */
+/* Q = clipping (the "Clipping" option of Section 3.2: the low-order bits of  */
+/* every number are dropped; deterministic, biased).  Reading: the number is */
+/* its binary32 word and its low b bits are cleared, which keeps the sign,   */
 /* exponent and the leading 23 - b fraction bits (b <= 23), i.e. truncates   */
 /* the magnitude toward zero.  What is sent per entry is the surviving high  */
 /* 32 - b bits; b is 16 or 24 so that an entry is a 16- or an 8-bit word.    */

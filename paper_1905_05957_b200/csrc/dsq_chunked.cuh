@@ -276,7 +276,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
 }
 
 template <int OP, int SRC, int V, int LOG2G>
-__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : kServerCtasPerSm) k_chunked(const SrcParams src, const ChunkParams p) {
+__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : (V >= 8 ? 2 : kServerCtasPerSm)) k_chunked(const SrcParams src, const ChunkParams p) {
   pdl_prologue();
   __shared__ float s_red[64];
   __shared__ float s_scal[16];

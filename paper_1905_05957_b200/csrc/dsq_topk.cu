@@ -9,20 +9,25 @@
 // Pipeline with a candidate list (the library's normal path):
 //   pass1      v = source (Eq. 2 / Eq. 4), written over delta.  With the thresholds of the two
 //              previous steps it predicts a band of keys [lo, hi] around this step's threshold and,
-//              while v is still in registers, (a) sets a bit in the "kept" bitmap for every entry
-//              above the band and counts them, (b) writes (key, index) of every entry inside the
-//              band to the candidate list.  The list has one fixed region per 4096-entry tile
-//              (as many slots as the tile has entries), so no reservation between CTAs is needed.
-//   lhist 1    copies the tile regions into one dense list and counts the top 12 key bits on the
-//              way; accepts the prediction only if the k-th entry falls inside the list
-//              (kept < k <= kept + candidates)
-//   hist, pick only after a miss (or without history): full 4096-bin histogram of v, exact bin tb
-//   mark, compact  only after a miss: re-read v, rebuild bitmap and candidate list for the exact tb
-//   lhist 2,3  the next 12, then the last 7 key bits from the candidate list: tau and r
-//   classify   candidates with key > tau join the kept bitmap, key == tau go to the tie bitmap
-//   count, scan  per-segment population counts and their exclusive prefix
-//   emit       every set bit knows its output slot: write (index, value), zero the entry in delta
-//              (delta = v - Q[v], Eq. 3), and on a fused server pass update x at that entry
+//              while v is still in registers, writes (value bits, index) of every entry with
+//              key >= lo into the tile's own region of the list, in index order (one region of
+//              4096 slots per 4096-entry tile, so CTAs never reserve space from each other).
+//              Entries above the band (key > hi) are kept whatever tau turns out to be: they are
+//              counted and already zeroed in the residual.  tile_info = (listed, above, 0, 0).
+//   lhist 1    copies the entries inside the band (the candidates) out of the regions into one
+//              dense (key, index) list and counts the top 12 key bits on the way; accepts the
+//              prediction only if the k-th entry is a candidate (above < k <= above + candidates)
+//   hist, pick only after a miss (or without history): entries zeroed by pass1 are restored from
+//              the regions, then a full 4096-bin histogram of v gives the exact bin tb
+//   mark, compact  only after a miss: re-read v, rebuild regions and dense list for the exact bin
+//   lhist 2,3  the next 12, then the last 7 key bits from the dense list: tau and r
+//   classify   every candidate with key >= tau adds one to its tile's counters in tile_info
+//              (.z: above tau, .w: equal to tau)
+//   scan       exclusive prefix over the tiles of (above the band + above tau, ties); checks that
+//              exactly k entries will be emitted
+//   emit       a warp per tile walks the region in index order; the prefix gives the tile's first
+//              output slot, ballots place the kept entries: write (index, value), zero the kept
+//              candidates in delta (delta = v - Q[v], Eq. 3), and on a fused server pass update x
 // In the steady state v is read once and written once; the kernels marked "only after a miss"
 // leave at once.  A wrong, missing or garbage history costs time, never correctness.
 //
@@ -31,7 +36,7 @@
 //   (candidates gathered through their bitmap) -> finalize -> scan -> emit.
 //
 // No float atomics, no spinning; integer atomics commute and output slots come from prefix sums
-// over index-ordered bitmaps, so the result does not depend on scheduling.
+// over index-ordered regions or bitmaps, so the result does not depend on scheduling.
 #include "dsq_common.cuh"
 #include "dsq_internal.h"
 

@@ -51,6 +51,14 @@ def test_layouts(lib):
     assert b.get_layout(cfg, 1).count[0] == 1000
     cfg = b.make_config(2, 1000, 0.1, Q("topk", k=0), Q("topk", k=0), 1)
     assert b.get_layout(cfg, 0).stride == 16     # never a zero stride
+    cfg = b.make_config(2, 1001, 0.1, Q("clip", bits=16), Q("clip", bits=24), 1)
+    c16, c24 = b.get_layout(cfg, 0), b.get_layout(cfg, 1)
+    assert c16.count[0] == 1001 and c16.stride == (2 * 1001 + 15) // 16 * 16
+    assert c24.count[0] == 1001 and c24.stride == (1001 + 15) // 16 * 16
+    # the l2-magnitude variant of the 1-bit operator shares the payload format
+    a = b.get_layout(b.make_config(2, 5000, 0.1, Q("sign1", chunk=128), Q("identity"), 1), 0)
+    l2 = b.get_layout(b.make_config(2, 5000, 0.1, Q("sign1", chunk=128, norm=2), Q("identity"), 1), 0)
+    assert (a.stride, list(a.off), list(a.count)) == (l2.stride, list(l2.off), list(l2.count))
 
 
 def test_query_mode_reports_sizes(lib):
@@ -70,6 +78,8 @@ def test_query_mode_reports_sizes(lib):
     dict(worker_q=Q("sign1", chunk=1000)), dict(worker_q=Q("sign1", chunk=64)), dict(worker_q=Q("sign1", chunk=16384)),
     dict(server_q=Q("qsgd", chunk=2048, levels=0)), dict(server_q=Q("qsgd", chunk=2048, levels=256)),
     dict(worker_q=Q("topk", k=1001)),
+    dict(worker_q=Q("sign1", chunk=4096, norm=3)), dict(server_q=Q("clip", bits=12)), dict(server_q=Q("clip", bits=0)),
+    dict(worker_q=Q("clip", bits=32)),
 ])
 def test_bad_configs_are_rejected(lib, kw):
     args = dict(n=4, d=1000, gamma=0.1, worker_q=Q("identity"), server_q=Q("identity"), seed=0)

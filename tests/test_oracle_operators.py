@@ -248,8 +248,8 @@ def test_qsgd_levels_bracket_the_value_and_decode_roundtrip():
 # ------------------------------------------------------------------ clipping
 
 def test_clip_worked_binary_cases():
-    """Section 3.2 "Clipping" clears low bits of the number (its example drops low decimal digits of
-    1.23456); for binary32 with b = 16 the sign, the exponent and 7 fraction bits survive."""
+    """The clipping option of Section 3.2 drops low-order bits of a number (its example drops decimal
+    digits); for binary32 with b = 16 the sign, the exponent and 7 fraction bits survive."""
     one = np.float32(1.0)
     cases16 = [
         (1.0, 1.0), (-2.0, -2.0), (1.5, 1.5), (0.0, 0.0),
