@@ -32,7 +32,11 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised under profiles/; valid only for the kernel sources with this digest.
 NCU_TRAFFIC = {
     # workload id: (kernel, bytes per launch, digest of the kernel's source files at capture time)
-    2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748234752 + 335448320, "cb37fb5109354746"),
+    2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748169472 + 331292672, "931e964813c046c9"),
+    # captured on the same recipe at d = 2^24 (a multi-pass capture must stay small) and scaled by
+    # the entries one launch processes: traffic of a streaming kernel grows in proportion
+    4: ("k_chunked<QSGD, WORKER, 2, 256>", int((1073976000 + 630305536) * (8 * 124_439_808) / (8 * 16_777_216)), "931e964813c046c9"),
+    7: ("k_clip<WORKER, 16>", 748320000 + 508970496, "74295ad39f94bb79"),
 }
 KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "sign1": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
@@ -244,7 +248,10 @@ def run_ours(args, wl):
     barrier()
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
+        t_wait = time.time() + 3.0
+        while not sampler.lines and time.time() < t_wait:   # the first answer takes a moment
+            time.sleep(0.05)
+        sampler.lines.clear()                               # samples of the idle GPU are dropped
     launches0 = lib.ds_kernel_launches()
     t_total = 0.0
     barrier()
@@ -263,7 +270,19 @@ def run_ours(args, wl):
         stop.record(stream)
     barrier()
     launches = lib.ds_kernel_launches() - launches0
+    # nvidia-smi answers every 100 ms and a short timed region may end before its first answer: keep
+    # the same steps running, untimed, until a few samples under this load are in
+    t_end = time.time() + 1.2
+    extra = 0
+    while time.time() < t_end and (rank != 0 or len(sampler.lines) < 8):
+        ds.step(ring[extra % R], W + K + extra)
+        extra += 1
+        if extra % 16 == 0:
+            torch.cuda.synchronize(dev)
+    torch.cuda.synchronize(dev)
     clocks = sampler.stop() if rank == 0 else None
+    if clocks is not None:
+        clocks["sampled"] = "during the timed steps and the same steps repeated untimed right after them"
     worker_ms = [ev[t][0].elapsed_time(ev[t][1]) for t in range(K)]
     server_ms = [ev[t][1].elapsed_time(ev[t][2]) for t in range(K)]
     step_ms = [ev[t][0].elapsed_time(ev[t][2]) for t in range(K)]
