@@ -262,3 +262,35 @@ def test_more_workers_than_one_batch_of_the_server_loops():
     # 150 sparse payloads (the ordered sum walks them in batches of 128) and 150 one-bit payloads
     run_lockstep(150, 9000, TOPK(90), TOPK(90), randn_steps(150, 9000, 2, seed=31))
     run_lockstep(150, 4096 + 100, SIGN(1024), QSGD(512, 63), randn_steps(150, 4096 + 100, 2, seed=32))
+
+
+# ------------------------------------------------------------------ seeded random configurations
+
+def _random_q(r, d):
+    kind = r.choice(["sign1", "sign1_l2", "qsgd", "topk", "clip", "identity"])
+    if kind == "sign1":
+        return SIGN(int(r.choice([128, 256, 512, 1024, 2048, 4096, 8192])))
+    if kind == "sign1_l2":
+        return SIGN_L2(int(r.choice([128, 512, 2048, 4096])))
+    if kind == "qsgd":
+        return QSGD(int(r.choice([128, 256, 1024, 2048, 4096])), int(r.choice([1, 2, 7, 100, 255])))
+    if kind == "topk":
+        return TOPK(int(r.integers(0, max(1, d // 20) + 1)))
+    if kind == "clip":
+        return CLIP(int(r.choice([16, 24])))
+    return IDENT
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_configurations(case):
+    """Operator pair, sizes, scale of the data and the form of the update all drawn from the case number."""
+    r = np.random.default_rng(1905 + case)
+    n = int(r.integers(1, 10))
+    d = int(r.choice([r.integers(1, 200), r.integers(200, 20_000), r.integers(20_000, 150_000)]))
+    if r.random() < 0.5:
+        d = max(4, d // 4 * 4)
+    wq, sq = _random_q(r, d), _random_q(r, d)
+    scale = float(10.0 ** r.uniform(-4, 2))
+    gs = randn_steps(n, d, 3, seed=case, scale=scale)
+    run_lockstep(n, d, wq, sq, gs, gamma=float(r.choice([0.1, 0.01, 1.0])), seed=int(r.integers(0, 2**62)),
+                 fuse=bool(r.random() < 0.5))
