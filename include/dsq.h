@@ -198,6 +198,35 @@ int ds_apply_update(ds_handle h, void* cuda_stream);
 int ds_destroy(ds_handle h);
 
 /*
+ * The same two passes for a deployment in which every GPU is one worker and owns one slice of the
+ * server (Section 3.1 notes that the method is not tied to a single parameter server): each
+ * rank runs the worker pass for its own rows, receives the other workers' payload slices into its
+ * worker_payload buffer, runs the server pass over its slice of d, and applies the update from the
+ * server payload slices it gathered.  Moving the slices between GPUs is the caller's business.
+ *
+ * ds_worker_compress_rows: Algorithm 1, "On worker", for workers row0 .. row0+nrows-1 only; g holds
+ *   those nrows rows ([nrows, d] device memory).  delta_w and worker_payload keep their [n, ...]
+ *   layout; only the named rows are read and written.  Randomised operators draw with the global
+ *   worker index, so the result equals what ds_worker_compress gives for these rows.
+ * ds_server_aggregate_compress_slice: Algorithm 1, "On parameter server" (Eq. 4), for the entries
+ *   lo .. hi-1 of every vector: decodes that slice of all n worker payloads, writes that slice of
+ *   delta_s and of the server payload and, with DS_FUSE_APPLY, of x.  lo must be a multiple of
+ *   DS_SLICE_ALIGN, hi a multiple of it or d.  The union of disjoint slices covering [0, d) equals
+ *   one ds_server_aggregate_compress bit for bit.
+ * ds_apply_update_slice: x = x - gamma Q[v] on lo .. hi-1 from that slice of the server payload.
+ *
+ * Operators that act per chunk or per entry (IDENTITY, SIGN1, QSGD, CLIP) are supported on both
+ * passes; a global TOPK on either pass is DS_ERR_UNSUPPORTED here (its threshold is a property of
+ * the whole vector).  These calls do not take part in the worker -> server -> apply order check
+ * of the whole-vector calls: the caller sequences its slices.  Errors as for the whole-vector calls.
+ */
+#define DS_SLICE_ALIGN 8192u
+int ds_worker_compress_rows(ds_handle h, const float* g, uint32_t row0, uint32_t nrows, uint32_t step, void* cuda_stream);
+int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flags, uint64_t lo, uint64_t hi,
+                                       void* cuda_stream);
+int ds_apply_update_slice(ds_handle h, uint64_t lo, uint64_t hi, void* cuda_stream);
+
+/*
  * Convenience for callers that hold data in HOST memory: copies g_host (float[n*d], ideally
  * pinned) into the caller's device staging buffer g_dev, runs worker + server(+fused apply), and
  * copies the server payload and/or x back to host if the respective pointer is non-NULL.  All

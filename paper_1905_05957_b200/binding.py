@@ -23,7 +23,9 @@ DS_DEV_TOPK_INCONSISTENT = 1
 OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4}
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
            "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
-           "ds_kernel_launches", "ds_topk_worker_static")
+           "ds_kernel_launches", "ds_topk_worker_static", "ds_worker_compress_rows",
+           "ds_server_aggregate_compress_slice", "ds_apply_update_slice")
+DS_SLICE_ALIGN = 8192
 
 
 class ds_qspec(C.Structure):
@@ -76,6 +78,9 @@ def load_library() -> C.CDLL:
     L.ds_destroy.argtypes = [vp]
     L.ds_step_host.argtypes = [vp, vp, vp, u32, vp, vp, vp]
     L.ds_topk_worker_static.argtypes = [vp, vp, C.c_uint64, C.c_uint64, vp, vp, vp, vp]
+    L.ds_worker_compress_rows.argtypes = [vp, vp, u32, u32, u32, vp]
+    L.ds_server_aggregate_compress_slice.argtypes = [vp, u32, u32, C.c_uint64, C.c_uint64, vp]
+    L.ds_apply_update_slice.argtypes = [vp, C.c_uint64, C.c_uint64, vp]
     for name in EXPORTS:
         getattr(L, name).restype = C.c_int
     L.ds_last_error.restype = C.c_char_p
@@ -204,6 +209,19 @@ class DoubleSqueeze:
 
     def apply_update(self, stream=None):
         self._check(self.lib.ds_apply_update(self.handle, self._stream(stream)), "ds_apply_update")
+
+    # -- the same passes over some of the workers / a slice of d (one GPU per worker deployments) ---
+    def worker_compress_rows(self, g_rows: torch.Tensor, row0: int, step: int, stream=None):
+        assert g_rows.is_cuda and g_rows.dtype == torch.float32 and g_rows.is_contiguous() and g_rows.numel() % self.d == 0
+        self._check(self.lib.ds_worker_compress_rows(self.handle, g_rows.data_ptr(), row0, g_rows.numel() // self.d, step,
+                                                     self._stream(stream)), "ds_worker_compress_rows")
+
+    def server_aggregate_compress_slice(self, step: int, lo: int, hi: int, fuse_apply: bool = False, stream=None):
+        self._check(self.lib.ds_server_aggregate_compress_slice(self.handle, step, DS_FUSE_APPLY if fuse_apply else 0, lo, hi,
+                                                                self._stream(stream)), "ds_server_aggregate_compress_slice")
+
+    def apply_update_slice(self, lo: int, hi: int, stream=None):
+        self._check(self.lib.ds_apply_update_slice(self.handle, lo, hi, self._stream(stream)), "ds_apply_update_slice")
 
     def step(self, g: torch.Tensor, t: int, fuse_apply: bool = True, stream=None):
         self.worker_compress(g, t, stream)

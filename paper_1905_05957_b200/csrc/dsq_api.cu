@@ -155,33 +155,46 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
 }
 
 // One compression pass over `rows` vectors: rows = n with the worker source, 1 with a server source.
+// Where a pass sits inside the whole problem: d_pass entries per vector starting at entry lo of every
+// row, first worker row0.  The whole-vector calls use {cfg.d, 0, 0}.
+struct PassWindow {
+  uint64_t d_pass, lo;
+  uint32_t row0;
+};
+
 int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, const ds_payload_layout& L,
              uint8_t* payload, float* delta, uint32_t rows, bool server, float* x_fused, uint32_t step,
-             cudaStream_t st) {
-  const uint64_t d = c->cfg.d;
+             cudaStream_t st, const PassWindow* win = nullptr) {
+  // a slice pass sees vectors of d_pass entries; pointers arrive already shifted to the slice, and
+  // rows stay cfg.d entries apart
+  const uint64_t d = win ? win->d_pass : c->cfg.d;
+  const uint64_t row_stride = c->cfg.d;
+  const uint64_t lo = win ? win->lo : 0;
   cudaError_t e = cudaSuccess;
   switch (q.op) {
     case DS_Q_IDENTITY:
-      e = launch_identity(src_kind, src, reinterpret_cast<float*>(payload + L.off[0]), L.stride / 4, delta, d, x_fused,
-                          c->cfg.gamma, rows, st);
+      e = launch_identity(src_kind, src, reinterpret_cast<float*>(payload + L.off[0]) + lo, L.stride / 4, delta, row_stride,
+                          x_fused, c->cfg.gamma, rows, st);
       break;
     case DS_Q_SIGN1:
     case DS_Q_QSGD: {
       ChunkParams p;
       memset(&p, 0, sizeof p);
       if (q.op == DS_Q_SIGN1) {
-        p.out_bits = reinterpret_cast<uint32_t*>(payload + L.off[0]);
-        p.out_scale = reinterpret_cast<float*>(payload + L.off[1]);
+        p.out_bits = reinterpret_cast<uint32_t*>(payload + L.off[0]) + lo / 32;
+        p.out_scale = reinterpret_cast<float*>(payload + L.off[1]) + lo / q.chunk;
       } else {
-        p.out_lvl = payload + L.off[0];
-        p.out_bits = reinterpret_cast<uint32_t*>(payload + L.off[1]);
-        p.out_scale = reinterpret_cast<float*>(payload + L.off[2]);
+        p.out_lvl = payload + L.off[0] + lo;
+        p.out_bits = reinterpret_cast<uint32_t*>(payload + L.off[1]) + lo / 32;
+        p.out_scale = reinterpret_cast<float*>(payload + L.off[2]) + lo / q.chunk;
       }
+      p.chunk0 = (uint32_t)(lo / q.chunk);
+      p.row0 = win ? win->row0 : 0;
       p.bits_stride = L.stride / 4;
       p.scale_stride = L.stride / 4;
       p.lvl_stride = L.stride;
       p.delta_out = delta;
-      p.delta_row_stride = d;
+      p.delta_row_stride = row_stride;
       p.x = x_fused;
       p.gamma = c->cfg.gamma;
       p.levels_f = (float)q.levels;
@@ -194,6 +207,7 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       break;
     }
     case DS_Q_TOPK: {
+      if (win) return DS_ERR_UNSUPPORTED;
       TopkIO io;
       io.idx = reinterpret_cast<uint32_t*>(payload + L.off[0]);
       io.val = reinterpret_cast<float*>(payload + L.off[1]);
@@ -206,7 +220,8 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       break;
     }
     case DS_Q_CLIP:
-      e = launch_clip(src_kind, src, q.levels, payload + L.off[0], L.stride, delta, d, x_fused, c->cfg.gamma, rows, st);
+      e = launch_clip(src_kind, src, q.levels, payload + L.off[0] + lo * ((32 - q.levels) / 8), L.stride, delta, row_stride,
+                      x_fused, c->cfg.gamma, rows, st);
       break;
     default: return DS_ERR_UNSUPPORTED;
   }
@@ -317,6 +332,77 @@ int ds_apply_update(ds_handle h, void* cuda_stream) {
   if (e != cudaSuccess) return cuda_fail(e, "apply update");
   h->phase = 0;
   return DS_OK;
+}
+
+namespace {
+
+bool slice_ok(const ds_ctx* h, uint64_t lo, uint64_t hi) {
+  const uint64_t d = h->cfg.d;
+  return lo < hi && hi <= d && lo % DS_SLICE_ALIGN == 0 && (hi == d || hi % DS_SLICE_ALIGN == 0);
+}
+
+bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK; }
+
+}  // namespace
+
+int ds_worker_compress_rows(ds_handle h, const float* g, uint32_t row0, uint32_t nrows, uint32_t step, void* cuda_stream) {
+  if (!h || !g || nrows == 0 || (uint64_t)row0 + nrows > h->cfg.n) return DS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(g) & 3u) != 0) return DS_ERR_ALIGN;
+  if (!sliceable(h->cfg.worker_q)) return DS_ERR_UNSUPPORTED;
+  const uint64_t d = h->cfg.d;
+  SrcParams src = worker_src(h, g);
+  src.delta = h->buf.delta_w + (uint64_t)row0 * d;
+  src.vec = (d % 4 == 0) && aligned16(g);
+  const PassWindow win{d, 0, row0};
+  return run_pass(h, SRC_WORKER, src, h->cfg.worker_q, h->wl,
+                  static_cast<uint8_t*>(h->buf.worker_payload) + (uint64_t)row0 * h->wl.stride,
+                  h->buf.delta_w + (uint64_t)row0 * d, nrows, false, nullptr, step, static_cast<cudaStream_t>(cuda_stream), &win);
+}
+
+int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flags, uint64_t lo, uint64_t hi,
+                                       void* cuda_stream) {
+  if (!h || (flags & ~DS_FUSE_APPLY) || !slice_ok(h, lo, hi)) return DS_ERR_INVALID_ARG;
+  if (!sliceable(h->cfg.worker_q) || !sliceable(h->cfg.server_q)) return DS_ERR_UNSUPPORTED;
+  int kind = 0;
+  SrcParams src = server_src(h, &kind);
+  const ds_qspec& wq = h->cfg.worker_q;
+  // the slice of every worker payload: shift each sub-array to entry lo
+  src.d = hi - lo;
+  src.delta = h->buf.delta_s + lo;
+  switch (wq.op) {
+    case DS_Q_IDENTITY: src.wp_off[0] += lo * 4; break;
+    case DS_Q_SIGN1: src.wp_off[0] += lo / 8; src.wp_off[1] += lo / wq.chunk * 4; break;
+    case DS_Q_QSGD: src.wp_off[0] += lo; src.wp_off[1] += lo / 8; src.wp_off[2] += lo / wq.chunk * 4; break;
+    case DS_Q_CLIP: src.wp_off[0] += lo * ((32 - wq.levels) / 8); break;
+    default: return DS_ERR_UNSUPPORTED;
+  }
+  const PassWindow win{hi - lo, lo, 0};
+  const bool fuse = (flags & DS_FUSE_APPLY) != 0;
+  return run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload), h->buf.delta_s + lo, 1,
+                  true, fuse ? h->buf.x + lo : nullptr, step, static_cast<cudaStream_t>(cuda_stream), &win);
+}
+
+int ds_apply_update_slice(ds_handle h, uint64_t lo, uint64_t hi, void* cuda_stream) {
+  if (!h || !slice_ok(h, lo, hi)) return DS_ERR_INVALID_ARG;
+  const ds_qspec& q = h->cfg.server_q;
+  if (!sliceable(q)) return DS_ERR_UNSUPPORTED;
+  PayloadView pv;
+  memset(&pv, 0, sizeof pv);
+  pv.op = q.op;
+  pv.base = static_cast<const uint8_t*>(h->buf.server_payload);
+  for (int i = 0; i < 3; ++i) pv.off[i] = h->sl.off[i];
+  pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD) ? log2u(q.chunk) : 0;
+  pv.levels_f = (float)q.levels;
+  pv.clip_bits = q.op == DS_Q_CLIP ? q.levels : 0;
+  switch (q.op) {
+    case DS_Q_IDENTITY: pv.off[0] += lo * 4; break;
+    case DS_Q_SIGN1: pv.off[0] += lo / 8; pv.off[1] += lo / q.chunk * 4; break;
+    case DS_Q_QSGD: pv.off[0] += lo; pv.off[1] += lo / 8; pv.off[2] += lo / q.chunk * 4; break;
+    case DS_Q_CLIP: pv.off[0] += lo * ((32 - q.levels) / 8); break;
+    default: return DS_ERR_UNSUPPORTED;
+  }
+  const cudaError_t e = launch_apply(pv, h->buf.x + lo, hi - lo, h->cfg.gamma, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "apply update");
 }
 
 int ds_step_host(ds_handle h, const float* g_host, float* g_dev, uint32_t step, void* server_payload_host, float* x_host,

@@ -209,7 +209,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
         comp(C, k) = nonneg ? s_or_q : -s_or_q;
       }
     } else {
-      const uint4 rnd = philox4x32_10(make_uint4(tq, (uint32_t)c, p.server_pass ? 0xFFFFFFFFu : row, p.step), p.keys);
+      const uint4 rnd = philox4x32_10(make_uint4(tq, (uint32_t)c + p.chunk0, p.server_pass ? 0xFFFFFFFFu : row + p.row0, p.step), p.keys);
       const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
       uint32_t lb[4];
       // r = |v| * (s / N), clamped to s

@@ -45,6 +45,8 @@ struct ChunkParams {
   uint32_t step;             // the step word of the counter
   uint32_t server_pass;      // 1: counter word 2 is 0xFFFFFFFF, else the row (worker) index
   uint32_t log2G;            // filled by the launcher
+  uint32_t chunk0;           // index of the pass's first chunk in the whole vector (a pass over a slice of d)
+  uint32_t row0;             // worker index of the pass's first row (a pass over some of the workers)
   uint32_t sign_l2;          // SIGN1: 1 = the scale is ||v_c||_2 / sqrt(len_c) instead of ||v_c||_1 / len_c
 };
 

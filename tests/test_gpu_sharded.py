@@ -1,0 +1,72 @@
+"""One worker per GPU with a sharded server (rows / slice entry points of the C ABI), checked on ONE
+GPU: all ranks live in this process, run one after the other, and exchange by plain copies.  The
+result must equal the whole-vector step bit for bit, which the other tests check against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1905_05957_b200 import DoubleSqueeze, Q
+from paper_1905_05957_b200.sharded import ShardedDoubleSqueeze, slice_bounds, step_in_process
+from tests.helpers import compare_state, to_oracle_q
+
+pytestmark = pytest.mark.gpu
+
+SIGN = Q("sign1", chunk=4096)
+PAIRS = [(SIGN, SIGN), (Q("qsgd", chunk=2048, levels=255), Q("qsgd", chunk=2048, levels=255)),
+         (Q("sign1", chunk=1024, norm=2), Q("clip", bits=16)), (Q("clip", bits=24), Q("qsgd", chunk=512, levels=7)),
+         (Q("identity"), SIGN), (Q("qsgd", chunk=8192, levels=31), Q("identity"))]
+
+
+def _bits(t):
+    return t.contiguous().view(torch.uint8).cpu()
+
+
+@pytest.mark.parametrize("wq,sq", PAIRS)
+@pytest.mark.parametrize("world,d", [(4, 5 * 8192 + 1234), (3, 8192 * 3), (5, 20_000), (2, 100)])
+def test_sharded_step_equals_whole_vector_step(wq, sq, world, d):
+    gamma, seed, T = 0.1, 77, 3
+    gen = torch.Generator().manual_seed(world * 1000 + d)
+    gs = [torch.randn(world, d, generator=gen).cuda() for _ in range(T)]
+    whole = DoubleSqueeze(world, d, gamma, wq, sq, seed)
+    st = oracle.State.zeros(world, d)
+    ranks = [ShardedDoubleSqueeze(DoubleSqueeze(world, d, gamma, wq, sq, seed), r, world) for r in range(world)]
+    bounds = slice_bounds(d, world)
+    assert bounds[0][0] == 0 and bounds[-1][1] == d and all(a[1] == b[0] for a, b in zip(bounds, bounds[1:]))
+    for t, g in enumerate(gs):
+        whole.step(g, t)
+        step_in_process(ranks, g, t)
+        torch.cuda.synchronize()
+        oracle.step(st, g.cpu().numpy(), to_oracle_q(wq), to_oracle_q(sq), gamma, seed, t)
+        compare_state(whole, st, g.cpu().numpy(), tag=f"whole, step {t}: ")
+        for r in ranks:
+            lo, hi = bounds[r.rank]
+            assert torch.equal(_bits(r.ds.x), _bits(whole.x)), f"x on rank {r.rank}, step {t}"
+            assert torch.equal(_bits(r.ds.delta_w[r.rank]), _bits(whole.delta_w[r.rank]))
+            assert torch.equal(_bits(r.ds.delta_s[lo:hi]), _bits(whole.delta_s[lo:hi]))
+            for name, view in r.ds.server_views().items():
+                assert torch.equal(_bits(view), _bits(whole.server_views()[name])), f"server payload {name} on rank {r.rank}"
+            mine, ref = r.ds.worker_views()[r.rank], whole.worker_views()[r.rank]
+            for name in mine:
+                assert torch.equal(_bits(mine[name]), _bits(ref[name])), f"worker payload {name} of rank {r.rank}"
+            assert r.ds.device_status() == 0
+    # the whole-vector result is itself the oracle's
+    assert np.array_equal(whole.x.cpu().numpy().view(np.uint32), st.x.view(np.uint32))
+
+
+def test_slices_reject_what_they_cannot_do():
+    ds = DoubleSqueeze(2, 40_000, 0.1, SIGN, SIGN)
+    g = torch.randn(2, 40_000, device="cuda")
+    ds.worker_compress_rows(g[1:2].contiguous(), 1, 0)
+    with pytest.raises(Exception, match="-1"):
+        ds.server_aggregate_compress_slice(0, 100, 8192)          # start off the grid
+    with pytest.raises(Exception, match="-1"):
+        ds.server_aggregate_compress_slice(0, 0, 8000)            # end neither on the grid nor d
+    with pytest.raises(Exception, match="-1"):
+        ds.worker_compress_rows(g, 1, 0)                          # rows 1..2 of 2
+    tk = DoubleSqueeze(2, 40_000, 0.1, Q("topk", k=10), SIGN)
+    with pytest.raises(Exception, match="-6"):
+        tk.worker_compress_rows(g[:1].contiguous(), 0, 0)
+    with pytest.raises(Exception, match="-6"):
+        tk.server_aggregate_compress_slice(0, 0, 8192)
+    torch.cuda.synchronize()
