@@ -379,6 +379,66 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+# ---------------------------------------------------------------------------------------------
+# extra mode: one worker per GPU, server sharded over the GPUs (not the headline configuration)
+# ---------------------------------------------------------------------------------------------
+
+def run_sharded(args, wl):
+    """Every rank is one worker (n = world size) and one slice of the server; the two compressed
+    hops go over NCCL point-to-point operations.  Same timing rules as the default mode; the line
+    says "mode": "sharded" and its value counts the n * d entries of one iteration."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_1905_05957_b200 import DoubleSqueeze, load_library
+    from paper_1905_05957_b200.replicas import max_over_ranks
+    from paper_1905_05957_b200.sharded import DistTransport, ShardedDoubleSqueeze
+    from paper_1905_05957_b200.workloads import make_worker_gradient
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29517")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    lib = load_library()
+    K, W = args.steps, max(args.warmup, 3)
+    swl = wl.scaled(d=wl.d, n=world)
+    ds = DoubleSqueeze(world, swl.d, swl.gamma, swl.worker_q, swl.server_q, swl.seed, device=dev)
+    sh = ShardedDoubleSqueeze(ds, rank, world)
+    tr = DistTransport()
+    R = max(2, min(K + W, int(8e9 // (swl.d * 4))))
+    ring = [make_worker_gradient(swl, t, rank, device=dev) for t in range(R)]
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for t in range(W):
+        sh.step(ring[t % R], t, tr)
+    barrier()
+    launches0 = lib.ds_kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(K):
+        sh.step(ring[(W + t) % R], W + t, tr)
+    e1.record(stream)
+    barrier()
+    (ms,) = max_over_ranks([e0.elapsed_time(e1)], device=dev)
+    if rank == 0:
+        line = {"metric": METRIC, "mode": "sharded", "value": world * swl.d * K / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": K, "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {**workload_config(swl), "workload": swl.name + "_one_worker_per_gpu", "n_workers": world},
+                "gpu_launches": int(lib.ds_kernel_launches() - launches0), "device_status": ds.device_status()}
+        print(json.dumps(line), flush=True)
+    ds.close()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -387,6 +447,9 @@ def main():
     ap.add_argument("--workload", type=int, default=2, help="1..5 = the five listed configurations, 2 = ResNet-18-sized 1-bit (the default); "
                          "6, 7 = shape of 2 with the l2-magnitude 1-bit scale / with 16-bit clipping")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "sharded"],
+                    help="replicas (default): the listed single-GPU configuration on every GPU; sharded: one worker "
+                         "per GPU with the server sharded over the GPUs (an extra, not the headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-steps", type=int, default=3)
     ap.add_argument("--dump-steps", action="store_true", help="add the per-step times to the JSON line")
@@ -398,6 +461,8 @@ def main():
         wl = wl.scaled(d=args.scale_d)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.mode == "sharded":
+        run_sharded(args, wl)
     else:
         run_ours(args, wl)
 

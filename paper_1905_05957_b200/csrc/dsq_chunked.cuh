@@ -27,6 +27,10 @@ namespace {
 // Template code of the 1-bit operator whose scale comes from l2 magnitudes (DS_NORM_L2); the
 // other values of OP are the ds_op codes.
 constexpr int kOpSign1L2 = 101;
+// ... and of the quantiser run over a window of the problem (some of the workers, or a slice of d):
+// its Philox counters carry the offsets of the window.  A separate instantiation, so that the
+// whole-vector kernels stay exactly as they were (the two extra additions cost them registers).
+constexpr int kOpQsgdWindow = 103;
 
 // Sum over the warp of row (lane % V) of a[.]; the butterfly order is lane bit 0, 1, ..., 4.
 template <int V>
@@ -209,7 +213,8 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
         comp(C, k) = nonneg ? s_or_q : -s_or_q;
       }
     } else {
-      const uint4 rnd = philox4x32_10(make_uint4(tq, (uint32_t)c + p.chunk0, p.server_pass ? 0xFFFFFFFFu : row + p.row0, p.step), p.keys);
+      const uint4 rnd = philox4x32_10(make_uint4(tq, OP == kOpQsgdWindow ? (uint32_t)c + p.chunk0 : (uint32_t)c,
+                                                  p.server_pass ? 0xFFFFFFFFu : (OP == kOpQsgdWindow ? row + p.row0 : row), p.step), p.keys);
       const uint32_t w[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
       uint32_t lb[4];
       // r = |v| * (s / N), clamped to s
@@ -275,8 +280,17 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
   }
 }
 
+// Resident CTAs the kernel is compiled for.  Worker passes take what the compiler gives, except the
+// windowed quantiser: its worker pass is bound by instruction issue and wants six CTAs (40
+// registers, what the whole-vector kernel gets by itself; with 48 it measured 8 % slower).  Server
+// passes see kServerCtasPerSm.
+constexpr int chunk_ctas(int op, int src, int v) {
+  if (src == SRC_WORKER) return (op == kOpQsgdWindow && v <= 2) ? 6 : 0;
+  return v >= 8 ? 2 : kServerCtasPerSm;
+}
+
 template <int OP, int SRC, int V, int LOG2G>
-__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : (V >= 8 ? 2 : kServerCtasPerSm)) k_chunked(const SrcParams src, const ChunkParams p) {
+__global__ void __launch_bounds__(kThreads, chunk_ctas(OP, SRC, V)) k_chunked(const SrcParams src, const ChunkParams p) {
   pdl_prologue();
   __shared__ float s_red[64];
   __shared__ float s_scal[16];

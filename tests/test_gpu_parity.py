@@ -195,6 +195,32 @@ def test_workload_recipes_scaled(wid):
     run_lockstep(wl.n, wl.d, wl.worker_q, wl.server_q, gs, gamma=wl.gamma, seed=wl.seed)
 
 
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7])
+def test_telescoping_identity_free_running_on_the_gpu(wid):
+    """Eq. 5-6 on the GPU alone, with no oracle in the loop: after T steps of any Q,
+    x_T - gamma (delta_T + mean_i delta_T^(i)) = x_0 - gamma sum_t mean_i g_t^(i), up to fp32 rounding."""
+    wl = WORKLOADS[wid]
+    wl = wl if wid == 1 else wl.scaled(d=300_000 + 8, n=min(wl.n, 8))
+    T = 20
+    ds = DoubleSqueeze.for_workload(wl, "cuda")
+    x0 = torch.randn(wl.d, generator=torch.Generator().manual_seed(wid)).cuda()
+    ds.x.copy_(x0)
+    rhs = x0.double()
+    gmax = 0.0
+    for t in range(T):
+        g = make_gradients(wl, t, device="cuda")
+        ds.step(g, t)
+        rhs -= wl.gamma * g.double().mean(dim=0)
+        gmax = max(gmax, float(g.abs().max()))
+    torch.cuda.synchronize()
+    omega = ds.delta_s.double() + ds.delta_w.double().mean(dim=0)
+    lhs = ds.x.double() - wl.gamma * omega
+    scale = max(float(rhs.abs().max()), gmax, float(omega.abs().max()))
+    assert float((lhs - rhs).abs().max()) <= 40 * T * 2.0**-24 * scale
+    assert ds.device_status() == 0
+    ds.close()
+
+
 def test_state_copied_into_a_fresh_instance_continues_identically():
     """x, delta_w and delta_s are the whole state (Algorithm 1): T steps, copy them into a new
     instance (which has no threshold history), T more steps -- same bits as 2T steps in one go."""
