@@ -14,7 +14,7 @@ import numpy as np
 
 from . import build as _build
 
-IDENTITY, SIGN1, TOPK, QSGD, CLIP = "identity", "sign1", "topk", "qsgd", "clip"
+IDENTITY, SIGN1, TOPK, QSGD, CLIP, RSPARSE = "identity", "sign1", "topk", "qsgd", "clip", "rsparse"
 SERVER_WID = 0xFFFFFFFF
 
 _lib = None
@@ -46,6 +46,8 @@ def load(path: str):
     L.orc_decode_qsgd.argtypes = [u8p, u32p, f32p, u64, u32, f32p]
     L.orc_q_clip.argtypes = [f32p, u64, u32, u8p, f32p]
     L.orc_decode_clip.argtypes = [u8p, u64, u32, f32p]
+    L.orc_q_rsparse.argtypes = [f32p, u64, u32, u32, u32, u64, u32, u32, f32p, u32p, f32p]
+    L.orc_decode_rsparse.argtypes = [f32p, u32p, u64, u32, u32, f32p]
     return L
 
 
@@ -127,6 +129,8 @@ class QSpec:
     norm: int = 1       # sign1: the scale is the ratio of l1 (1) or l2 (2) magnitudes
     k: int = 0          # topk
     levels: int = 0     # qsgd: s
+    keep_one_in: int = 0  # rsparse: S, an element survives with probability 1/S
+    scaled: int = 0     # rsparse: 1 = survivors are multiplied by S (unbiased), 0 = kept as they are
     bits: int = 0       # clip: how many low bits of each binary32 number are set to zero (16 or 24)
 
 
@@ -217,6 +221,26 @@ def decode_clip(hi, d, b):
     return Cv
 
 
+def q_rsparse(v, L, S, scaled, seed, step, wid):
+    v = _f32(v)
+    d = v.size
+    nc = (d + L - 1) // L
+    val = np.zeros(nc * max(L // max(S, 1), 1), dtype=np.float32)
+    off = np.zeros(nc, dtype=np.uint32)
+    Cv = np.empty_like(v)
+    _check(lib().orc_q_rsparse(_p(v, C.c_float), d, L, S, scaled, C.c_uint64(seed), step, wid, _p(val, C.c_float),
+                               _p(off, C.c_uint32), _p(Cv, C.c_float)), "rsparse")
+    return Cv, {"val": val, "off": off}
+
+
+def decode_rsparse(val, off, d, L, S):
+    val = _f32(val)
+    off = np.ascontiguousarray(off, dtype=np.uint32)
+    Cv = np.empty(d, dtype=np.float32)
+    _check(lib().orc_decode_rsparse(_p(val, C.c_float), _p(off, C.c_uint32), d, L, S, _p(Cv, C.c_float)), "decode_rsparse")
+    return Cv
+
+
 def compress(q: QSpec, v, seed=0, step=0, wid=0):
     """Q_omega[v] for the operator ``q``; omega = (seed, step, wid) where Q is random."""
     if q.op == IDENTITY:
@@ -229,6 +253,8 @@ def compress(q: QSpec, v, seed=0, step=0, wid=0):
         return q_qsgd(v, q.chunk, q.levels, seed, step, wid)
     if q.op == CLIP:
         return q_clip(v, q.bits)
+    if q.op == RSPARSE:
+        return q_rsparse(v, q.chunk, q.keep_one_in, q.scaled, seed, step, wid)
     raise ValueError(q.op)
 
 

@@ -25,7 +25,8 @@
  * (Eq. 5-6); sign scale == ||v||_1/len (or ||v||_2/sqrt(len)) and its closed-form residual energy;
  * top-k against a brute-force stable sort; QSGD unbiasedness and variance by
  * Monte Carlo plus its deterministic special cases; clipping against worked
- * binary cases, its error bound and idempotence; Philox4x32-10 against an
+ * binary cases, its error bound and idempotence; randomised sparsification by
+ * its keep frequency, its mean, and the structure of what it sends; Philox4x32-10 against an
  * independent library implementation; pairwise summation against hand-derived
  * rounding cases.  No function here is "parity unpinned".
  */
@@ -244,6 +245,68 @@ int orc_decode_clip(const uint8_t* hi, uint64_t d, uint32_t b, float* C) {
     for (uint32_t t = 0; t < bytes; ++t) kept |= (uint32_t)hi[j * bytes + t] << (8 * t);
     uint32_t u = kept << b;
     memcpy(&C[j], &u, sizeof u);
+  }
+  return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Q = randomised sparsification (the last option of Section 3.2: a number   */
+/* survives with probability p, scaled by 1/p so that the operator is        */
+/* unbiased, else it becomes 0).  Reading: p = 1/S with S a power of two,    */
+/* and the numbers of a chunk of L consecutive elements share one random     */
+/* draw (systematic sampling): with o uniform in {0, ..., S-1}, the element  */
+/* at offset t in the chunk survives iff t mod S == o.  Every element still  */
+/* survives with probability exactly 1/S, which is all the option states,    */
+/* and every chunk sends exactly L/S values whose positions follow from o.   */
+/* The draw is the first output word of Philox4x32-10 with key = seed and    */
+/* counter = (0xFFFFFFFF, chunk, wid, step), reduced mod S.                  */
+/*   scaled = 1: survivors become S * v (exact, a power of two): the option  */
+/*               as printed.  Unbiased, but E||v - Q[v]||^2 = (S-1)||v||^2,  */
+/*               no contraction: the compensated error grows under it.       */
+/*   scaled = 0: survivors keep v: E||v - Q[v]||^2 = (1 - 1/S)||v||^2, a     */
+/*               contraction, the form error compensation can carry.         */
+/*   val : ceil(d/L) * (L/S) floats; slot j/S holds Q[v]_j of the survivor   */
+/*         j, slots of positions past d stay +0                              */
+/*   off : ceil(d/L) words, the o of every chunk                             */
+/*   C   : d floats (may be NULL)                                            */
+/* ------------------------------------------------------------------------ */
+
+int orc_q_rsparse(const float* v, uint64_t d, uint32_t L, uint32_t S, uint32_t scaled, uint64_t seed, uint32_t step,
+                  uint32_t wid, float* val, uint32_t* off, float* C) {
+  if (!is_pow2_u32(L) || !is_pow2_u32(S) || S < 2 || S > L || scaled > 1) return ORC_ERR_ARG;
+  uint64_t nc = (d + L - 1) / L;
+  uint32_t per = L / S;
+  const uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
+  const float factor = scaled ? (float)S : 1.0f;
+  for (uint64_t c = 0; c < nc; ++c) {
+    uint64_t lo = c * L, hi = lo + L < d ? lo + L : d;
+    uint32_t ctr[4] = {0xFFFFFFFFu, (uint32_t)c, wid, step};
+    uint32_t rnd[4];
+    orc_philox4x32_10(ctr, key, rnd);
+    uint32_t o = rnd[0] % S;
+    off[c] = o;
+    for (uint32_t u = 0; u < per; ++u) val[c * per + u] = 0.0f;
+    for (uint64_t j = lo; j < hi; ++j) {
+      uint32_t t = (uint32_t)(j - lo);
+      if (t % S == o) {
+        float kept = factor * v[j];
+        val[c * per + t / S] = kept;
+        if (C) C[j] = kept;
+      } else if (C) {
+        C[j] = 0.0f;
+      }
+    }
+  }
+  return ORC_OK;
+}
+
+int orc_decode_rsparse(const float* val, const uint32_t* off, uint64_t d, uint32_t L, uint32_t S, float* C) {
+  if (L == 0 || S == 0 || S > L) return ORC_ERR_ARG;
+  uint32_t per = L / S;
+  for (uint64_t j = 0; j < d; ++j) {
+    uint64_t c = j / L;
+    uint32_t t = (uint32_t)(j % L);
+    C[j] = (t % S == off[c]) ? val[c * per + t / S] : 0.0f;
   }
   return ORC_OK;
 }

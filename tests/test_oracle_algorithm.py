@@ -12,10 +12,12 @@ QS = {
     "topk": QSpec(oracle.TOPK, k=37),
     "qsgd": QSpec(oracle.QSGD, chunk=128, levels=15),
     "clip": QSpec(oracle.CLIP, bits=16),
+    "rsparse": QSpec(oracle.RSPARSE, chunk=128, keep_one_in=4, scaled=0),
 }
 PAIRS = [("identity", "identity"), ("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"),
          ("sign1", "topk"), ("topk", "identity"), ("qsgd", "sign1"), ("sign1_l2", "sign1_l2"), ("sign1_l2", "sign1"),
-         ("clip", "clip"), ("clip", "topk"), ("sign1", "clip")]
+         ("clip", "clip"), ("clip", "topk"), ("sign1", "clip"),
+         ("rsparse", "rsparse"), ("rsparse", "sign1"), ("topk", "rsparse")]
 
 
 def _grads(n, d, T, seed=0):
@@ -50,7 +52,7 @@ def test_residual_reconstructs_compensated_gradient(wq, sq):
         v_w = g + old_w
         tol = 2.0**-23 * np.maximum(np.abs(v_w), np.abs(C_all))
         assert np.all(np.abs((C_all.astype(np.float64) + st.delta_w) - v_w) <= tol)
-        if wq in ("identity", "topk", "clip"):
+        if wq in ("identity", "topk", "clip", "rsparse"):
             assert np.array_equal(C_all + st.delta_w, v_w)
         Cv = oracle.server_pass(st, C_all, QS[sq], 1, t)
         v_s = oracle.server_mean_add(C_all, old_s)
@@ -76,7 +78,8 @@ def test_telescoping_identity_of_the_global_update_rule(wq, sq):
     assert np.max(np.abs(lhs - rhs)) <= 40 * T * 2.0**-24 * scale
 
 
-@pytest.mark.parametrize("wq,sq", [("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"), ("sign1_l2", "sign1_l2")])
+@pytest.mark.parametrize("wq,sq", [("sign1", "sign1"), ("topk", "topk"), ("qsgd", "qsgd"), ("sign1_l2", "sign1_l2"),
+                                   ("rsparse", "rsparse")])
 def test_error_stays_bounded_on_stationary_gradients(wq, sq):
     """Section 4: a contracting Q keeps ||delta_t|| bounded; a broken residual makes it grow."""
     n, d, T = 2, 512, 120
@@ -86,6 +89,23 @@ def test_error_stays_bounded_on_stationary_gradients(wq, sq):
         oracle.step(st, g, QS[wq], QS[sq], 0.1, 8, t)
         norms.append(np.linalg.norm(st.delta_w) + np.linalg.norm(st.delta_s))
     assert max(norms[T // 2:]) <= 1.5 * max(norms[:T // 2]) + 1e-6
+
+
+def test_scaled_sparsifier_is_no_contraction_and_its_error_grows():
+    """The unbiased form of Section 3.2's last option has E||v - Q[v]||^2 = (1/p - 1)||v||^2 >= ||v||^2 for
+    p <= 1/2, outside the bounded-error assumption of Section 4: under compensation the error grows
+    geometrically, while the unscaled form (a contraction) stays bounded on the same inputs."""
+    n, d, T = 2, 512, 14
+    grown = {}
+    for scaled in (0, 1):
+        q = QSpec(oracle.RSPARSE, chunk=128, keep_one_in=4, scaled=scaled)
+        st = oracle.State.zeros(n, d)
+        norms = []
+        for t, g in enumerate(_grads(n, d, T, seed=4)):
+            oracle.worker_pass(st, g, q, 8, t)
+            norms.append(float(np.linalg.norm(st.delta_w)))
+        grown[scaled] = norms[-1] / norms[1]
+    assert grown[1] > 1e3 and grown[0] < 5
 
 
 def test_server_uses_its_own_stream_and_workers_differ():

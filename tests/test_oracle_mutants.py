@@ -33,6 +33,15 @@ MUTANTS = [
     ("clipping rounds to nearest instead of clearing bits",
      "uint32_t kept = u >> b;       /* the high 32 - b bits */", "uint32_t kept = (u + (1u << (b - 1))) >> b;",
      t_ops.test_clip_worked_binary_cases),
+    ("sparsifier scales by S - 1",
+     "const float factor = scaled ? (float)S : 1.0f;", "const float factor = scaled ? (float)(S - 1) : 1.0f;",
+     t_ops.test_rsparse_keeps_each_entry_with_probability_one_in_S_and_scaled_form_is_unbiased),
+    ("sparsifier draws from the second Philox word",
+     "uint32_t o = rnd[0] % S;", "uint32_t o = rnd[1] % S;",
+     lambda: t_ops.test_rsparse_structure_of_what_is_sent(1)),
+    ("sparsifier keeps offsets o and o + 1",
+     "if (t % S == o) {", "if (t % S == o || t % S == (o + 1) % S) {",
+     lambda: t_ops.test_rsparse_structure_of_what_is_sent(0)),
     ("sign bit is v > 0",
      "int nonneg = v[j] >= 0.0f;\n      if (nonneg) bits[j / 32]", "int nonneg = v[j] > 0.0f;\n      if (nonneg) bits[j / 32]",
      lambda: t_ops.test_sign1_scale_is_l1_mean_per_chunk_and_bits_are_signs(10000, 4096)),

@@ -297,3 +297,62 @@ def test_clip_error_bound_idempotence_exact_residual_and_decode(b):
     assert np.array_equal(oracle.decode_clip(p["hi"], v.size, b).view(np.uint32), C.view(np.uint32))
     # a contraction (Section 4 needs ||v - Q[v]|| <= alpha ||v|| with alpha < 1 on what it is applied to)
     assert np.linalg.norm(delta.astype(np.float64)) < np.linalg.norm(v.astype(np.float64))
+
+
+# ------------------------------------------------------------------ randomised sparsification
+
+@pytest.mark.parametrize("scaled", [0, 1])
+def test_rsparse_structure_of_what_is_sent(scaled):
+    """One draw per chunk: exactly L/S survivors per full chunk, S apart; scaled by S exactly or kept."""
+    L, S, d = 256, 8, 3 * 256 + 100
+    v = _rng(61).standard_normal(d).astype(np.float32)
+    C, p = oracle.q_rsparse(v, L, S, scaled, seed=5, step=2, wid=1)
+    f = np.float32(S if scaled else 1)
+    assert p["off"].shape == (4,) and np.all(p["off"] < S) and p["val"].shape == (4 * L // S,)
+    for c in range(4):
+        seg = slice(c * L, min((c + 1) * L, d))
+        o = int(p["off"][c])
+        want = np.arange(o, seg.stop - seg.start, S)
+        mask = np.zeros(seg.stop - seg.start, bool)
+        mask[want] = True
+        assert np.array_equal(C[seg][mask], f * v[seg][mask]) and not C[seg][~mask].any()   # power of two: exact
+        slots = p["val"][c * (L // S):(c + 1) * (L // S)]
+        assert np.array_equal(slots[:len(want)], C[seg][want]) and not slots[len(want):].any()
+        w = oracle.philox4x32_10([0xFFFFFFFF, c, 1, 2], [5, 0])     # the draw: first word, counter as documented
+        assert o == int(w[0]) % S
+    assert np.array_equal(oracle.decode_rsparse(p["val"], p["off"], d, L, S), C)
+    others = [oracle.q_rsparse(v, L, S, scaled, 5, 2, 2)[1]["off"], oracle.q_rsparse(v, L, S, scaled, 5, 3, 1)[1]["off"],
+              oracle.q_rsparse(v, L, S, scaled, 6, 2, 1)[1]["off"]]
+    assert all(not np.array_equal(o2, p["off"]) for o2 in others)   # other worker, step, seed: other draws
+    with pytest.raises(ValueError):
+        oracle.q_rsparse(v, L, 3, scaled, 5, 2, 1)
+    with pytest.raises(ValueError):
+        oracle.q_rsparse(v, L, 2 * L, scaled, 5, 2, 1)
+
+
+def test_rsparse_keeps_each_entry_with_probability_one_in_S_and_scaled_form_is_unbiased():
+    """Section 3.2: survive with probability p (here 1/S) and scale by 1/p, else 0 => E Q[v] = v."""
+    L, S, d, M = 128, 4, 512, 4000
+    v = _rng(62).standard_normal(d).astype(np.float32)
+    acc = np.zeros(d)
+    kept = np.zeros(d)
+    err2 = [0.0, 0.0]
+    for t in range(M):
+        C, _ = oracle.q_rsparse(v, L, S, 1, seed=9, step=t, wid=0)
+        acc += C
+        kept += C != 0
+        err2[1] += float(((v - C).astype(np.float64) ** 2).sum())
+        C0, _ = oracle.q_rsparse(v, L, S, 0, seed=9, step=t, wid=0)
+        err2[0] += float(((v - C0).astype(np.float64) ** 2).sum())
+    freq = kept / M
+    sigma = math.sqrt((1 / S) * (1 - 1 / S) / M)
+    assert np.all(np.abs(freq - 1 / S) < 5 * sigma)                 # per-entry keep frequency
+    tol = 5 * np.abs(v) * math.sqrt((S - 1) / M) + 1e-12            # Var Q_j = v_j^2 (S - 1)
+    assert np.all(np.abs(acc / M - v) <= tol)
+    # the four offsets of a chunk are equally likely (chi-square, 3 degrees of freedom)
+    offs = np.array([oracle.q_rsparse(v[:L], L, S, 1, 9, t, 0)[1]["off"][0] for t in range(M)])
+    counts = np.bincount(offs, minlength=S)
+    assert ((counts - M / S) ** 2 / (M / S)).sum() < 21.1           # P(chi2_3 > 21.1) ~ 1e-4
+    # mean squared error: (S - 1) ||v||^2 scaled (no contraction), (1 - 1/S) ||v||^2 unscaled (a contraction)
+    n2 = float((v.astype(np.float64) ** 2).sum())
+    assert abs(err2[1] / M / n2 - (S - 1)) < 0.05 * (S - 1) and abs(err2[0] / M / n2 - (1 - 1 / S)) < 0.05
