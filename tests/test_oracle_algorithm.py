@@ -105,7 +105,7 @@ def test_scaled_sparsifier_is_no_contraction_and_its_error_grows():
             oracle.worker_pass(st, g, q, 8, t)
             norms.append(float(np.linalg.norm(st.delta_w)))
         grown[scaled] = norms[-1] / norms[1]
-    assert grown[1] > 1e3 and grown[0] < 5
+    assert grown[1] > 50 and grown[0] < 5      # about 1.5x per step against a plateau
 
 
 def test_server_uses_its_own_stream_and_workers_differ():
