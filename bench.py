@@ -44,6 +44,7 @@ KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "topk": ("dsq_topk.cu", "dsq_common.cuh", "dsq_internal.h"),
     "identity": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
     "clip": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
+    "rsparse": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
 }
 
 
@@ -57,6 +58,9 @@ def payload_bytes(q, d: int) -> int:
         return 8 * q.k
     if q.op == "clip":
         return d * (32 - q.bits) // 8
+    if q.op == "rsparse":
+        nc = (d + q.chunk - 1) // q.chunk
+        return 4 * nc * (q.chunk // q.keep_one_in) + 4 * nc
     return 4 * d
 
 
@@ -195,7 +199,8 @@ def workload_config(wl) -> dict:
     def q(s):
         return {"op": s.op, **({"chunk": s.chunk} if s.chunk else {}), **({"k": s.k} if s.op == "topk" else {}),
                 **({"levels": s.levels} if s.levels else {}), **({"norm": "l2"} if s.op == "sign1" and s.norm == 2 else {}),
-                **({"bits_cleared": s.bits} if s.op == "clip" else {})}
+                **({"bits_cleared": s.bits} if s.op == "clip" else {}),
+                **({"keep_one_in": s.keep_one_in, "scaled": bool(s.scaled)} if s.op == "rsparse" else {})}
     return {"workload": wl.name, "n_workers": wl.n, "d": wl.d, "gradient_dist": wl.dist, "worker_q": q(wl.worker_q),
             "server_q": q(wl.server_q), "gamma": wl.gamma,
             "l2": "inputs larger than L2: g and delta_w are streamed once per step and exceed 126 MB"
@@ -344,7 +349,8 @@ def run_ours(args, wl):
             traffic = NCU_TRAFFIC[wl.wid][1]
         dominant = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
                     "topk": "top-k worker pass (pass1, mark, refine, finalize, emit)",
-                    "identity": "k_identity<WORKER>", "clip": "k_clip<WORKER>"}[wl.worker_q.op]
+                    "identity": "k_identity<WORKER>", "clip": "k_clip<WORKER>",
+                    "rsparse": "k_rsparse<WORKER>"}[wl.worker_q.op]
         line = {
             "metric": METRIC, "value": aggregate_throughput(wl.n * wl.d, K, t_total, world), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": t_total / K, "higher_is_better": True, "scaling": "weak",
@@ -445,7 +451,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", type=int, default=2, help="1..5 = the five listed configurations, 2 = ResNet-18-sized 1-bit (the default); "
-                         "6, 7 = shape of 2 with the l2-magnitude 1-bit scale / with 16-bit clipping")
+                         "6, 7, 8 = shape of 2 with the l2-magnitude 1-bit scale / 16-bit clipping / randomised sparsification")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="replicas", choices=["replicas", "sharded"],
                     help="replicas (default): the listed single-GPU configuration on every GPU; sharded: one worker "

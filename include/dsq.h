@@ -89,21 +89,36 @@ typedef enum {
  *                the surviving high 32 - levels bits of every entry.  The residual v - Q[v] is
  *                exact.
  *
+ * DS_Q_RSPARSE   "Randomized Sparsification" of Section 3.2: a number survives with probability 1/S
+ *                (S = `levels`, a power of two) and becomes 0 otherwise.  The entries of a chunk of
+ *                `chunk` consecutive entries share one draw o, uniform in 0..S-1 (Philox4x32-10,
+ *                key = seed, counter = (0xFFFFFFFF, chunk index, worker index or 0xFFFFFFFF on
+ *                the server pass, step), first output word mod S): the entry at offset t of its
+ *                chunk survives iff t mod S == o, so each entry survives with probability exactly
+ *                1/S and a chunk always sends chunk/S values.  norm = DS_RSPARSE_SCALED: survivors
+ *                are multiplied by S, the unbiased form the paper prints (no contraction: its
+ *                compensated error grows; offered for completeness).  norm = DS_RSPARSE_PLAIN:
+ *                survivors keep their value (a contraction).
+ *
  * Chunk reductions (sum of |v| or of v*v) are pairwise sums in index order over the chunk padded
  * with zeros to `chunk` entries, so results do not depend on launch geometry.
  */
-typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3, DS_Q_CLIP = 4 } ds_op;
+typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3, DS_Q_CLIP = 4, DS_Q_RSPARSE = 5 } ds_op;
 
 /* ds_qspec.norm for DS_Q_SIGN1 */
 #define DS_NORM_L1 0u /* s_c = ||v_c||_1 / len_c (also selected by 1) */
 #define DS_NORM_L2 2u /* s_c = ||v_c||_2 / sqrt(len_c) */
+/* ds_qspec.norm for DS_Q_RSPARSE */
+#define DS_RSPARSE_PLAIN 0u  /* survivors keep their value */
+#define DS_RSPARSE_SCALED 1u /* survivors are multiplied by S */
 
 typedef struct {
   int32_t op;        /* ds_op */
-  uint32_t chunk;    /* SIGN1, QSGD: a power of two in [128, 8192]; else ignored */
+  uint32_t chunk;    /* SIGN1, QSGD, RSPARSE: a power of two in [128, 8192]; else ignored */
   uint64_t k;        /* TOPK: 0 <= k <= d; else ignored */
-  uint32_t levels;   /* QSGD: 1 <= levels <= 255; CLIP: bits set to zero, 16 or 24; else ignored */
-  uint32_t norm;     /* SIGN1: DS_NORM_L1 (0 or 1) or DS_NORM_L2 (2); else must be 0 */
+  uint32_t levels;   /* QSGD: 1 <= levels <= 255; CLIP: bits set to zero, 16 or 24;
+                        RSPARSE: S, a power of two in [2, 128]; else ignored */
+  uint32_t norm;     /* SIGN1: DS_NORM_L1 (0 or 1) or DS_NORM_L2 (2); RSPARSE: DS_RSPARSE_*; else must be 0 */
 } ds_qspec;
 
 typedef struct {
@@ -154,6 +169,8 @@ typedef struct {
  *             [2] float  step[ceil(d/chunk)] (the grid step q = N_c / levels that multiplies the
  *                 levels; 0 for a chunk sent as all zeros)
  *   CLIP      [0] uint16 hi[d] (levels = 16) or uint8 hi[d] (levels = 24): bits(v) >> levels
+ *   RSPARSE   [0] float  val[ceil(d/chunk) * chunk/S]  slot j/S = Q[v]_j of the survivor j, +0 where j >= d
+ *             [1] uint32 off[ceil(d/chunk)]            the draw o of every chunk
  */
 typedef struct {
   uint64_t stride;
@@ -216,7 +233,7 @@ int ds_destroy(ds_handle h);
  * ds_apply_update_slice: x = x - gamma Q[v] on lo .. hi-1 from that slice of the server payload.
  *
  * Operators that act per chunk or per entry (IDENTITY, SIGN1, QSGD, CLIP) are supported on both
- * passes; a global TOPK on either pass is DS_ERR_UNSUPPORTED here (its threshold is a property of
+ * passes; a global TOPK on either pass, and RSPARSE, are DS_ERR_UNSUPPORTED here (its threshold is a property of
  * the whole vector).  These calls do not take part in the worker -> server -> apply order check
  * of the whole-vector calls: the caller sequences its slices.  Errors as for the whole-vector calls.
  */

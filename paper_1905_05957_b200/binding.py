@@ -20,7 +20,7 @@ DS_ERR_INVALID_ARG, DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL = -1, -2, -3
 DS_ERR_STATE, DS_ERR_CUDA, DS_ERR_UNSUPPORTED = -4, -5, -6
 DS_FUSE_APPLY = 1
 DS_DEV_TOPK_INCONSISTENT = 1
-OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4}
+OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4, "rsparse": 5}
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
            "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
            "ds_kernel_launches", "ds_topk_worker_static", "ds_worker_compress_rows",
@@ -90,7 +90,9 @@ def load_library() -> C.CDLL:
 
 
 def _qspec(q: Q) -> ds_qspec:
-    return ds_qspec(OPS[q.op], q.chunk, q.k, q.bits if q.op == "clip" else q.levels, q.norm if q.op == "sign1" else 0)
+    levels = {"clip": q.bits, "rsparse": q.keep_one_in}.get(q.op, q.levels)
+    norm = {"sign1": q.norm, "rsparse": q.scaled}.get(q.op, 0)
+    return ds_qspec(OPS[q.op], q.chunk, q.k, levels, norm)
 
 
 def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int) -> ds_config:
@@ -110,6 +112,7 @@ _VIEW_DTYPES = {
     "sign1": (("bits", torch.int32), ("scale", torch.float32)),
     "topk": (("idx", torch.int32), ("val", torch.float32)),
     "qsgd": (("lvl", torch.uint8), ("sgn", torch.int32), ("step", torch.float32)),
+    "rsparse": (("val", torch.float32), ("off", torch.int32)),
     "clip": (("hi", torch.int16),),      # 8-bit entries when 24 bits are cleared, see payload_views
 }
 

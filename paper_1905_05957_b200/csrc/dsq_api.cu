@@ -28,13 +28,17 @@ inline uint32_t log2u(uint32_t x) { uint32_t l = 0; while ((1u << l) < x) ++l; r
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 bool qspec_ok(const ds_qspec& q, uint64_t d) {
-  if (q.op == DS_Q_SIGN1 ? (q.norm != DS_NORM_L1 && q.norm != 1u && q.norm != DS_NORM_L2) : q.norm != 0) return false;
+  if (q.op == DS_Q_SIGN1 ? (q.norm != DS_NORM_L1 && q.norm != 1u && q.norm != DS_NORM_L2)
+                         : (q.op == DS_Q_RSPARSE ? q.norm > DS_RSPARSE_SCALED : q.norm != 0))
+    return false;
   switch (q.op) {
     case DS_Q_IDENTITY: return true;
     case DS_Q_SIGN1: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192;
     case DS_Q_QSGD: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192 && q.levels >= 1 && q.levels <= 255;
     case DS_Q_TOPK: return q.k <= d;
     case DS_Q_CLIP: return q.levels == 16 || q.levels == 24;
+    case DS_Q_RSPARSE:
+      return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192 && is_pow2(q.levels) && q.levels >= 2 && q.levels <= 128;
     default: return false;
   }
 }
@@ -62,6 +66,7 @@ void layout_of(const ds_qspec& q, uint64_t d, ds_payload_layout* L) {
     case DS_Q_TOPK: put(0, q.k, 4); put(1, q.k, 4); break;
     case DS_Q_QSGD: put(0, d, 1); put(1, nw, 4); put(2, (d + q.chunk - 1) / q.chunk, 4); break;
     case DS_Q_CLIP: put(0, d, (32 - q.levels) / 8); break;
+    case DS_Q_RSPARSE: put(0, (d + q.chunk - 1) / q.chunk * (q.chunk / q.levels), 4); put(1, (d + q.chunk - 1) / q.chunk, 4); break;
   }
   L->stride = pos ? pos : 16;
 }
@@ -139,7 +144,8 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
   s.wp = static_cast<const uint8_t*>(c->buf.worker_payload);
   s.wp_stride = c->wl.stride;
   for (int i = 0; i < 3; ++i) s.wp_off[i] = c->wl.off[i];
-  s.w_log2_chunk = (wq.op == DS_Q_SIGN1 || wq.op == DS_Q_QSGD) ? log2u(wq.chunk) : 0;
+  s.w_log2_chunk = (wq.op == DS_Q_SIGN1 || wq.op == DS_Q_QSGD || wq.op == DS_Q_RSPARSE) ? log2u(wq.chunk) : 0;
+  s.w_log2_keep = wq.op == DS_Q_RSPARSE ? log2u(wq.levels) : 0;
   s.w_levels = (float)wq.levels;
   s.w_clip_bits = wq.op == DS_Q_CLIP ? wq.levels : 0;
   s.acc = c->acc;
@@ -149,6 +155,7 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
     case DS_Q_SIGN1: *kind = SRC_SRV_SIGN1; break;
     case DS_Q_TOPK: *kind = SRC_SRV_TOPK; break;
     case DS_Q_CLIP: *kind = SRC_SRV_CLIP; break;
+    case DS_Q_RSPARSE: *kind = SRC_SRV_RSPARSE; break;
     default: *kind = SRC_SRV_QSGD; break;
   }
   return s;
@@ -223,6 +230,23 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       e = launch_clip(src_kind, src, q.levels, payload + L.off[0] + lo * ((32 - q.levels) / 8), L.stride, delta, row_stride,
                       x_fused, c->cfg.gamma, rows, st);
       break;
+    case DS_Q_RSPARSE: {
+      if (win) return DS_ERR_UNSUPPORTED;
+      RsparseParams rp;
+      memset(&rp, 0, sizeof rp);
+      rp.out_val = reinterpret_cast<float*>(payload + L.off[0]);
+      rp.out_off = reinterpret_cast<uint32_t*>(payload + L.off[1]);
+      rp.val_stride = L.stride / 4;
+      rp.off_stride = L.stride / 4;
+      rp.log2_chunk = log2u(q.chunk);
+      rp.log2_keep = log2u(q.levels);
+      rp.scaled = q.norm == DS_RSPARSE_SCALED ? 1u : 0u;
+      rp.keys = philox_key_schedule((uint32_t)(c->cfg.seed & 0xFFFFFFFFu), (uint32_t)(c->cfg.seed >> 32));
+      rp.step = step;
+      rp.server_pass = server ? 1u : 0u;
+      e = launch_rsparse(src_kind, src, rp, delta, row_stride, x_fused, c->cfg.gamma, rows, st);
+      break;
+    }
     default: return DS_ERR_UNSUPPORTED;
   }
   return e == cudaSuccess ? DS_OK : cuda_fail(e, "kernel launch");
@@ -324,9 +348,10 @@ int ds_apply_update(ds_handle h, void* cuda_stream) {
   pv.op = q.op;
   pv.base = static_cast<const uint8_t*>(h->buf.server_payload);
   for (int i = 0; i < 3; ++i) pv.off[i] = h->sl.off[i];
-  pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD) ? log2u(q.chunk) : 0;
+  pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD || q.op == DS_Q_RSPARSE) ? log2u(q.chunk) : 0;
   pv.levels_f = (float)q.levels;
   pv.clip_bits = q.op == DS_Q_CLIP ? q.levels : 0;
+  pv.log2_keep = q.op == DS_Q_RSPARSE ? log2u(q.levels) : 0;
   pv.k = q.k;
   const cudaError_t e = launch_apply(pv, h->buf.x, h->cfg.d, h->cfg.gamma, static_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return cuda_fail(e, "apply update");
@@ -341,7 +366,7 @@ bool slice_ok(const ds_ctx* h, uint64_t lo, uint64_t hi) {
   return lo < hi && hi <= d && lo % DS_SLICE_ALIGN == 0 && (hi == d || hi % DS_SLICE_ALIGN == 0);
 }
 
-bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK; }
+bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK && q.op != DS_Q_RSPARSE; }
 
 }  // namespace
 

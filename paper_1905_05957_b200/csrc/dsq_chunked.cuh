@@ -332,6 +332,7 @@ cudaError_t launch_src(int srck, const SrcParams& src, const ChunkParams& p, uin
     case SRC_SRV_TOPK: return launch_v<OP, SRC_SRV_TOPK>(src, p, rows, chunk, st);
     case SRC_SRV_QSGD: return launch_v<OP, SRC_SRV_QSGD>(src, p, rows, chunk, st);
     case SRC_SRV_CLIP: return launch_v<OP, SRC_SRV_CLIP>(src, p, rows, chunk, st);
+    case SRC_SRV_RSPARSE: return launch_v<OP, SRC_SRV_RSPARSE>(src, p, rows, chunk, st);
   }
   return cudaErrorInvalidValue;
 }

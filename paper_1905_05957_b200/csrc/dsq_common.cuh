@@ -30,6 +30,7 @@ enum Src : int {
   SRC_SRV_TOPK = 3,      // the sparse payloads were summed into a dense accumulator beforehand
   SRC_SRV_QSGD = 4,
   SRC_SRV_CLIP = 5,      // payload = the high bits of every entry
+  SRC_SRV_RSPARSE = 6,   // payload = the survivors of every chunk and the chunk's draw
 };
 
 // Where v comes from.  Worker payload sub-arrays follow the documented payload layout.
@@ -45,6 +46,7 @@ struct SrcParams {
   uint32_t w_log2_chunk;   // worker chunk length (SIGN1, QSGD)
   float w_levels;          // worker QSGD level count as a float
   uint32_t w_clip_bits;    // worker CLIP: low bits that were set to zero (16 or 24)
+  uint32_t w_log2_keep;    // worker RSPARSE: log2 S (one entry in S survives)
   const float* acc;        // SRC_SRV_TOPK: dense accumulator [d] holding the sum of the sparse payloads
   int vec;                 // 1 if every row starts 16-byte aligned (d % 4 == 0)
 };
@@ -257,6 +259,26 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
             }
           }
         }
+      }
+    } else if constexpr (SRC == SRC_SRV_RSPARSE) {
+      // entry j of worker i survives iff (offset of j in its chunk) mod S equals the chunk's draw;
+      // its value sits in slot j / S
+      const uint32_t smask = (1u << p.w_log2_keep) - 1u;
+      for (uint32_t i = 0; i < p.n; ++i) {
+        const float* val = reinterpret_cast<const float*>(p.wp + (uint64_t)i * p.wp_stride + p.wp_off[0]);
+        const uint32_t* off = reinterpret_cast<const uint32_t*>(p.wp + (uint64_t)i * p.wp_stride + p.wp_off[1]);
+        float4 c[V];
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          c[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (!cnt[j]) continue;
+          const uint32_t o = __ldg(off + (e[j] >> p.w_log2_chunk));
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if ((uint32_t)k < cnt[j] && (((uint32_t)e[j] + k) & smask) == o) comp(c[j], k) = __ldg(val + ((e[j] + k) >> p.w_log2_keep));
+        }
+#pragma unroll
+        for (int j = 0; j < V; ++j) acc[j] = add4_rn(acc[j], c[j]);
       }
     } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc (cleared before every use)
 #pragma unroll

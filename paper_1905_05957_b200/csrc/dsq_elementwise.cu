@@ -51,6 +51,7 @@ cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64
     case SRC_SRV_TOPK: DSQ_ID(SRC_SRV_TOPK); break;
     case SRC_SRV_QSGD: DSQ_ID(SRC_SRV_QSGD); break;
     case SRC_SRV_CLIP: DSQ_ID(SRC_SRV_CLIP); break;
+    case SRC_SRV_RSPARSE: DSQ_ID(SRC_SRV_RSPARSE); break;
     default: return cudaErrorInvalidValue;
   }
 #undef DSQ_ID
@@ -120,6 +121,7 @@ static cudaError_t launch_clip_bits(int srck, const SrcParams& src, uint8_t* out
     case SRC_SRV_TOPK: DSQ_CL(SRC_SRV_TOPK); break;
     case SRC_SRV_QSGD: DSQ_CL(SRC_SRV_QSGD); break;
     case SRC_SRV_CLIP: DSQ_CL(SRC_SRV_CLIP); break;
+    case SRC_SRV_RSPARSE: DSQ_CL(SRC_SRV_RSPARSE); break;
     default: return cudaErrorInvalidValue;
   }
 #undef DSQ_CL
@@ -132,6 +134,76 @@ cudaError_t launch_clip(int srck, const SrcParams& src, uint32_t bits, uint8_t* 
   if (bits == 16) return launch_clip_bits<16>(srck, src, out_hi, hi_row_stride, delta_out, delta_row_stride, x, gamma, rows, st);
   if (bits == 24) return launch_clip_bits<24>(srck, src, out_hi, hi_row_stride, delta_out, delta_row_stride, x, gamma, rows, st);
   return cudaErrorInvalidValue;
+}
+
+// Q = randomised sparsification (Section 3.2): the entries of a chunk share one draw o in 0..S-1 and
+// the entry at offset t survives iff t mod S == o; survivors go to slot j / S of the payload.
+template <int SRC>
+__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : kServerCtasPerSm)
+k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_t delta_row_stride, float* x, float gamma) {
+  pdl_prologue();
+  const uint32_t row = blockIdx.y;
+  const uint64_t nq = (src.d + 3) / 4;
+  const uint32_t smask = (1u << rp.log2_keep) - 1u;
+  const float factor = rp.scaled ? (float)(1u << rp.log2_keep) : 1.0f;
+  float* val = rp.out_val + (uint64_t)row * rp.val_stride;
+  uint32_t* off = rp.out_off + (uint64_t)row * rp.off_stride;
+  // the loop bound is the same for all threads of the CTA: the source is read warp-cooperatively
+  for (uint64_t q0 = (uint64_t)blockIdx.x * kThreads; q0 < nq; q0 += (uint64_t)gridDim.x * kThreads) {
+    const uint64_t ee[1] = {(q0 + threadIdx.x) * 4};
+    const uint64_t e = ee[0];
+    const uint32_t cc[1] = {e < src.d ? (uint32_t)min((uint64_t)4, src.d - e) : 0u};
+    const uint32_t cnt = cc[0];
+    float4 vv[1];
+    src_load_tile<SRC, 1>(src, row, ee, cc, vv);
+    const float4 v = vv[0];
+    if (!cnt) continue;
+    const uint64_t c = e >> rp.log2_chunk;
+    const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c, rp.server_pass ? 0xFFFFFFFFu : row, rp.step), rp.keys);
+    const uint32_t o = rnd.x & smask;
+    if ((e & ((1ull << rp.log2_chunk) - 1ull)) == 0) off[c] = o;  // the chunk's first row records the draw
+    float4 C = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if ((uint32_t)k < cnt && (((uint32_t)e + k) & smask) == o) {
+        const float kept = __fmul_rn(factor, compc(v, k));
+        comp(C, k) = kept;
+        val[(e + k) >> rp.log2_keep] = kept;
+      }
+    }
+    // the group of S positions that holds the last entry: if its survivor lies past the end, its slot
+    // is sent as +0 (it may still hold a survivor of an earlier step)
+    if (e + cnt == src.d) {
+      const uint64_t group = (src.d - 1) >> rp.log2_keep;
+      if ((group << rp.log2_keep) + o >= src.d) val[group] = 0.f;
+    }
+    store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
+    if (x) {
+      float4 xv = load_row4(x, e, cnt, 1);
+      xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
+      xv.z = __fsub_rn(xv.z, __fmul_rn(gamma, C.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(gamma, C.w));
+      store_row4(x, e, cnt, 1, xv);
+    }
+  }
+}
+
+cudaError_t launch_rsparse(int srck, const SrcParams& src, const RsparseParams& rp, float* delta_out, uint64_t delta_row_stride,
+                           float* x, float gamma, uint32_t rows, cudaStream_t st) {
+  dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
+#define DSQ_RS(S) launch_pdl(k_rsparse<S>, grid, kThreads, st, src, rp, delta_out, delta_row_stride, x, gamma)
+  switch (srck) {
+    case SRC_WORKER: DSQ_RS(SRC_WORKER); break;
+    case SRC_SRV_IDENTITY: DSQ_RS(SRC_SRV_IDENTITY); break;
+    case SRC_SRV_SIGN1: DSQ_RS(SRC_SRV_SIGN1); break;
+    case SRC_SRV_TOPK: DSQ_RS(SRC_SRV_TOPK); break;
+    case SRC_SRV_QSGD: DSQ_RS(SRC_SRV_QSGD); break;
+    case SRC_SRV_CLIP: DSQ_RS(SRC_SRV_CLIP); break;
+    case SRC_SRV_RSPARSE: DSQ_RS(SRC_SRV_RSPARSE); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef DSQ_RS
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 // Dense decode of a server payload and update of x.
@@ -148,6 +220,13 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, 
       const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]) + (e >> 5)) >> (uint32_t)(e & 31);
       const float s = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
       C = make_float4(signed_by_bit(s, w, 0), signed_by_bit(s, w, 1), signed_by_bit(s, w, 2), signed_by_bit(s, w, 3));
+    } else if (pv.op == DS_Q_RSPARSE) {
+      const uint32_t o = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
+      const float* val = reinterpret_cast<const float*>(pv.base + pv.off[0]);
+      C = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if ((uint32_t)k < cnt && (((uint32_t)e + k) & ((1u << pv.log2_keep) - 1u)) == o) comp(C, k) = __ldg(val + ((e + k) >> pv.log2_keep));
     } else if (pv.op == DS_Q_CLIP) {
       uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll

@@ -58,6 +58,7 @@ struct PayloadView {
   uint32_t log2_chunk;
   float levels_f;
   uint32_t clip_bits;
+  uint32_t log2_keep;
   uint64_t k;
 };
 
@@ -116,6 +117,18 @@ cudaError_t launch_identity(int src_kind, const SrcParams& src, float* out_c, ui
 // Q = clipping: payload hi = bits(v) >> bits (16- or 8-bit entries), residual v - Q[v], optional fused update.
 cudaError_t launch_clip(int src_kind, const SrcParams& src, uint32_t bits, uint8_t* out_hi, uint64_t hi_row_stride,
                         float* delta_out, uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);
+
+// Q = randomised sparsification: one entry in 2^log2_keep of every chunk survives (see include/dsq.h).
+struct RsparseParams {
+  float* out_val;            // survivors, row stride val_stride (floats)
+  uint32_t* out_off;         // the draw of every chunk, row stride off_stride (words)
+  uint64_t val_stride, off_stride;
+  uint32_t log2_chunk, log2_keep, scaled;
+  PhiloxKeys keys;
+  uint32_t step, server_pass;
+};
+cudaError_t launch_rsparse(int src_kind, const SrcParams& src, const RsparseParams& rp, float* delta_out,
+                           uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);
 
 // x = x - gamma * decode(payload)
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);

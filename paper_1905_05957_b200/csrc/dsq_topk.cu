@@ -1233,6 +1233,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
       case SRC_SRV_TOPK: DSQ_P1(SRC_SRV_TOPK); break;
       case SRC_SRV_QSGD: DSQ_P1(SRC_SRV_QSGD); break;
       case SRC_SRV_CLIP: DSQ_P1(SRC_SRV_CLIP); break;
+      case SRC_SRV_RSPARSE: DSQ_P1(SRC_SRV_RSPARSE); break;
       default: return cudaErrorInvalidValue;
     }
 #undef DSQ_P1
@@ -1268,6 +1269,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
       case SRC_SRV_TOPK: DSQ_P1(SRC_SRV_TOPK); break;
       case SRC_SRV_QSGD: DSQ_P1(SRC_SRV_QSGD); break;
       case SRC_SRV_CLIP: DSQ_P1(SRC_SRV_CLIP); break;
+      case SRC_SRV_RSPARSE: DSQ_P1(SRC_SRV_RSPARSE); break;
       default: return cudaErrorInvalidValue;
     }
 #undef DSQ_P1

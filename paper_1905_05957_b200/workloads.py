@@ -38,11 +38,13 @@ assert len(RESNET18_SLICES) == 62 and sum(RESNET18_SLICES) == 11_689_512
 
 @dataclass(frozen=True)
 class Q:
-    op: str = "identity"     # identity | sign1 | topk | qsgd | clip
+    op: str = "identity"     # identity | sign1 | topk | qsgd | clip | rsparse
     chunk: int = 0
     k: int = 0
     levels: int = 0
     norm: int = 1            # sign1: scale from l1 (1) or l2 (2) magnitudes
+    keep_one_in: int = 0     # rsparse: S, an entry survives with probability 1/S
+    scaled: int = 0          # rsparse: 1 = survivors are multiplied by S (unbiased, no contraction)
     bits: int = 0            # clip: low bits of every number set to zero (16 or 24)
 
 
@@ -85,6 +87,9 @@ def _wl() -> dict[int, Workload]:
                     Q("sign1", chunk=4096, norm=2), Q("sign1", chunk=4096, norm=2)),
         # ... and with clipping of the low 16 bits (Section 3.2) on both passes
         7: Workload(7, "clip16_n8_resnet18", 8, 11_689_512, 20, "layered", Q("clip", bits=16), Q("clip", bits=16)),
+        # ... and with randomised sparsification (one entry in 32 survives, unscaled) on both passes
+        8: Workload(8, "rsparse32_n8_resnet18", 8, 11_689_512, 20, "layered",
+                    Q("rsparse", chunk=4096, keep_one_in=32), Q("rsparse", chunk=4096, keep_one_in=32)),
     }
 
 

@@ -10,7 +10,8 @@ REL_TOL = 1e-5   # bar for fp32 values, scales and delta (reduction order may di
 
 
 def to_oracle_q(q: Q) -> oracle.QSpec:
-    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels, norm=q.norm, bits=q.bits)
+    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels, norm=q.norm, bits=q.bits,
+                        keep_one_in=q.keep_one_in, scaled=q.scaled)
 
 
 def u32(t) -> np.ndarray:
@@ -56,6 +57,9 @@ def compare_payload(name: str, op: str, gpu_views: dict, ora: dict):
         assert_bits_match(f"{name}.lvl", u32(gpu_views["lvl"]), ora["lvl"])
         assert_bits_match(f"{name}.sgn", u32(gpu_views["sgn"]), ora["sgn"])
         assert_float_match(f"{name}.step", gpu_views["step"].cpu().numpy(), ora["step"])
+    elif op == "rsparse":
+        assert_bits_match(f"{name}.off", u32(gpu_views["off"]), ora["off"])
+        assert_bits_match(f"{name}.val", u32(gpu_views["val"].view(dtype=__import__("torch").int32)), ora["val"].view(np.uint32))
     elif op == "clip":
         assert_bits_match(f"{name}.hi", u32(gpu_views["hi"]), ora["hi"])
     else:

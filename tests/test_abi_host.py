@@ -55,6 +55,9 @@ def test_layouts(lib):
     c16, c24 = b.get_layout(cfg, 0), b.get_layout(cfg, 1)
     assert c16.count[0] == 1001 and c16.stride == (2 * 1001 + 15) // 16 * 16
     assert c24.count[0] == 1001 and c24.stride == (1001 + 15) // 16 * 16
+    cfg = b.make_config(2, 10_000, 0.1, Q("rsparse", chunk=4096, keep_one_in=32), Q("identity"), 1)
+    rs = b.get_layout(cfg, 0)
+    assert list(rs.count)[:2] == [3 * 128, 3] and rs.off[1] == 3 * 128 * 4
     # the l2-magnitude variant of the 1-bit operator shares the payload format
     a = b.get_layout(b.make_config(2, 5000, 0.1, Q("sign1", chunk=128), Q("identity"), 1), 0)
     l2 = b.get_layout(b.make_config(2, 5000, 0.1, Q("sign1", chunk=128, norm=2), Q("identity"), 1), 0)
@@ -80,6 +83,8 @@ def test_query_mode_reports_sizes(lib):
     dict(worker_q=Q("topk", k=1001)),
     dict(worker_q=Q("sign1", chunk=4096, norm=3)), dict(server_q=Q("clip", bits=12)), dict(server_q=Q("clip", bits=0)),
     dict(worker_q=Q("clip", bits=32)),
+    dict(worker_q=Q("rsparse", chunk=4096, keep_one_in=3)), dict(server_q=Q("rsparse", chunk=4096, keep_one_in=256)),
+    dict(server_q=Q("rsparse", chunk=100, keep_one_in=4)), dict(worker_q=Q("rsparse", chunk=4096, keep_one_in=4, scaled=2)),
 ])
 def test_bad_configs_are_rejected(lib, kw):
     args = dict(n=4, d=1000, gamma=0.1, worker_q=Q("identity"), server_q=Q("identity"), seed=0)

@@ -12,7 +12,7 @@ from tests.helpers import compare_state, to_oracle_q
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_full_size_step_matches_oracle(wid):
     wl = WORKLOADS[wid]
     need = 4 * wl.n * wl.d * 4 + (2 << 30)

@@ -15,6 +15,7 @@ QSGD = lambda L=2048, s=255: Q("qsgd", chunk=L, levels=s)
 TOPK = lambda k: Q("topk", k=k)
 IDENT = Q("identity")
 CLIP = lambda b=16: Q("clip", bits=b)
+RSP = lambda S=4, L=4096, scaled=0: Q("rsparse", chunk=L, keep_one_in=S, scaled=scaled)
 
 
 def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None, scribble=False):
@@ -94,6 +95,23 @@ def test_clip_mixed_with_other_operators_unaligned_rows_and_unfused_update():
     run_lockstep(3, 30_000, CLIP(16), CLIP(16), randn_steps(3, 30_000, 3, seed=44), fuse=False)
     run_lockstep(3, 30_001, CLIP(24), CLIP(24), randn_steps(3, 30_001, 2, seed=45), fuse=False)
     run_lockstep(37, 9000, CLIP(16), CLIP(16), randn_steps(37, 9000, 2, seed=46))
+
+
+@pytest.mark.parametrize("d", [4096, 10_000, 65_536 + 4 * 37, 33, 5, 1])
+@pytest.mark.parametrize("S,L,scaled", [(4, 4096, 0), (2, 128, 0), (32, 4096, 0), (128, 1024, 0), (4, 512, 1), (8, 8192, 1)])
+def test_rsparse_both_passes(d, S, L, scaled):
+    run_lockstep(3, d, RSP(S, L, scaled), RSP(S, L, scaled), randn_steps(3, d, 4, seed=d + S + L))
+
+
+def test_rsparse_mixed_with_other_operators_unaligned_rows_and_unfused_update():
+    d = 50_000 + 13
+    for wq, sq in [(RSP(8), TOPK(500)), (RSP(4, 256), SIGN(2048)), (QSGD(1024, 31), RSP(16)), (TOPK(700), RSP(2, 128)),
+                   (RSP(32), QSGD(2048)), (SIGN(4096), RSP(4)), (IDENT, RSP(8, 512)), (RSP(4), IDENT), (RSP(4), CLIP(16)),
+                   (CLIP(24), RSP(8, 1024, 1))]:
+        run_lockstep(5, d, wq, sq, randn_steps(5, d, 3, seed=47))
+    run_lockstep(3, 30_000, RSP(4), RSP(4), randn_steps(3, 30_000, 3, seed=48), fuse=False)
+    run_lockstep(3, 30_001, RSP(8, 256), RSP(8, 256), randn_steps(3, 30_001, 3, seed=49), fuse=False)
+    run_lockstep(37, 9000, RSP(4, 128), RSP(4, 128), randn_steps(37, 9000, 2, seed=50))
 
 
 def test_identity_is_parallel_sgd():
@@ -187,7 +205,7 @@ def test_many_workers_and_one_worker():
 
 # ------------------------------------------------------------------ the five workloads, scaled down
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_workload_recipes_scaled(wid):
     wl = WORKLOADS[wid]
     wl = wl if wid == 1 else wl.scaled(d=200_000 + 40, n=min(wl.n, 8), steps=4)
@@ -195,7 +213,7 @@ def test_workload_recipes_scaled(wid):
     run_lockstep(wl.n, wl.d, wl.worker_q, wl.server_q, gs, gamma=wl.gamma, seed=wl.seed)
 
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_telescoping_identity_free_running_on_the_gpu(wid):
     """Eq. 5-6 on the GPU alone, with no oracle in the loop: after T steps of any Q,
     x_T - gamma (delta_T + mean_i delta_T^(i)) = x_0 - gamma sum_t mean_i g_t^(i), up to fp32 rounding."""
@@ -293,7 +311,9 @@ def test_more_workers_than_one_batch_of_the_server_loops():
 # ------------------------------------------------------------------ seeded random configurations
 
 def _random_q(r, d):
-    kind = r.choice(["sign1", "sign1_l2", "qsgd", "topk", "clip", "identity"])
+    kind = r.choice(["sign1", "sign1_l2", "qsgd", "topk", "clip", "identity", "rsparse"])
+    if kind == "rsparse":
+        return RSP(int(r.choice([2, 4, 16, 64])), int(r.choice([128, 1024, 4096])), int(r.integers(0, 2)))
     if kind == "sign1":
         return SIGN(int(r.choice([128, 256, 512, 1024, 2048, 4096, 8192])))
     if kind == "sign1_l2":
