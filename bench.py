@@ -32,11 +32,12 @@ FALLBACK_HBM_GBS = 6650.0
 # captures summarised under profiles/; valid only for the kernel sources with this digest.
 NCU_TRAFFIC = {
     # workload id: (kernel, bytes per launch, digest of the kernel's source files at capture time)
-    2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748168448 + 333265152, "eb1f2dcf6abb2c1e"),
+    2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748169472 + 332183040, "5be2583994dd727b"),
     # captured on the same recipe at d = 2^24 (a multi-pass capture must stay small) and scaled by
     # the entries one launch processes: traffic of a streaming kernel grows in proportion
-    4: ("k_chunked<QSGD, WORKER, 2, 256>", int((1073774000 + 630327552) * (8 * 124_439_808) / (8 * 16_777_216)), "eb1f2dcf6abb2c1e"),
-    7: ("k_clip<WORKER, 16>", 748315136 + 508957696, "2936cbf6ee56b3f1"),
+    4: ("k_chunked<QSGD, WORKER, 2, 256>", int((1073773000 + 629989632) * (8 * 124_439_808) / (8 * 16_777_216)), "5be2583994dd727b"),
+    7: ("k_clip<WORKER, 16>", 748325376 + 508748800, "8936b8b285292618"),
+    8: ("k_rsparse<WORKER>", 748242176 + 331810048, "8936b8b285292618"),
 }
 KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "sign1": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),

@@ -262,23 +262,36 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
       }
     } else if constexpr (SRC == SRC_SRV_RSPARSE) {
       // entry j of worker i survives iff (offset of j in its chunk) mod S equals the chunk's draw;
-      // its value sits in slot j / S
+      // its value sits in slot j / S.  Four workers at a time: their draws are fetched together,
+      // then their survivors, then they are added in worker order.
       const uint32_t smask = (1u << p.w_log2_keep) - 1u;
-      for (uint32_t i = 0; i < p.n; ++i) {
-        const float* val = reinterpret_cast<const float*>(p.wp + (uint64_t)i * p.wp_stride + p.wp_off[0]);
-        const uint32_t* off = reinterpret_cast<const uint32_t*>(p.wp + (uint64_t)i * p.wp_stride + p.wp_off[1]);
-        float4 c[V];
+      for (uint32_t i0 = 0; i0 < p.n; i0 += 4) {
+        uint32_t o[V][4];
+        float4 c[V][4];
 #pragma unroll
-        for (int j = 0; j < V; ++j) {
-          c[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (!cnt[j]) continue;
-          const uint32_t o = __ldg(off + (e[j] >> p.w_log2_chunk));
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t* off = reinterpret_cast<const uint32_t*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[1]);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            if ((uint32_t)k < cnt[j] && (((uint32_t)e[j] + k) & smask) == o) comp(c[j], k) = __ldg(val + ((e[j] + k) >> p.w_log2_keep));
+          for (int j = 0; j < V; ++j) o[j][u] = (i0 + u < p.n && cnt[j]) ? __ldg(off + (e[j] >> p.w_log2_chunk)) : 0xFFFFFFFFu;
         }
 #pragma unroll
-        for (int j = 0; j < V; ++j) acc[j] = add4_rn(acc[j], c[j]);
+        for (int u = 0; u < 4; ++u) {
+          const float* val = reinterpret_cast<const float*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[0]);
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            c[j][u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if ((uint32_t)k < cnt[j] && (((uint32_t)e[j] + k) & smask) == o[j][u])   // never true for the filler 0xFFFFFFFF
+                comp(c[j][u], k) = __ldg(val + ((e[j] + k) >> p.w_log2_keep));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (i0 + u < p.n) {
+#pragma unroll
+            for (int j = 0; j < V; ++j) acc[j] = add4_rn(acc[j], c[j][u]);
+          }
       }
     } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc (cleared before every use)
 #pragma unroll

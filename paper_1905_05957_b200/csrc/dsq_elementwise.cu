@@ -136,6 +136,17 @@ cudaError_t launch_clip(int srck, const SrcParams& src, uint32_t bits, uint8_t* 
   return cudaErrorInvalidValue;
 }
 
+// The draw of every chunk of every vector of a pass, straight into the payload: o = first Philox word
+// of counter (0xFFFFFFFF, chunk, worker or 0xFFFFFFFF on the server pass, step), mod S.
+__global__ void __launch_bounds__(kThreads) k_rsparse_draw(const RsparseParams rp, uint64_t nc) {
+  pdl_prologue();
+  const uint32_t row = blockIdx.y;
+  const uint64_t c = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (c >= nc) return;
+  const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c, rp.server_pass ? 0xFFFFFFFFu : row, rp.step), rp.keys);
+  rp.out_off[(uint64_t)row * rp.off_stride + c] = rnd.x & ((1u << rp.log2_keep) - 1u);
+}
+
 // Q = randomised sparsification (Section 3.2): the entries of a chunk share one draw o in 0..S-1 and
 // the entry at offset t survives iff t mod S == o; survivors go to slot j / S of the payload.
 template <int SRC>
@@ -147,7 +158,7 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
   const uint32_t smask = (1u << rp.log2_keep) - 1u;
   const float factor = rp.scaled ? (float)(1u << rp.log2_keep) : 1.0f;
   float* val = rp.out_val + (uint64_t)row * rp.val_stride;
-  uint32_t* off = rp.out_off + (uint64_t)row * rp.off_stride;
+  const uint32_t* off = rp.out_off + (uint64_t)row * rp.off_stride;
   // the loop bound is the same for all threads of the CTA: the source is read warp-cooperatively
   for (uint64_t q0 = (uint64_t)blockIdx.x * kThreads; q0 < nq; q0 += (uint64_t)gridDim.x * kThreads) {
     const uint64_t ee[1] = {(q0 + threadIdx.x) * 4};
@@ -158,10 +169,7 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
     src_load_tile<SRC, 1>(src, row, ee, cc, vv);
     const float4 v = vv[0];
     if (!cnt) continue;
-    const uint64_t c = e >> rp.log2_chunk;
-    const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c, rp.server_pass ? 0xFFFFFFFFu : row, rp.step), rp.keys);
-    const uint32_t o = rnd.x & smask;
-    if ((e & ((1ull << rp.log2_chunk) - 1ull)) == 0) off[c] = o;  // the chunk's first row records the draw
+    const uint32_t o = __ldg(off + (e >> rp.log2_chunk));  // the chunk's draw, made by k_rsparse_draw
     float4 C = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -189,6 +197,9 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
 
 cudaError_t launch_rsparse(int srck, const SrcParams& src, const RsparseParams& rp, float* delta_out, uint64_t delta_row_stride,
                            float* x, float gamma, uint32_t rows, cudaStream_t st) {
+  const uint64_t nc = (src.d + (1ull << rp.log2_chunk) - 1) >> rp.log2_chunk;
+  launch_pdl(k_rsparse_draw, dim3((unsigned)((nc + kThreads - 1) / kThreads), rows, 1), kThreads, st, rp, nc);
+  count_launches(1);
   dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
 #define DSQ_RS(S) launch_pdl(k_rsparse<S>, grid, kThreads, st, src, rp, delta_out, delta_row_stride, x, gamma)
   switch (srck) {
