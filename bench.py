@@ -1,18 +1,29 @@
 #!/usr/bin/env python
 """Benchmark of the DoubleSqueeze step (worker pass + server pass with fused model update).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..8] [--impl ours|reference]
 
 One "step" is one whole iteration of Algorithm 1 over one batch of synthetic gradients
 (ds_worker_compress + ds_server_aggregate_compress with the fused update).  Prints ONE JSON line.
+
+Without --workload the five listed configurations are all measured in one run; the headline keys
+(value, ms_per_step, roofline, e2e, cpu_baseline, config) are those of the largest one, workload 5
+(32 workers x 60 M entries, 1-bit workers, top-k server with the paper's k = 300000), and
+"per_workload" carries the record of each.  With --workload N only that one is run.
+
+A workload is timed in blocks of K steps (CUDA events on the launching stream); blocks are repeated
+until at least --min-seconds of GPU time are in, and the median block gives the headline, the
+spread over blocks and over steps is reported beside it.
+
 For N > 1 (launched by torch.distributed.run) every rank steps an independent replica of the same
-workload on its own GPU -- the path has no exchange between GPUs -- and the value is the aggregate.
+workloads on its own GPU -- the path has no exchange between GPUs -- and the value is the aggregate.
 """
 from __future__ import annotations
 
 import argparse
 import hashlib
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -27,17 +38,21 @@ if ROOT not in sys.path:
 METRIC = "doublesqueeze_step_gradient_elements_per_s"
 UNIT = "elements/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+LISTED = (1, 2, 3, 4, 5)     # the five listed configurations
+HEADLINE = 5                 # the largest one that fits one GPU
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/; valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {
-    # workload id: (kernel, bytes per launch, digest of the kernel's source files at capture time)
-    2: ("k_chunked<SIGN1, WORKER, 4, 256>", 748169472 + 332183040, "5be2583994dd727b"),
-    # captured on the same recipe at d = 2^24 (a multi-pass capture must stay small) and scaled by
-    # the entries one launch processes: traffic of a streaming kernel grows in proportion
-    4: ("k_chunked<QSGD, WORKER, 2, 256>", int((1073773000 + 629989632) * (8 * 124_439_808) / (8 * 16_777_216)), "5be2583994dd727b"),
-    7: ("k_clip<WORKER, 16>", 748325376 + 508748800, "8936b8b285292618"),
-    8: ("k_rsparse<WORKER>", 748242176 + 331810048, "8936b8b285292618"),
+# (kernel, bytes in the captured launch, gradient entries the captured launch processed, digest of
+# the kernel's source files at capture time).  A capture taken at a smaller size than the workload
+# (a multi-pass capture must stay small) is scaled by the entries one launch processes: the
+# traffic of a streaming kernel grows in proportion.
+NCU_CAPTURES = {
+    "sign1": ("k_chunked<SIGN1, WORKER, 4, 256>", 748169472 + 332183040, 8 * 11_689_512, "5be2583994dd727b"),
+    "qsgd": ("k_chunked<QSGD, WORKER, 2, 256>", 1073773000 + 629989632, 8 * 16_777_216, "5be2583994dd727b"),
+    "clip": ("k_clip<WORKER, 16>", 748325376 + 508748800, 8 * 11_689_512, "8936b8b285292618"),
+    "rsparse": ("k_rsparse<WORKER>", 748242176 + 331810048, 8 * 11_689_512, "8936b8b285292618"),
 }
 KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "sign1": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
@@ -47,6 +62,9 @@ KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "clip": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
     "rsparse": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
 }
+DOMINANT = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
+            "topk": "top-k worker pass (k_topk_pass1<WORKER> and the selection tail)",
+            "identity": "k_identity<WORKER>", "clip": "k_clip<WORKER>", "rsparse": "k_rsparse<WORKER>"}
 
 
 def payload_bytes(q, d: int) -> int:
@@ -85,12 +103,26 @@ def csrc_digest(op: str) -> str:
     return h.hexdigest()[:16]
 
 
+def captured_traffic(wl):
+    """DRAM bytes per launch of the workload's dominant kernel from the committed capture, scaled to
+    this launch's entries; None without a capture or once the kernel's sources have changed."""
+    cap = NCU_CAPTURES.get(wl.worker_q.op)
+    if cap is None or cap[3] != csrc_digest(wl.worker_q.op):
+        return None
+    return int(cap[1] * (wl.n * wl.d) / cap[2])
+
+
 def measured_peak() -> tuple[float, str]:
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         return float(json.load(open(p))["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def pct(xs, q: float) -> float:
+    s = sorted(xs)
+    return s[int(q * (len(s) - 1))]
 
 
 class ClockSampler:
@@ -114,6 +146,13 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
+
+    def wait_first(self, seconds: float = 3.0):
+        """The first answer takes a moment; what came before the load is dropped."""
+        t_wait = time.time() + seconds
+        while self.proc is not None and not self.lines and time.time() < t_wait:
+            time.sleep(0.05)
+        self.lines.clear()
 
     def stop(self) -> dict:
         if self.proc is None:
@@ -145,27 +184,31 @@ class ClockSampler:
 # reference arm and CPU baseline: the oracle, as it stands, on the host cores
 # ---------------------------------------------------------------------------------------------
 
-def oracle_sample_workload(wl):
-    """A bounded sample of the workload for the CPU oracle: same recipe, n workers, d cut so that
-    one step is a few seconds of single-thread work (the oracle runs ~30-80 M entries/s; top-k
-    sorts every vector)."""
-    budget = 120_000_000 if wl.worker_q.op != "topk" else 24_000_000
-    if wl.n * wl.d <= budget:
+# rough single-thread cost of the oracle per vector entry (seconds), used only to size the sample
+ORACLE_COST = {"identity": 0.6e-8, "sign1": 1.2e-8, "qsgd": 3.0e-8, "topk": 1.3e-7, "clip": 0.8e-8, "rsparse": 0.8e-8,
+               "ternary": 3.0e-8}
+
+
+def oracle_sample_workload(wl, seconds_per_step: float):
+    """A bounded sample of the workload for the CPU oracle: same recipe and n workers, d cut so that
+    one step is about `seconds_per_step` of single-thread work."""
+    per_d = wl.n * (ORACLE_COST.get(wl.worker_q.op, 3e-8) + 1.0e-8) + ORACLE_COST.get(wl.server_q.op, 3e-8) + 1.0e-8
+    d = int(seconds_per_step / per_d)
+    if d >= wl.d:
         return wl, "full workload"
-    d = max(8192, (budget // wl.n) // 8192 * 8192)
+    d = max(8192, d // 8192 * 8192)
     return wl.scaled(d=d), f"same recipe with d cut to {d} (n={wl.n})"
 
 
-def time_oracle(wl, steps: int, warmup: int) -> dict:
+def time_oracle(wl, steps: int, warmup: int, seconds_per_step: float) -> dict:
     import numpy as np
 
     import oracle
     from paper_1905_05957_b200.workloads import make_gradients
-    from tests.helpers import to_oracle_q
 
-    swl, what = oracle_sample_workload(wl)
+    swl, what = oracle_sample_workload(wl, seconds_per_step)
     st = oracle.State.zeros(swl.n, swl.d)
-    wq, sq = to_oracle_q(swl.worker_q), to_oracle_q(swl.server_q)
+    wq, sq = oracle.qspec_from(swl.worker_q), oracle.qspec_from(swl.server_q)
     gs = [make_gradients(swl, t, device="cpu").numpy() for t in range(2)]
     for t in range(warmup):
         oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, t)
@@ -179,11 +222,15 @@ def time_oracle(wl, steps: int, warmup: int) -> dict:
 
 
 def run_reference(args, wl):
+    """The reference arm: the oracle, as it stands, for exactly --steps timed steps after --warmup
+    untimed ones; the sample of the workload is sized so that the whole run takes about two and a
+    half minutes whatever K and W are."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    steps, warmup = max(1, min(args.steps, 5)), min(args.warmup, 1)
-    r = time_oracle(wl, steps, warmup)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    per_step = min(5.0, 150.0 / (steps + warmup))
+    r = time_oracle(wl, steps, warmup, per_step)
     line = {
         "impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
@@ -212,25 +259,35 @@ def workload_config(wl) -> dict:
 # our arm
 # ---------------------------------------------------------------------------------------------
 
-def run_ours(args, wl):
-    import torch
-    import torch.distributed as dist
+class Env:
+    def __init__(self):
+        import torch
+        import torch.distributed as dist
+        self.torch, self.dist = torch, dist
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if self.world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            dist.init_process_group("nccl")
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
 
-    from paper_1905_05957_b200 import DoubleSqueeze, load_library
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize(self.dev)
+
+
+def measure_workload(env: Env, wl, args, lib, want_e2e: bool) -> dict:
+    """Times one workload on this rank's GPU; rank 0 gets the record."""
+    torch = env.torch
+    from paper_1905_05957_b200 import DoubleSqueeze
     from paper_1905_05957_b200.replicas import aggregate_throughput, max_over_ranks
     from paper_1905_05957_b200.workloads import make_gradients
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    lib = load_library()          # raises if the CUDA library is missing: there is no other path
+    dev, world, rank = env.dev, env.world, env.rank
     K, W = args.steps, max(args.warmup, 3)
-
     ds = DoubleSqueeze.for_workload(wl, dev)
     # distinct g_t resident in HBM: a fresh draw for every step where 48 GB hold them, else a ring of
     # as many as fit (a training run never sees the same gradient twice; a short ring makes the
@@ -240,60 +297,70 @@ def run_ours(args, wl):
     need_flush = wl.n * wl.d * 8 <= 2 * 126e6
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
     stream = torch.cuda.current_stream(dev)
+    E = lambda: torch.cuda.Event(enable_timing=True)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
-    # ---- device-resident timing
-    for t in range(W):
-        ds.step(ring[t % R], t)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    sampler = ClockSampler(local)
-    barrier()
+    step_no = 0
+    for _ in range(W):
+        ds.step(ring[step_no % R], step_no)
+        step_no += 1
+    sampler = ClockSampler(env.local)
+    env.barrier()
     if rank == 0:
         sampler.start()
-        t_wait = time.time() + 3.0
-        while not sampler.lines and time.time() < t_wait:   # the first answer takes a moment
-            time.sleep(0.05)
-        sampler.lines.clear()                               # samples of the idle GPU are dropped
+        sampler.wait_first()
     launches0 = lib.ds_kernel_launches()
-    t_total = 0.0
-    barrier()
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if not need_flush:
+
+    def timed_block():
+        """EXACTLY K steps between a barrier + synchronize on both sides; returns the block's events."""
+        nonlocal step_no
+        ev = [[E() for _ in range(3)] for _ in range(K)]
+        start, stop = E(), E()
+        env.barrier()
         start.record(stream)
-    for t in range(K):
-        if need_flush:
-            flush.fill_(t & 0xFF)
-        ev[t][0].record(stream)
-        ds.worker_compress(ring[(W + t) % R], W + t)
-        ev[t][1].record(stream)
-        ds.server_aggregate_compress(W + t, fuse_apply=True)
-        ev[t][2].record(stream)
-    if not need_flush:
+        for t in range(K):
+            if need_flush:
+                flush.fill_(t & 0xFF)
+            ev[t][0].record(stream)
+            ds.worker_compress(ring[step_no % R], step_no)
+            ev[t][1].record(stream)
+            ds.server_aggregate_compress(step_no, fuse_apply=True)
+            ev[t][2].record(stream)
+            step_no += 1
         stop.record(stream)
-    barrier()
+        env.barrier()
+        steps = [(e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])) for e in ev]
+        # the flush writes are not part of a step: with them the block is the sum of its steps
+        total = sum(a + b for a, b in steps) if need_flush else start.elapsed_time(stop)
+        return total, steps
+
+    blocks, steps_all = [], []
+    total, steps = timed_block()
+    blocks.append(total)
+    steps_all += steps
+    # repeat the block until enough GPU time is in (every rank takes the same count)
+    (slowest,) = max_over_ranks([total], device=dev)
+    more = min(args.max_blocks, math.ceil(args.min_seconds * 1e3 / max(slowest, 1e-3))) - 1
+    for _ in range(max(0, more)):
+        total, steps = timed_block()
+        blocks.append(total)
+        steps_all += steps
     launches = lib.ds_kernel_launches() - launches0
-    # nvidia-smi answers every 100 ms and a short timed region may end before its first answer: keep
-    # the same steps running, untimed, until a few samples under this load are in
+    # nvidia-smi answers every 100 ms: keep the same steps running, untimed, until a few samples under
+    # this load are in
     t_end = time.time() + 1.2
     extra = 0
     while time.time() < t_end and (rank != 0 or len(sampler.lines) < 8):
-        ds.step(ring[extra % R], W + K + extra)
+        ds.step(ring[step_no % R], step_no)
+        step_no += 1
         extra += 1
         if extra % 16 == 0:
             torch.cuda.synchronize(dev)
     torch.cuda.synchronize(dev)
     clocks = sampler.stop() if rank == 0 else None
     if clocks is not None:
-        clocks["sampled"] = "during the timed steps and the same steps repeated untimed right after them"
-    worker_ms = [ev[t][0].elapsed_time(ev[t][1]) for t in range(K)]
-    server_ms = [ev[t][1].elapsed_time(ev[t][2]) for t in range(K)]
-    step_ms = [ev[t][0].elapsed_time(ev[t][2]) for t in range(K)]
-    t_total = sum(step_ms) if need_flush else start.elapsed_time(stop)   # flush writes are not part of the step
+        clocks["sampled"] = "during the timed blocks" + (" and the same steps repeated untimed right after them" if extra else "")
     status = ds.device_status()
+    routes = ds.topk_routes()
 
     # ---- launch-bound workloads: the same step replayed from a CUDA graph (one graph per ring slot)
     graph_ms = None
@@ -306,84 +373,127 @@ def run_ours(args, wl):
                     ds.step(ring[slot], 0)
                 graphs.append(gr)
             stream = torch.cuda.current_stream(dev)
-            gev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+            gev = [[E() for _ in range(2)] for _ in range(K)]
             for t in range(3):
                 graphs[t % 2].replay()
-            barrier()
+            env.barrier()
             for t in range(K):
                 flush.fill_(t & 0xFF)
                 gev[t][0].record(stream)
                 graphs[t % 2].replay()
                 gev[t][1].record(stream)
-            barrier()
+            env.barrier()
             graph_ms = statistics.median(gev[t][0].elapsed_time(gev[t][1]) for t in range(K))
         except Exception as exc:  # the number is an extra; the run does not depend on it
             graph_ms = f"unavailable: {type(exc).__name__}"
 
     # ---- end to end: pinned host g -> device, fused step, server payload -> host, every step
-    g_host = [torch.empty(wl.n, wl.d, dtype=torch.float32, pin_memory=True) for _ in range(2)]
-    for a, b in zip(g_host, ring):
-        a.copy_(b)
-    out_host = torch.empty(ds.server_payload.numel(), dtype=torch.uint8, pin_memory=True)
-    Ke = max(1, min(K, 10))
-    for t in range(2):
-        ds.step_host(g_host[t % 2], ring[0], 10_000 + t, server_payload_host=out_host)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for t in range(Ke):
-        ds.step_host(g_host[t % 2], ring[0], 20_000 + t, server_payload_host=out_host)
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
+    e2e = None
+    if want_e2e:
+        big = wl.n * wl.d * 4 > 4e9     # pinning several GB takes seconds: one host buffer is enough there
+        g_host = [torch.empty(wl.n, wl.d, dtype=torch.float32, pin_memory=True) for _ in range(1 if big else 2)]
+        for a, b in zip(g_host, ring):
+            a.copy_(b)
+        out_host = torch.empty(ds.server_payload.numel(), dtype=torch.uint8, pin_memory=True)
+        Ke = max(1, min(K, 10))
+        for t in range(2):
+            ds.step_host(g_host[t % len(g_host)], ring[0], 10_000_000 + t, server_payload_host=out_host)
+        env.barrier()
+        e0, e1 = E(), E()
+        e0.record(stream)
+        for t in range(Ke):
+            ds.step_host(g_host[t % len(g_host)], ring[0], 20_000_000 + t, server_payload_host=out_host)
+        e1.record(stream)
+        env.barrier()
+        (e2e_ms,) = max_over_ranks([e0.elapsed_time(e1)], device=dev)
+        e2e = {"value": aggregate_throughput(wl.n * wl.d, Ke, e2e_ms, world), "unit": UNIT,
+               "h2d_bytes_per_step": wl.n * wl.d * 4, "d2h_bytes_per_step": int(ds.server_payload.numel()), "steps": Ke}
+        del g_host, out_host
 
-    t_total, e2e_ms = max_over_ranks([t_total, e2e_ms], device=dev)
-
-    if rank == 0:
-        ab = algorithmic_bytes(wl)
-        peak, peak_kind = measured_peak()
-        wk_ms = statistics.mean(worker_ms)
-        achieved = ab["worker"] / (wk_ms * 1e-3) / 1e9
-        digest = csrc_digest(wl.worker_q.op)
-        traffic = None
-        if wl.wid in NCU_TRAFFIC and NCU_TRAFFIC[wl.wid][2] == digest:
-            traffic = NCU_TRAFFIC[wl.wid][1]
-        dominant = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
-                    "topk": "top-k worker pass (pass1, mark, refine, finalize, emit)",
-                    "identity": "k_identity<WORKER>", "clip": "k_clip<WORKER>",
-                    "rsparse": "k_rsparse<WORKER>"}[wl.worker_q.op]
-        line = {
-            "metric": METRIC, "value": aggregate_throughput(wl.n * wl.d, K, t_total, world), "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": W, "ms_per_step": t_total / K, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl),
-            "clocks": clocks,
-            "e2e": {"value": aggregate_throughput(wl.n * wl.d, Ke, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": wl.n * wl.d * 4,
-                    "d2h_bytes_per_step": int(ds.server_payload.numel()), "steps": Ke},
-            "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": traffic,
-                         "algorithmic_bytes_per_launch": ab["worker"], "ms_per_launch": wk_ms},
-            "step_breakdown": {
-                "worker_ms": wk_ms, "server_ms": statistics.mean(server_ms),
-                "step_ms_median": statistics.median(step_ms), "step_ms_p10": sorted(step_ms)[int(0.1 * (K - 1))],
-                "step_ms_p90": sorted(step_ms)[int(0.9 * (K - 1))],
-                "algorithmic_gb_per_step": ab["total"] / 1e9,
-                "step_gbs": ab["total"] / (statistics.median(step_ms) * 1e-3) / 1e9,
-                "step_frac_of_peak": ab["total"] / (statistics.median(step_ms) * 1e-3) / 1e9 / peak,
-                "step_frac_of_nominal_8000": ab["total"] / (statistics.median(step_ms) * 1e-3) / 1e9 / 8000.0,
-                "server_gbs": ab["server"] / (statistics.mean(server_ms) * 1e-3) / 1e9,
-                "cuda_graph_step_ms_median": graph_ms,
-            },
-            "device_status": status,
-        }
-        if args.dump_steps:
-            line["step_ms_all"] = [round(x, 4) for x in step_ms]
-        if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = {k: v for k, v in time_oracle(wl, args.cpu_steps, 0).items() if k != "ms_per_step"}
-        print(json.dumps(line), flush=True)
+    block_med = statistics.median(blocks)
+    (block_med_slowest,) = max_over_ranks([block_med], device=dev)
     ds.close()
-    if world > 1:
-        dist.destroy_process_group()
+    del ds, ring, flush
+    torch.cuda.empty_cache()
+    if rank != 0:
+        return {}
+
+    ab = algorithmic_bytes(wl)
+    peak, peak_kind = measured_peak()
+    worker_ms = [a for a, _ in steps_all]
+    server_ms = [b for _, b in steps_all]
+    step_ms = [a + b for a, b in steps_all]
+    wk_ms = statistics.mean(worker_ms)
+    achieved = ab["worker"] / (wk_ms * 1e-3) / 1e9
+    traffic = captured_traffic(wl)
+    ms_per_step = block_med_slowest / K
+    step_gbs = ab["total"] / (ms_per_step * 1e-3) / 1e9
+    roof = {"bound": "hbm", "kernel": DOMINANT[wl.worker_q.op], "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": traffic,
+            "algorithmic_bytes_per_launch": ab["worker"], "ms_per_launch": wk_ms,
+            "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+            "dram_gbs_from_traffic": None if traffic is None else traffic / (wk_ms * 1e-3) / 1e9}
+    if roof["frac"] > 1.0:
+        roof["note"] = ("above 1: the peak is a plain device copy (read + write), not a hardware bound; this kernel reads "
+                        "two bytes for every byte it writes, and reads run faster than writes")
+    rec = {
+        "workload": wl.name, "wid": wl.wid, "n_workers": wl.n, "d": wl.d,
+        "ms_per_step": ms_per_step, "value": aggregate_throughput(wl.n * wl.d, K, block_med_slowest, world),
+        "blocks": len(blocks), "steps_per_block": K, "gpu_seconds_timed": sum(blocks) * 1e-3,
+        "block_ms_per_step": {"median": block_med / K, "p10": pct(blocks, 0.1) / K, "p90": pct(blocks, 0.9) / K},
+        "step_ms": {"median": statistics.median(step_ms), "p10": pct(step_ms, 0.1), "p90": pct(step_ms, 0.9)},
+        "worker_ms": wk_ms, "server_ms": statistics.mean(server_ms),
+        "algorithmic_bytes": ab, "step_gbs": step_gbs,
+        "step_frac_of_measured": step_gbs / peak, "step_frac_of_nominal_8000": step_gbs / NOMINAL_HBM_GBS,
+        "server_gbs": ab["server"] / (statistics.mean(server_ms) * 1e-3) / 1e9,
+        "roofline": roof, "clocks": clocks,
+        "ms_per_step_x_sm_mhz": None if not clocks or not clocks.get("sm_mhz") else ms_per_step * clocks["sm_mhz"],
+        "device_status": status, "gpu_launches": int(launches),
+        "topk_routes": {"predicted": routes[0], "full": routes[1]},
+    }
+    if need_flush:
+        rec["note"] = "launch-bound (a few MB per step): reported, not graded as a fraction of HBM bandwidth"
+        rec["cuda_graph_step_ms_median"] = graph_ms
+    if e2e is not None:
+        rec["e2e"] = e2e
+    if args.dump_steps:
+        rec["step_ms_all"] = [round(x, 4) for x in step_ms]
+    return rec
+
+
+def run_ours(args, wids, headline):
+    from paper_1905_05957_b200 import load_library
+    from paper_1905_05957_b200.workloads import WORKLOADS
+
+    env = Env()
+    lib = load_library()          # raises if the CUDA library is missing: there is no other path
+    recs = {}
+    for wid in wids:
+        wl = WORKLOADS[wid]
+        if args.scale_d:
+            wl = wl.scaled(d=args.scale_d)
+        recs[wid] = measure_workload(env, wl, args, lib, want_e2e=(wid == headline))
+    if env.rank == 0:
+        wl = WORKLOADS[headline] if not args.scale_d else WORKLOADS[headline].scaled(d=args.scale_d)
+        h = recs[headline]
+        line = {
+            "metric": METRIC, "value": h["value"], "unit": UNIT, "n_gpus": env.world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": h["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl),
+            "timing": f"median of {h['blocks']} blocks of {args.steps} steps each ({h['gpu_seconds_timed']:.2f} s of GPU time); "
+                      "per_workload gives the spread",
+            "clocks": h["clocks"], "e2e": h.get("e2e"), "gpu_launches": sum(r["gpu_launches"] for r in recs.values()),
+            "roofline": h["roofline"],
+            "step_frac_of_measured": h["step_frac_of_measured"], "step_frac_of_nominal_8000": h["step_frac_of_nominal_8000"],
+            "device_status": max(r["device_status"] for r in recs.values()),
+            "per_workload": [recs[w] for w in wids],
+        }
+        if not args.no_cpu_baseline and env.world == 1:
+            r = time_oracle(wl, args.cpu_steps, 0, 5.0)
+            line["cpu_baseline"] = {k: v for k, v in r.items() if k != "ms_per_step"}
+        print(json.dumps(line), flush=True)
+    if env.world > 1:
+        env.dist.destroy_process_group()
 
 
 # ---------------------------------------------------------------------------------------------
@@ -449,21 +559,26 @@ def run_sharded(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=50, help="steps per timed block")
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", type=int, default=2, help="1..5 = the five listed configurations, 2 = ResNet-18-sized 1-bit (the default); "
+    ap.add_argument("--workload", type=int, default=0,
+                    help="0 (default): the five listed configurations in one run, headline = workload 5; 1..5 = one of them; "
                          "6, 7, 8 = shape of 2 with the l2-magnitude 1-bit scale / 16-bit clipping / randomised sparsification")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="replicas", choices=["replicas", "sharded"],
                     help="replicas (default): the listed single-GPU configuration on every GPU; sharded: one worker "
                          "per GPU with the server sharded over the GPUs (an extra, not the headline)")
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="GPU time to collect per workload (blocks are repeated)")
+    ap.add_argument("--max-blocks", type=int, default=40)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-steps", type=int, default=3)
     ap.add_argument("--dump-steps", action="store_true", help="add the per-step times to the JSON line")
     ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this d (profiling captures)")
     args = ap.parse_args()
     from paper_1905_05957_b200.workloads import WORKLOADS
-    wl = WORKLOADS[args.workload]
+    headline = args.workload or HEADLINE
+    wids = (args.workload,) if args.workload else LISTED
+    wl = WORKLOADS[headline]
     if args.scale_d:
         wl = wl.scaled(d=args.scale_d)
     if args.impl == "reference":
@@ -471,7 +586,7 @@ def main():
     elif args.mode == "sharded":
         run_sharded(args, wl)
     else:
-        run_ours(args, wl)
+        run_ours(args, wids, headline)
 
 
 if __name__ == "__main__":

@@ -23,7 +23,7 @@
  *    is the default stream); they never synchronise.  One handle must be used on
  *    one stream at a time.
  *  - Every function returns a ds_status.  Nothing throws across the boundary.
- *    Conditions detected on the device are OR-ed into *dev_status (DS_DEV_*),
+ *    Conditions detected on the device are OR-ed into dev_status[0] (DS_DEV_*),
  *    which the caller reads when it chooses; kernels never trap.
  *  - All multi-byte payload fields are little-endian; all arithmetic is IEEE-754
  *    binary32 round-to-nearest-even with no fused multiply-add.
@@ -51,8 +51,15 @@ typedef enum {
   DS_ERR_UNSUPPORTED = -6
 } ds_status;
 
-/* bits of *dev_status */
+/* dev_status is four words.  Word 0 holds flags: */
 #define DS_DEV_TOPK_INCONSISTENT 0x1u /* top-k selection counted a number of entries other than k */
+/* Words 1 and 2 count top-k selections (one per vector and pass) by the route they took: with the
+ * threshold band predicted from the previous steps ("predicted": v is read once), or through the
+ * full histogram after a missing or wrong prediction ("full": v is read three times).  Both routes
+ * give the same result; the counters are for tests and tuning.  Word 3 is reserved. */
+#define DS_DEV_WORD_FLAGS 0
+#define DS_DEV_WORD_TOPK_PREDICTED 1
+#define DS_DEV_WORD_TOPK_FULL 2
 
 /* flags of ds_server_aggregate_compress */
 #define DS_FUSE_APPLY 0x1u /* also perform x = x - gamma Q[v]; ds_apply_update is then not called */
@@ -142,8 +149,8 @@ typedef struct {
  *   workspace                scratch of the top-k path; may be NULL when workspace_bytes is 0.
  *                            Zero-fill it once.  Between calls it holds only hints (the previous
  *                            steps' threshold bins); whatever it holds, results are the same
- *   dev_status uint32[1]     the caller zero-fills
- * Every non-NULL pointer must be 16-byte aligned and at least *_bytes long.
+ *   dev_status uint32[4]     the caller zero-fills (flags and counters, see DS_DEV_*)
+ * Every non-NULL pointer must be 16-byte aligned and at least *_bytes long (dev_status: 4-byte aligned).
  */
 typedef struct {
   float* x;

@@ -134,6 +134,12 @@ class QSpec:
     bits: int = 0       # clip: how many low bits of each binary32 number are set to zero (16 or 24)
 
 
+def qspec_from(q) -> "QSpec":
+    """A QSpec with the fields of any object that names an operator the same way (duck-typed: the
+    oracle imports nothing from the code it checks)."""
+    return QSpec(**{f: getattr(q, f) for f in QSpec.__dataclass_fields__ if hasattr(q, f)})
+
+
 def q_identity(v):
     v = _f32(v)
     Cv = np.empty_like(v)

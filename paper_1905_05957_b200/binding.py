@@ -137,15 +137,16 @@ def payload_views(buf: torch.Tensor, layout: ds_payload_layout, q: Q, rows: int)
 DS_STATIC_TOPK_MAX_D = 1 << 23
 
 
-def topk_worker_static(g: torch.Tensor, delta: torch.Tensor, k: int, idx: torch.Tensor, val: torch.Tensor,
+def topk_worker_static(g: torch.Tensor, delta: torch.Tensor, k: int, idx: torch.Tensor | None, val: torch.Tensor | None,
                        dev_status: torch.Tensor, stream=None) -> None:
     """ds_topk_worker_static: top-k with error feedback for one vector, using the library's built-in
     scratch array, for callers that cannot allocate device memory where they compress (inside a
     stream capture, or as a guest of a framework that owns the memory pool).  All tensors are the
     caller's; delta is updated in place.  Calls on different streams must not overlap."""
     s = stream if stream is not None else torch.cuda.current_stream(g.device)
-    rc = load_library().ds_topk_worker_static(g.data_ptr(), delta.data_ptr(), g.numel(), k, idx.data_ptr(),
-                                              val.data_ptr(), dev_status.data_ptr(), s.cuda_stream)
+    rc = load_library().ds_topk_worker_static(g.data_ptr(), delta.data_ptr(), g.numel(), k,
+                                              None if idx is None else idx.data_ptr(),
+                                              None if val is None else val.data_ptr(), dev_status.data_ptr(), s.cuda_stream)
     if rc != DS_OK:
         raise DsqError(rc, "ds_topk_worker_static")
 
@@ -153,8 +154,16 @@ def topk_worker_static(g: torch.Tensor, delta: torch.Tensor, k: int, idx: torch.
 class DoubleSqueeze:
     """One DoubleSqueeze state (x, delta_w, delta_s) on one GPU, stepped through the C ABI."""
 
+    GUARD_BYTES = 256          # sentinel bytes on each side of a buffer when guard=True
+    GUARD_PATTERN = 0xA5
+
     def __init__(self, n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int = 0,
-                 device: str | torch.device = "cuda", x0: torch.Tensor | None = None):
+                 device: str | torch.device = "cuda", x0: torch.Tensor | None = None, guard: bool = False,
+                 payload_fill: int = 0):
+        """guard=True surrounds every buffer handed to the library with GUARD_BYTES sentinel bytes
+        (check_guards() tells whether any was overwritten): a debugging aid for out-of-bounds writes.
+        payload_fill: byte the payload buffers start out with (the library must overwrite every byte
+        it defines whatever they held)."""
         if not torch.cuda.is_available():
             raise RuntimeError("paper_1905_05957_b200 needs a CUDA device; there is no CPU path")
         self.lib = load_library()
@@ -167,14 +176,28 @@ class DoubleSqueeze:
         if rc != DS_NEED_BUFFERS:
             raise DsqError(rc, "ds_create (size query)")
         dev = self.device
-        self.x = torch.zeros(d, dtype=torch.float32, device=dev) if x0 is None else \
-            x0.to(device=dev, dtype=torch.float32).contiguous().clone()
-        self.delta_w = torch.zeros(n, d, dtype=torch.float32, device=dev)
-        self.delta_s = torch.zeros(d, dtype=torch.float32, device=dev)
-        self.worker_payload = torch.zeros(bufs.worker_payload_bytes, dtype=torch.uint8, device=dev)
-        self.server_payload = torch.zeros(bufs.server_payload_bytes, dtype=torch.uint8, device=dev)
-        self.workspace = torch.zeros(max(bufs.workspace_bytes, 16), dtype=torch.uint8, device=dev)
-        self.dev_status = torch.zeros(4, dtype=torch.int32, device=dev)
+        self._guarded = []
+
+        def alloc(nbytes: int, fill: int = 0) -> torch.Tensor:
+            """nbytes of device memory as a byte tensor (16-byte aligned), optionally between guards."""
+            if not guard:
+                return torch.full((nbytes,), fill, dtype=torch.uint8, device=dev) if fill else \
+                    torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+            G = self.GUARD_BYTES
+            raw = torch.full((nbytes + 2 * G,), self.GUARD_PATTERN, dtype=torch.uint8, device=dev)
+            raw[G:G + nbytes] = fill
+            self._guarded.append((raw, nbytes))
+            return raw[G:G + nbytes]
+
+        self.x = alloc(d * 4).view(torch.float32)
+        if x0 is not None:
+            self.x.copy_(x0.to(device=dev, dtype=torch.float32).reshape(-1))
+        self.delta_w = alloc(n * d * 4).view(torch.float32).view(n, d)
+        self.delta_s = alloc(d * 4).view(torch.float32)
+        self.worker_payload = alloc(bufs.worker_payload_bytes, payload_fill)
+        self.server_payload = alloc(bufs.server_payload_bytes, payload_fill)
+        self.workspace = alloc(max(bufs.workspace_bytes, 16))
+        self.dev_status = alloc(16).view(torch.int32)
         bufs.x, bufs.delta_w, bufs.delta_s = self.x.data_ptr(), self.delta_w.data_ptr(), self.delta_s.data_ptr()
         bufs.worker_payload, bufs.server_payload = self.worker_payload.data_ptr(), self.server_payload.data_ptr()
         bufs.workspace, bufs.dev_status = self.workspace.data_ptr(), self.dev_status.data_ptr()
@@ -187,6 +210,14 @@ class DoubleSqueeze:
         self.handle = h
         self.worker_layout = get_layout(self.cfg, 0)
         self.server_layout = get_layout(self.cfg, 1)
+
+    def check_guards(self) -> bool:
+        """True if no sentinel byte around any buffer has changed (always True without guard=True)."""
+        G = self.GUARD_BYTES
+        for raw, nbytes in self._guarded:
+            if not bool((raw[:G] == self.GUARD_PATTERN).all()) or not bool((raw[G + nbytes:] == self.GUARD_PATTERN).all()):
+                return False
+        return True
 
     @classmethod
     def for_workload(cls, wl: Workload, device="cuda") -> "DoubleSqueeze":
@@ -249,7 +280,14 @@ class DoubleSqueeze:
         return payload_views(self.server_payload, self.server_layout, self.server_q, 1)[0]
 
     def device_status(self) -> int:
+        """Word 0 of dev_status: the DS_DEV_* flags."""
         return int(self.dev_status[0].item())
+
+    def topk_routes(self) -> tuple[int, int]:
+        """(predicted, full): how many top-k selections so far ran with the threshold band predicted
+        from earlier steps, and how many went through the full histogram (dev_status words 1, 2)."""
+        w = self.dev_status.cpu()
+        return int(w[1]), int(w[2])
 
     def close(self):
         if getattr(self, "handle", None):

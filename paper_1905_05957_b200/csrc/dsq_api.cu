@@ -9,18 +9,20 @@
 
 using namespace dsq;
 
-namespace dsq {
-uint64_t g_kernel_launches = 0;
+namespace {
+thread_local char g_last_error[256] = "";
 }
 
-namespace {
-
-thread_local char g_last_error[256] = "";
+namespace dsq {
+std::atomic<uint64_t> g_kernel_launches{0};
 
 int cuda_fail(cudaError_t e, const char* where) {
   snprintf(g_last_error, sizeof g_last_error, "%s: %s", where, cudaGetErrorString(e));
   return DS_ERR_CUDA;
 }
+}  // namespace dsq
+
+namespace {
 
 inline uint64_t round16(uint64_t b) { return (b + 15u) & ~uint64_t(15); }
 inline bool is_pow2(uint32_t x) { return x && !(x & (x - 1)); }
@@ -258,7 +260,7 @@ extern "C" {
 
 int ds_version(void) { return 100; }
 
-uint64_t ds_kernel_launches(void) { return g_kernel_launches; }
+uint64_t ds_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 const char* ds_last_error(void) { return g_last_error; }
 

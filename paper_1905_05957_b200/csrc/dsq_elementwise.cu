@@ -138,13 +138,22 @@ cudaError_t launch_clip(int srck, const SrcParams& src, uint32_t bits, uint8_t* 
 
 // The draw of every chunk of every vector of a pass, straight into the payload: o = first Philox word
 // of counter (0xFFFFFFFF, chunk, worker or 0xFFFFFFFF on the server pass, step), mod S.
-__global__ void __launch_bounds__(kThreads) k_rsparse_draw(const RsparseParams rp, uint64_t nc) {
+// The CTA that holds the last chunk also stores +0 into the value slots of the positions wholly past
+// d (a short last chunk): no entry ever lands there, and the payload must not depend on what the
+// buffer held before.
+__global__ void __launch_bounds__(kThreads) k_rsparse_draw(const RsparseParams rp, uint64_t nc, uint64_t d) {
   pdl_prologue();
   const uint32_t row = blockIdx.y;
   const uint64_t c = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (c >= nc) return;
-  const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c, rp.server_pass ? 0xFFFFFFFFu : row, rp.step), rp.keys);
-  rp.out_off[(uint64_t)row * rp.off_stride + c] = rnd.x & ((1u << rp.log2_keep) - 1u);
+  if (c < nc) {
+    const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c, rp.server_pass ? 0xFFFFFFFFu : row, rp.step), rp.keys);
+    rp.out_off[(uint64_t)row * rp.off_stride + c] = rnd.x & ((1u << rp.log2_keep) - 1u);
+  }
+  if (blockIdx.x == gridDim.x - 1) {
+    const uint64_t slots = nc << (rp.log2_chunk - rp.log2_keep);
+    float* val = rp.out_val + (uint64_t)row * rp.val_stride;
+    for (uint64_t s = ((d - 1) >> rp.log2_keep) + 1 + threadIdx.x; s < slots; s += kThreads) val[s] = 0.f;
+  }
 }
 
 // Q = randomised sparsification (Section 3.2): the entries of a chunk share one draw o in 0..S-1 and
@@ -180,7 +189,8 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
       }
     }
     // the group of S positions that holds the last entry: if its survivor lies past the end, its slot
-    // is sent as +0 (it may still hold a survivor of an earlier step)
+    // is sent as +0 (it may still hold a survivor of an earlier step); the slots of the groups
+    // wholly past the end are cleared by k_rsparse_draw
     if (e + cnt == src.d) {
       const uint64_t group = (src.d - 1) >> rp.log2_keep;
       if ((group << rp.log2_keep) + o >= src.d) val[group] = 0.f;
@@ -198,7 +208,7 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
 cudaError_t launch_rsparse(int srck, const SrcParams& src, const RsparseParams& rp, float* delta_out, uint64_t delta_row_stride,
                            float* x, float gamma, uint32_t rows, cudaStream_t st) {
   const uint64_t nc = (src.d + (1ull << rp.log2_chunk) - 1) >> rp.log2_chunk;
-  launch_pdl(k_rsparse_draw, dim3((unsigned)((nc + kThreads - 1) / kThreads), rows, 1), kThreads, st, rp, nc);
+  launch_pdl(k_rsparse_draw, dim3((unsigned)((nc + kThreads - 1) / kThreads), rows, 1), kThreads, st, rp, nc, src.d);
   count_launches(1);
   dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
 #define DSQ_RS(S) launch_pdl(k_rsparse<S>, grid, kThreads, st, src, rp, delta_out, delta_row_stride, x, gamma)

@@ -3,14 +3,19 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/dsq.h"
 #include "dsq_common.cuh"
 
 namespace dsq {
 
 // Kernels launched by this library since it was loaded (reported by ds_kernel_launches()).
-extern uint64_t g_kernel_launches;
-inline void count_launches(uint64_t n) { g_kernel_launches += n; }
+extern std::atomic<uint64_t> g_kernel_launches;
+inline void count_launches(uint64_t n) { g_kernel_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Records the text of a CUDA error for ds_last_error() (kept per host thread) and returns DS_ERR_CUDA.
+int cuda_fail(cudaError_t e, const char* where);
 
 // kernel<<<grid, block, 0, st>>>(args...) with programmatic stream serialization allowed (the
 // kernel begins with pdl_prologue()).  A failed launch shows in cudaGetLastError().

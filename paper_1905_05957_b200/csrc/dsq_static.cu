@@ -55,7 +55,8 @@ extern "C" int ds_topk_worker_static(const float* g, float* delta, uint64_t d, u
   topk_plan(d, 1, k, false, &plan);  // no candidate list: the scratch stays small
   if (plan.bytes > kScratchBytes) return DS_ERR_UNSUPPORTED;
   void* scratch = nullptr;
-  if (scratch_for_current_device(&scratch) != cudaSuccess) return DS_ERR_CUDA;
+  const cudaError_t es = scratch_for_current_device(&scratch);
+  if (es != cudaSuccess) return cuda_fail(es, "address of the built-in top-k scratch");
 
   SrcParams src = {};
   src.g = g;
@@ -75,5 +76,5 @@ extern "C" int ds_topk_worker_static(const float* g, float* delta, uint64_t d, u
   // the segment counts are fully rewritten before they are read, so nothing of an earlier call
   // survives into this one.
   const cudaError_t e = launch_topk(SRC_WORKER, src, plan, scratch, io, 1, k, static_cast<cudaStream_t>(cuda_stream));
-  return e == cudaSuccess ? DS_OK : DS_ERR_CUDA;
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "top-k with built-in scratch");
 }

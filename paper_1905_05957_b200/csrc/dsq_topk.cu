@@ -545,7 +545,7 @@ template <int LEVEL>
 __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t cap, const uint4* tile_info, uint64_t ntile,
                                                      uint2* dense, uint32_t* dense_count, uint32_t* kept_count,
                                                      TopkState* state, uint32_t* hist, uint32_t* done, uint32_t k,
-                                                     TopkPred* pred) {
+                                                     TopkPred* pred, uint32_t* dev_status) {
   pdl_prologue();
   __shared__ uint32_t s_hist[kBins1];
   __shared__ uint32_t s_warp[34], s_out[3];
@@ -619,6 +619,7 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
   if (LEVEL == 1) {
     // the prediction holds iff the k-th largest entry is one of the listed candidates
     const bool hit = readable && want >= 1 && want <= s_out[2];
+    atomicAdd(&dev_status[hit ? DS_DEV_WORD_TOPK_PREDICTED : DS_DEV_WORD_TOPK_FULL], 1u);  // one per selection
     if (hit) {
       st->tb1 = s_out[0];
       st->k_rem = s_out[1];
@@ -1242,15 +1243,15 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     dim3 gl1((unsigned)(148ull / rows ? 148ull / rows : 1), rows, 1);
     dim3 gl((unsigned)(148ull * 2ull / rows ? 148ull * 2ull / rows : 1), rows, 1);
     launch_pdl(k_topk_lhist<1>, gl1, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
-                                         k32, pred);
+                                         k32, pred, io.dev_status);
     launch_pdl(k_topk_hist, gm, kThreads, st, io.v_inout, d, src.vec, state, pred, list, cap, tile_info, hist);
     launch_pdl(k_topk_pick1, rows, 1024, st, hist, state, k32);
     launch_pdl(k_topk_mark, gm, kThreads, st, io.v_inout, d, src.vec, state, list, cap, tile_info, pl.ntile);
     launch_pdl(k_topk_compact, gm, kThreads, st, list, cap, tile_info, pl.ntile, dense, list_count, state);
     launch_pdl(k_topk_lhist<2>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
-                                         k32, pred);
+                                         k32, pred, io.dev_status);
     launch_pdl(k_topk_lhist<3>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
-                                         k32, pred);
+                                         k32, pred, io.dev_status);
     dim3 gc((unsigned)(148ull * 8ull / rows ? 148ull * 8ull / rows : 1), rows, 1);
     launch_pdl(k_topk_classify, gc, kThreads, st, dense, list_count, cap, state, tile_info, pl.ntile);
     launch_pdl(k_topk_scan<true>, rows, 1024, st, seg, tile_info, pl.ntile, state, k32, io.dev_status);

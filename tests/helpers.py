@@ -10,8 +10,7 @@ REL_TOL = 1e-5   # bar for fp32 values, scales and delta (reduction order may di
 
 
 def to_oracle_q(q: Q) -> oracle.QSpec:
-    return oracle.QSpec(op=q.op, chunk=q.chunk, k=q.k, levels=q.levels, norm=q.norm, bits=q.bits,
-                        keep_one_in=q.keep_one_in, scaled=q.scaled)
+    return oracle.qspec_from(q)
 
 
 def u32(t) -> np.ndarray:

@@ -21,7 +21,9 @@ RSP = lambda S=4, L=4096, scaled=0: Q("rsparse", chunk=L, keep_one_in=S, scaled=
 def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None, scribble=False):
     """Free-running: both sides start from the same state and see the same gradients; after every
     step every output must agree."""
-    ds = DoubleSqueeze(n, d, gamma, wq, sq, seed, x0=x0)
+    # every buffer sits between sentinel bytes and the payloads start out as 0xFF: a write outside a
+    # buffer, or a payload byte the library leaves to chance, fails the comparison
+    ds = DoubleSqueeze(n, d, gamma, wq, sq, seed, x0=x0, guard=True, payload_fill=0xFF)
     st = oracle.State.zeros(n, d, None if x0 is None else x0.cpu().numpy())
     if state0 is not None:
         dw, dsv = state0
@@ -38,6 +40,7 @@ def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None
         g_host = g.cpu().numpy()
         oracle.step(st, g_host, to_oracle_q(wq), to_oracle_q(sq), gamma, seed, t)
         compare_state(ds, st, g_host, tag=f"step {t}: ")
+        assert ds.check_guards(), f"step {t}: bytes outside a buffer were overwritten"
     ds.close()
     return ds, st
 
@@ -180,7 +183,11 @@ def test_topk_threshold_prediction_hits_misses_and_garbage():
     gen = torch.Generator().manual_seed(8)
     scales = [1, 1, 1, 1, 1.02, 1.05, 8.0, 8.0, 0.01, 0.01, 0.01, 1, 1]
     gs = [torch.randn(n, d, generator=gen) * s for s in scales]
-    run_lockstep(n, d, TOPK(k), TOPK(k), gs)
+    ds, _ = run_lockstep(n, d, TOPK(k), TOPK(k), gs)
+    predicted, full = ds.topk_routes()
+    assert predicted + full == (n + 1) * len(gs)
+    assert full >= 3 * (n + 1)          # the first step and the two jumps by 8x and 800x cannot be predicted
+    assert predicted >= 4 * (n + 1)     # the steady stretches are
     run_lockstep(n, d, SIGN(4096), TOPK(k // 2), gs[:6])
     run_lockstep(n, d, TOPK(k), TOPK(k), gs[:5], scribble=True)
 

@@ -91,21 +91,51 @@ def test_error_stays_bounded_on_stationary_gradients(wq, sq):
     assert max(norms[T // 2:]) <= 1.5 * max(norms[:T // 2]) + 1e-6
 
 
-def test_scaled_sparsifier_is_no_contraction_and_its_error_grows():
-    """The unbiased form of Section 3.2's last option has E||v - Q[v]||^2 = (1/p - 1)||v||^2 >= ||v||^2 for
-    p <= 1/2, outside the bounded-error assumption of Section 4: under compensation the error grows
-    geometrically, while the unscaled form (a contraction) stays bounded on the same inputs."""
-    n, d, T = 2, 512, 14
-    grown = {}
+def test_sparsifier_error_follows_from_the_draws_and_the_scaled_form_grows():
+    """Section 3.2's last option under Algorithm 1, worked out from the operator's definition.  An entry
+    that survives leaves the residual v - S v = (1 - S) v in the scaled (unbiased) form and 0 in the
+    plain form; an entry that is dropped leaves v.  So, given the draws, the residual is a known
+    linear function of the gradients: delta_T = sum_t g_t * prod_{s >= t} m_s with m_s = 1 - S (scaled)
+    or 0 (plain) where the entry's offset mod S equals the chunk's draw of step s, else 1.  The
+    multipliers are small integers, so the only differences are the binary32 roundings of g + delta and of
+    v - Q[v], whose bound is carried along, and the oracle's residual must reproduce the closed form within it.  The scaled form has E||v - Q[v]||^2 = (S - 1)||v||^2 >= ||v||^2
+    for S >= 2: no contraction, outside the bounded-error assumption of Section 4, and its error must
+    grow the way the multipliers say; the plain form multiplies by 0 or 1 and cannot grow."""
+    n, d, T, L, S, seed = 2, 512, 14, 128, 4, 8
+    gs = _grads(n, d, T, seed=4)
+    offs_in_chunk = np.arange(d) % L
+    ratio = {}
     for scaled in (0, 1):
-        q = QSpec(oracle.RSPARSE, chunk=128, keep_one_in=4, scaled=scaled)
+        q = QSpec(oracle.RSPARSE, chunk=L, keep_one_in=S, scaled=scaled)
         st = oracle.State.zeros(n, d)
-        norms = []
-        for t, g in enumerate(_grads(n, d, T, seed=4)):
-            oracle.worker_pass(st, g, q, 8, t)
+        want = np.zeros((n, d), dtype=np.float64)     # the closed form, carried along step by step
+        bound = np.zeros((n, d), dtype=np.float64)    # binary32 rounding of g + delta and of v - Q[v], carried the same way
+        u = 2.0**-24
+        norms, want_norms = [], []
+        for t, g in enumerate(gs):
+            oracle.worker_pass(st, g, q, seed, t)
+            for i in range(n):
+                draw = np.repeat(st.worker_payloads[i]["off"], L)[:d]       # the draws the operator reports
+                # ... which are the documented Philox words, not something the operator could choose
+                for c in (0, d // L - 1):
+                    assert draw[c * L] == oracle.philox4x32_10([0xFFFFFFFF, c, i, t], [seed, 0])[0] % S
+                m = np.where(offs_in_chunk % S == draw, (1.0 - S) if scaled else 0.0, 1.0)
+                v = want[i] + g[i].astype(np.float64)
+                want[i] = v * m
+                bound[i] = (bound[i] + u * np.abs(v)) * np.abs(m) + u * np.abs(v * m)
             norms.append(float(np.linalg.norm(st.delta_w)))
-        grown[scaled] = norms[-1] / norms[1]
-    assert grown[1] > 50 and grown[0] < 5      # about 1.5x per step against a plateau
+            want_norms.append(float(np.linalg.norm(want)))
+            err = np.abs(st.delta_w.astype(np.float64) - want)
+            assert np.all(err <= 2.0 * bound + 1e-30)
+        ratio[scaled] = (norms[-1] / norms[1], want_norms[-1] / want_norms[1])
+    for scaled in (0, 1):
+        assert abs(ratio[scaled][0] / ratio[scaled][1] - 1.0) < 1e-5
+    # growth per step of the scaled form: E m^2 = (1/S)(S-1)^2 + (1 - 1/S) = S - 1, so the norm gains a
+    # factor sqrt(S - 1) per step on average, 3^6 = 729 over the twelve steps compared; entries differ in
+    # how often they were drawn, so the realised factor is allowed an order of magnitude below that
+    assert ratio[1][0] > (S - 1) ** ((T - 2) / 2) / 10
+    # the plain form keeps |delta| <= the gradients summed since the entry last survived: no growth
+    assert ratio[0][0] < 5
 
 
 def test_server_uses_its_own_stream_and_workers_differ():
