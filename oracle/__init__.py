@@ -14,7 +14,7 @@ import numpy as np
 
 from . import build as _build
 
-IDENTITY, SIGN1, TOPK, QSGD, CLIP, RSPARSE = "identity", "sign1", "topk", "qsgd", "clip", "rsparse"
+IDENTITY, SIGN1, TOPK, QSGD, CLIP, RSPARSE, TERNARY = "identity", "sign1", "topk", "qsgd", "clip", "rsparse", "ternary"
 SERVER_WID = 0xFFFFFFFF
 
 _lib = None
@@ -27,6 +27,12 @@ def load(path: str):
     u64, u32 = C.c_uint64, C.c_uint32
     L.orc_pairwise_sum.restype = C.c_float
     L.orc_pairwise_sum.argtypes = [f32p, u64]
+    L.orc_pairwise_sum_padded.restype = C.c_float
+    L.orc_pairwise_sum_padded.argtypes = [f32p, u64, u64]
+    L.orc_server_mean.restype = None
+    L.orc_server_mean.argtypes = [f32p, u32, u64, f32p]
+    L.orc_q_ternary.argtypes = [f32p, u64, u64, u32, u32, u32p, u32p, f32p, f32p, f32p]
+    L.orc_decode_ternary.argtypes = [u32p, u32p, f32p, u64, f32p]
     L.orc_philox4x32_10.restype = None
     L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
     L.orc_ef_add.restype = None
@@ -81,6 +87,12 @@ def pairwise_sum(a) -> np.float32:
     return np.float32(lib().orc_pairwise_sum(_p(a, C.c_float), a.size))
 
 
+def pairwise_sum_padded(a, L) -> np.float32:
+    """Pairwise sum of a padded with +0 to L entries (L a power of two >= len(a))."""
+    a = _f32(a)
+    return np.float32(lib().orc_pairwise_sum_padded(_p(a, C.c_float), a.size, L))
+
+
 def philox4x32_10(ctr, key) -> np.ndarray:
     c = np.ascontiguousarray(ctr, dtype=np.uint32)
     k = np.ascontiguousarray(key, dtype=np.uint32)
@@ -111,6 +123,15 @@ def server_mean_add(C_all, delta_s) -> np.ndarray:
     return v
 
 
+def server_mean(C_all) -> np.ndarray:
+    """(1/n) sum_i Q[v_i] alone: the server's vector when no error is carried."""
+    C_all = _f32(C_all)
+    n, d = C_all.shape
+    v = np.empty(d, dtype=np.float32)
+    lib().orc_server_mean(_p(C_all, C.c_float), n, d, _p(v, C.c_float))
+    return v
+
+
 def apply_update(x, Cv, gamma) -> np.ndarray:
     x = _f32(x).copy()
     Cv = _f32(Cv)
@@ -125,7 +146,7 @@ def apply_update(x, Cv, gamma) -> np.ndarray:
 @dataclass(frozen=True)
 class QSpec:
     op: str = IDENTITY
-    chunk: int = 0      # sign1 / qsgd: chunk length L (power of two)
+    chunk: int = 0      # sign1 / qsgd / rsparse: chunk length L (power of two); sign1: 0 = one factor for the whole vector
     norm: int = 1       # sign1: the scale is the ratio of l1 (1) or l2 (2) magnitudes
     k: int = 0          # topk
     levels: int = 0     # qsgd: s
@@ -151,7 +172,7 @@ def q_sign1(v, L, norm=1):
     v = _f32(v)
     d = v.size
     bits = np.zeros((d + 31) // 32, dtype=np.uint32)
-    scale = np.zeros((d + L - 1) // L, dtype=np.float32)
+    scale = np.zeros((d + L - 1) // L if L else 1, dtype=np.float32)
     Cv = np.empty_like(v)
     _check(lib().orc_q_sign1(_p(v, C.c_float), d, L, norm, _p(bits, C.c_uint32), _p(scale, C.c_float),
                              _p(Cv, C.c_float)), "sign1")
@@ -164,6 +185,30 @@ def decode_sign1(bits, scale, d, L):
     scale = _f32(scale)
     _check(lib().orc_decode_sign1(_p(bits, C.c_uint32), _p(scale, C.c_float), d, L, _p(Cv, C.c_float)),
            "decode_sign1")
+    return Cv
+
+
+def q_ternary(v, seed, step, wid):
+    v = _f32(v)
+    d = v.size
+    sgn = np.zeros((d + 31) // 32, dtype=np.uint32)
+    nz = np.zeros((d + 31) // 32, dtype=np.uint32)
+    scale = np.zeros(1, dtype=np.float32)
+    vmax = np.zeros(1, dtype=np.float32)
+    Cv = np.empty_like(v)
+    _check(lib().orc_q_ternary(_p(v, C.c_float), d, C.c_uint64(seed), step, wid, _p(sgn, C.c_uint32), _p(nz, C.c_uint32),
+                               _p(scale, C.c_float), _p(vmax, C.c_float), _p(Cv, C.c_float)), "ternary")
+    # the payload is (sgn, nz, scale); the largest magnitude is returned as well for the tests that pin it
+    return Cv, {"sgn": sgn, "nz": nz, "scale": scale, "max": vmax}
+
+
+def decode_ternary(sgn, nz, scale, d):
+    sgn = np.ascontiguousarray(sgn, dtype=np.uint32)
+    nz = np.ascontiguousarray(nz, dtype=np.uint32)
+    scale = _f32(scale)
+    Cv = np.empty(d, dtype=np.float32)
+    _check(lib().orc_decode_ternary(_p(sgn, C.c_uint32), _p(nz, C.c_uint32), _p(scale, C.c_float), d, _p(Cv, C.c_float)),
+           "decode_ternary")
     return Cv
 
 
@@ -261,6 +306,8 @@ def compress(q: QSpec, v, seed=0, step=0, wid=0):
         return q_clip(v, q.bits)
     if q.op == RSPARSE:
         return q_rsparse(v, q.chunk, q.keep_one_in, q.scaled, seed, step, wid)
+    if q.op == TERNARY:
+        return q_ternary(v, seed, step, wid)
     raise ValueError(q.op)
 
 
@@ -283,33 +330,40 @@ class State:
         return State(x, np.zeros((n, d), dtype=np.float32), np.zeros(d, dtype=np.float32))
 
 
-def worker_pass(st: State, g, worker_q: QSpec, seed: int, step: int) -> np.ndarray:
-    """Worker side of Algorithm 1 for all n workers; returns the dense [n, d] Q[v_i]."""
+def worker_pass(st: State, g, worker_q: QSpec, seed: int, step: int, compensate: bool = True) -> np.ndarray:
+    """Worker side of Algorithm 1 for all n workers; returns the dense [n, d] Q[v_i].
+    compensate=False: Section 5.1's methods without compensation: Q[g_i] is sent, no error is kept."""
     g = _f32(g)
     n, d = g.shape
     C_all = np.empty((n, d), dtype=np.float32)
     st.worker_payloads = []
     for i in range(n):
-        v = ef_add(g[i], st.delta_w[i])                       # Eq. 2
+        if compensate:
+            v = ef_add(g[i], st.delta_w[i])                    # Eq. 2
+        else:
+            v = g[i]
         Cv, payload = compress(worker_q, v, seed, step, i)     # compress
-        st.delta_w[i] = residual(v, Cv)                        # Eq. 3
+        if compensate:
+            st.delta_w[i] = residual(v, Cv)                    # Eq. 3
         C_all[i] = Cv
         st.worker_payloads.append(payload)
     return C_all
 
 
-def server_pass(st: State, C_all, server_q: QSpec, seed: int, step: int) -> np.ndarray:
+def server_pass(st: State, C_all, server_q: QSpec, seed: int, step: int, compensate: bool = True) -> np.ndarray:
     """Server side of Algorithm 1 (Eq. 4); returns the dense Q[v] sent to the workers."""
-    v = server_mean_add(C_all, st.delta_s)
+    v = server_mean_add(C_all, st.delta_s) if compensate else server_mean(C_all)
     Cv, payload = compress(server_q, v, seed, step, SERVER_WID)
-    st.delta_s = residual(v, Cv)
+    if compensate:
+        st.delta_s = residual(v, Cv)
     st.server_payload = payload
     return Cv
 
 
-def step(st: State, g, worker_q: QSpec, server_q: QSpec, gamma: float, seed: int, t: int) -> np.ndarray:
+def step(st: State, g, worker_q: QSpec, server_q: QSpec, gamma: float, seed: int, t: int,
+         compensate: bool = True) -> np.ndarray:
     """One full iteration of Algorithm 1; mutates ``st`` and returns the dense server Q[v]."""
-    C_all = worker_pass(st, g, worker_q, seed, t)
-    Cv = server_pass(st, C_all, server_q, seed, t)
+    C_all = worker_pass(st, g, worker_q, seed, t, compensate)
+    Cv = server_pass(st, C_all, server_q, seed, t, compensate)
     st.x = apply_update(st.x, Cv, gamma)
     return Cv

@@ -28,7 +28,9 @@
  * binary cases, its error bound and idempotence; randomised sparsification by
  * its keep frequency, its mean, and the structure of what it sends; Philox4x32-10 against an
  * independent library implementation; pairwise summation against hand-derived
- * rounding cases.  No function here is "parity unpinned".
+ * rounding cases; the ternary quantiser by Monte Carlo (unbiased before its
+ * scaling), its always-kept largest entry and its l1 factor; the passes without
+ * compensation against plain compressed SGD.  No function here is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -59,6 +61,30 @@ static float pairwise_sum(const float* a, size_t len) {
   float right = pairwise_sum(a + half, half);
   float s = left + right;
   return s;
+}
+
+/* The same sum over a[0..len) padded with +0 up to L entries (L a power of two, len <= L), without
+ * storing the padding: a half that holds only padding sums to +0, and x + (+0) = x for every x that
+ * can occur here (the terms are |v| or v*v, never -0). */
+static float pairwise_sum_padded(const float* a, uint64_t len, uint64_t L) {
+  if (len == 0) return 0.0f;
+  if (L == 1) return a[0];
+  uint64_t half = L / 2;
+  float left = pairwise_sum_padded(a, len < half ? len : half, half);
+  float right = pairwise_sum_padded(a + half, len > half ? len - half : 0, half);
+  float s = left + right;
+  return s;
+}
+
+static uint64_t next_pow2_u64(uint64_t x) {
+  uint64_t p = 1;
+  while (p < x) p <<= 1;
+  return p;
+}
+
+float orc_pairwise_sum_padded(const float* a, uint64_t len, uint64_t L) {
+  if (L == 0 || (L & (L - 1)) != 0 || len > L) return NAN;
+  return pairwise_sum_padded(a, len, L);
 }
 
 /* Exposed for the tests that pin the summation order. */
@@ -167,8 +193,12 @@ int orc_q_identity(const float* v, uint64_t d, float* C) {
 /*   C    : d floats (may be NULL)                                           */
 /* ------------------------------------------------------------------------ */
 
+static int q_sign1_whole(const float* v, uint64_t d, uint32_t norm, uint32_t* bits, float* scale, float* C);
+
 int orc_q_sign1(const float* v, uint64_t d, uint32_t L, uint32_t norm, uint32_t* bits, float* scale, float* C) {
-  if (!is_pow2_u32(L) || (norm != 1 && norm != 2)) return ORC_ERR_ARG;
+  if (norm != 1 && norm != 2) return ORC_ERR_ARG;
+  if (L == 0) return q_sign1_whole(v, d, norm, bits, scale, C);
+  if (!is_pow2_u32(L)) return ORC_ERR_ARG;
   uint64_t nw = (d + 31) / 32, nc = (d + L - 1) / L;
   float* term = (float*)malloc(sizeof(float) * L);
   if (!term) return ORC_ERR_NOMEM;
@@ -203,10 +233,43 @@ int orc_q_sign1(const float* v, uint64_t d, uint32_t L, uint32_t norm, uint32_t*
   return ORC_OK;
 }
 
-int orc_decode_sign1(const uint32_t* bits, const float* scale, uint64_t d, uint32_t L, float* C) {
-  if (L == 0) return ORC_ERR_ARG;
+/* L = 0: the operator exactly as Section 3.2 and Section 5.1 state it, with ONE scaling factor for the
+ * whole vector: magnitude of v over magnitude of sign(v), i.e. ||v||_1 / d (norm = 1) or
+ * ||v||_2 / sqrt(d) (norm = 2).  The sum runs pairwise over the vector padded with +0 to the next
+ * power of two.  scale holds one float. */
+static int q_sign1_whole(const float* v, uint64_t d, uint32_t norm, uint32_t* bits, float* scale, float* C) {
+  uint64_t nw = (d + 31) / 32;
+  float* term = (float*)malloc(sizeof(float) * (d ? d : 1));
+  if (!term) return ORC_ERR_NOMEM;
+  memset(bits, 0, sizeof(uint32_t) * nw);
+  float s;
+  if (norm == 1) {
+    for (uint64_t j = 0; j < d; ++j) term[j] = fabsf(v[j]);
+    float l1 = pairwise_sum_padded(term, d, next_pow2_u64(d));
+    s = l1 / (float)d;
+  } else {
+    for (uint64_t j = 0; j < d; ++j) {
+      float e2 = v[j] * v[j];
+      term[j] = e2;
+    }
+    float ss = pairwise_sum_padded(term, d, next_pow2_u64(d));
+    float l2 = sqrtf(ss);
+    float root_d = sqrtf((float)d);
+    s = l2 / root_d;
+  }
+  scale[0] = s;
   for (uint64_t j = 0; j < d; ++j) {
-    float s = scale[j / L];
+    int nonneg = v[j] >= 0.0f;
+    if (nonneg) bits[j / 32] |= (uint32_t)1 << (j % 32);
+    if (C) C[j] = nonneg ? s : -s;
+  }
+  free(term);
+  return ORC_OK;
+}
+
+int orc_decode_sign1(const uint32_t* bits, const float* scale, uint64_t d, uint32_t L, float* C) {
+  for (uint64_t j = 0; j < d; ++j) {
+    float s = L ? scale[j / L] : scale[0];
     int nonneg = (bits[j / 32] >> (j % 32)) & 1u;
     C[j] = nonneg ? s : -s;
   }
@@ -451,4 +514,105 @@ int orc_decode_qsgd(const uint8_t* lvl, const uint32_t* sgn, const float* qstep,
     C[j] = nonneg ? mag : -mag;
   }
   return ORC_OK;
+}
+
+
+/* ------------------------------------------------------------------------ */
+/* Q = ternary quantisation, the "QSGD" of Section 5.1 ("Implementations and  */
+/* setups", item 2): every entry becomes -1, 0 or +1.  With m the entry of   */
+/* largest absolute value of the whole vector, an entry e becomes sign(e)    */
+/* with probability |e|/|m| and 0 otherwise; then one scaling factor,        */
+/* magnitude of the vector over magnitude of the ternary vector, multiplies  */
+/* it.  Reading: magnitudes are l1 norms (as for the 1-bit operator), so the */
+/* factor is ||v||_1 / (number of non-zero entries); the sum is pairwise     */
+/* over the vector padded with +0 to the next power of two.  The sign of an  */
+/* entry is the bit (v >= 0).  Uniform variate: 24-bit fraction of a         */
+/* Philox4x32-10 word, key = seed, counter = (j/4, 0xFFFFFFFE, wid, step),   */
+/* entry j using output word j%4; the entry survives iff u < |e|/|m| (one    */
+/* binary32 division), so the largest entry survives always (u < 1).  A      */
+/* vector of zeros is sent as zeros with factor 0.                           */
+/*   sgn : ceil(d/32) words, bit = (v >= 0)                                  */
+/*   nz  : ceil(d/32) words, bit = entry is non-zero in the ternary vector   */
+/*   scale: one float;  vmax: one float (|m|, for the tests that pin it)     */
+/* ------------------------------------------------------------------------ */
+
+int orc_q_ternary(const float* v, uint64_t d, uint64_t seed, uint32_t step, uint32_t wid, uint32_t* sgn,
+                  uint32_t* nz, float* scale, float* vmax, float* C) {
+  if (d == 0 || d > 0xFFFFFFFFull) return ORC_ERR_ARG;
+  uint64_t nw = (d + 31) / 32;
+  float* term = (float*)malloc(sizeof(float) * d);
+  if (!term) return ORC_ERR_NOMEM;
+  memset(sgn, 0, sizeof(uint32_t) * nw);
+  memset(nz, 0, sizeof(uint32_t) * nw);
+  const uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)};
+  const float two_m24 = 1.0f / 16777216.0f;
+  float m = 0.0f;
+  for (uint64_t j = 0; j < d; ++j) {
+    float a = fabsf(v[j]);
+    term[j] = a;
+    if (a > m) m = a;
+  }
+  float l1 = pairwise_sum_padded(term, d, next_pow2_u64(d));
+  uint64_t count = 0;
+  for (uint64_t j = 0; j < d; ++j) {
+    uint32_t ctr[4] = {(uint32_t)(j / 4), 0xFFFFFFFEu, wid, step};
+    uint32_t rnd[4];
+    orc_philox4x32_10(ctr, key, rnd);
+    uint32_t w = rnd[j % 4];
+    float u = (float)(w >> 8) * two_m24; /* exact, in [0, 1) */
+    int kept = 0;
+    if (m > 0.0f) {
+      float p = term[j] / m;
+      kept = u < p;
+    }
+    if (v[j] >= 0.0f) sgn[j / 32] |= (uint32_t)1 << (j % 32);
+    if (kept) {
+      nz[j / 32] |= (uint32_t)1 << (j % 32);
+      ++count;
+    }
+  }
+  float s = 0.0f;
+  if (count > 0) s = l1 / (float)count;
+  scale[0] = s;
+  if (vmax) vmax[0] = m;
+  if (C) {
+    for (uint64_t j = 0; j < d; ++j) {
+      int kept = (nz[j / 32] >> (j % 32)) & 1u;
+      int nonneg = (sgn[j / 32] >> (j % 32)) & 1u;
+      C[j] = kept ? (nonneg ? s : -s) : 0.0f;
+    }
+  }
+  free(term);
+  return ORC_OK;
+}
+
+int orc_decode_ternary(const uint32_t* sgn, const uint32_t* nz, const float* scale, uint64_t d, float* C) {
+  float s = scale[0];
+  for (uint64_t j = 0; j < d; ++j) {
+    int kept = (nz[j / 32] >> (j % 32)) & 1u;
+    int nonneg = (sgn[j / 32] >> (j % 32)) & 1u;
+    C[j] = kept ? (nonneg ? s : -s) : 0.0f;
+  }
+  return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* The same passes without error compensation (Section 5.1, items 2 and 5:   */
+/* "QSGD" and "Top-k SGD" compress the gradient itself and keep no error):   */
+/* the vector that is compressed is g on a worker and the plain mean on the  */
+/* server; no error is read, none is written.                                */
+/* ------------------------------------------------------------------------ */
+
+void orc_server_mean(const float* C_all, uint32_t n, uint64_t d, float* v) {
+  float one = 1.0f;
+  float inv_n = one / (float)n;
+  for (uint64_t j = 0; j < d; ++j) {
+    float acc = 0.0f;
+    for (uint32_t i = 0; i < n; ++i) {
+      float t = acc + C_all[(uint64_t)i * d + j];
+      acc = t;
+    }
+    float mean = acc * inv_n;
+    v[j] = mean;
+  }
 }

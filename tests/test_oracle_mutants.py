@@ -9,6 +9,7 @@ import oracle
 from tests import test_oracle_algorithm as t_alg
 from tests import test_oracle_operators as t_ops
 from tests import test_oracle_primitives as t_prim
+from tests import test_oracle_whole_vector as t_whole
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "dsq_oracle.c")
 
@@ -70,6 +71,28 @@ MUTANTS = [
     ("update adds instead of subtracting",
      "float r = x[j] - t;", "float r = x[j] + t;",
      t_alg.test_identity_reduces_to_parallel_sgd_bitwise),
+    ("whole-vector factor divides by the padded length",
+     "s = l1 / (float)d;", "s = l1 / (float)next_pow2_u64(d);",
+     t_whole.test_whole_vector_sign_short_vector_divides_by_its_true_length),
+    ("padded sum forgets a partly filled right half",
+     "float right = pairwise_sum_padded(a + half, len > half ? len - half : 0, half);",
+     "float right = len >= L ? pairwise_sum_padded(a + half, half, half) : 0.0f;",
+     lambda: t_whole.test_padded_pairwise_sum_equals_the_sum_over_the_written_out_padding(1025, 2048)),
+    ("ternary keeps an entry with probability 1 - |e|/|m|",
+     "kept = u < p;", "kept = u < 1.0f - p;",
+     t_whole.test_ternary_is_unbiased_before_scaling_and_keeps_the_largest_entry_always),
+    ("ternary factor divides by the length instead of the non-zero count",
+     "if (count > 0) s = l1 / (float)count;", "if (count > 0) s = l1 / (float)d;",
+     t_whole.test_ternary_structure_scale_and_the_documented_philox_word),
+    ("ternary takes the largest signed value as m",
+     "if (a > m) m = a;", "if (v[j] > m) m = v[j];",
+     t_whole.test_ternary_degenerate_vectors),
+    ("ternary draws from the quantiser's counter",
+     "uint32_t ctr[4] = {(uint32_t)(j / 4), 0xFFFFFFFEu, wid, step};", "uint32_t ctr[4] = {(uint32_t)(j / 4), 0u, wid, step};",
+     t_whole.test_ternary_structure_scale_and_the_documented_philox_word),
+    ("uncompensated server forgets the 1/n",
+     "float mean = acc * inv_n;\n    v[j] = mean;", "float mean = acc;\n    v[j] = mean;",
+     lambda: t_whole.test_without_compensation_the_model_follows_plain_compressed_sgd("sign1", "topk")),
 ]
 
 

@@ -27,14 +27,17 @@ DRIVER = textwrap.dedent("""
     for d in (1, 3, 4, 5, 31, 32, 33, 127, 128, 129, 255, 256, 257, 1000, 4095, 4096, 4097):
         v = (r.standard_normal(d) * 10.0 ** r.uniform(-3, 3)).astype(np.float32)
         v[r.integers(0, d)] = 0.0
-        for L in (4, 128, 256, 4096):
+        oracle.q_ternary(v, 2**40 + 3, 7, 2)
+        c, p = oracle.q_ternary(v, 5, 1, oracle.SERVER_WID)
+        oracle.decode_ternary(p["sgn"], p["nz"], p["scale"], d)
+        for L in (0, 4, 128, 256, 4096):
             oracle.q_sign1(v, L, 1); oracle.q_sign1(v, L, 2)
             c, p = oracle.q_sign1(v, L)
             oracle.decode_sign1(p["bits"], p["scale"], d, L)
-            for s in (1, 15, 255):
+            for s in ((1, 15, 255) if L else ()):
                 c, p = oracle.q_qsgd(v, L, s, 2**40 + 3, 7, 2)
                 oracle.decode_qsgd(p["lvl"], p["sgn"], p["step"], d, L)
-            for S in (2, 4):
+            for S in ((2, 4) if L else ()):
                 for scaled in (0, 1):
                     c, p = oracle.q_rsparse(v, L, S, scaled, 5, 1, 0)
                     oracle.decode_rsparse(p["val"], p["off"], d, L, S)
@@ -48,14 +51,14 @@ DRIVER = textwrap.dedent("""
     for n in (1, 2, 128):
         oracle.pairwise_sum(r.standard_normal(n).astype(np.float32))
     oracle.philox4x32_10([1, 2, 3, 4], [5, 6])
-    ops = [Q("identity"), Q("sign1", chunk=128), Q("sign1", chunk=128, norm=2), Q("topk", k=17), Q("qsgd", chunk=128, levels=15),
+    ops = [Q("identity"), Q("ternary"), Q("sign1", chunk=0), Q("sign1", chunk=128), Q("sign1", chunk=128, norm=2), Q("topk", k=17), Q("qsgd", chunk=128, levels=15),
            Q("clip", bits=16), Q("clip", bits=24), Q("rsparse", chunk=128, keep_one_in=4)]
     for wq in ops:
         for sq in ops:
             n, d = 3, 333
             st = oracle.State.zeros(n, d)
             for t in range(2):
-                oracle.step(st, r.standard_normal((n, d)).astype(np.float32), wq, sq, 0.1, 9, t)
+                oracle.step(st, r.standard_normal((n, d)).astype(np.float32), wq, sq, 0.1, 9, t, compensate=bool(t))
     print("sanitized oracle ok")
 """)
 
