@@ -61,8 +61,9 @@ KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "identity": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
     "clip": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
     "rsparse": ("dsq_elementwise.cu", "dsq_common.cuh", "dsq_internal.h"),
+    "ternary": ("dsq_whole.cu", "dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
 }
-DOMINANT = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
+DOMINANT = {"ternary": "k_whole_reduce / k_whole_ternary_draw / k_whole_ternary_apply <WORKER>", "sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER>",
             "topk": "top-k worker pass (k_topk_pass1<WORKER> and the selection tail)",
             "identity": "k_identity<WORKER>", "clip": "k_clip<WORKER>", "rsparse": "k_rsparse<WORKER>"}
 
@@ -70,7 +71,7 @@ DOMINANT = {"sign1": "k_chunked<SIGN1, WORKER>", "qsgd": "k_chunked<QSGD, WORKER
 def payload_bytes(q, d: int) -> int:
     nw = (d + 31) // 32
     if q.op == "sign1":
-        return 4 * nw + 4 * ((d + q.chunk - 1) // q.chunk)
+        return 4 * nw + 4 * ((d + q.chunk - 1) // q.chunk if q.chunk else 1)
     if q.op == "qsgd":
         return d + 4 * nw + 4 * ((d + q.chunk - 1) // q.chunk)
     if q.op == "topk":
@@ -80,6 +81,8 @@ def payload_bytes(q, d: int) -> int:
     if q.op == "rsparse":
         nc = (d + q.chunk - 1) // q.chunk
         return 4 * nc * (q.chunk // q.keep_one_in) + 4 * nc
+    if q.op == "ternary":
+        return 8 * nw + 4
     return 4 * d
 
 
@@ -89,9 +92,10 @@ def algorithmic_bytes(wl) -> dict:
     reads and writes x (only the k kept entries for top-k)."""
     n, d = wl.n, wl.d
     pw, ps = payload_bytes(wl.worker_q, d), payload_bytes(wl.server_q, d)
-    worker = n * d * 12 + n * pw
+    err = 8 if wl.compensate else 0          # an error is read and written, or there is none
+    worker = n * d * (4 + err) + n * pw
     x_bytes = 8 * wl.server_q.k if wl.server_q.op == "topk" else 8 * d
-    server = n * pw + 8 * d + ps + x_bytes
+    server = n * pw + err * d + ps + x_bytes
     return {"worker": worker, "server": server, "total": worker + server}
 
 
@@ -107,7 +111,8 @@ def captured_traffic(wl):
     """DRAM bytes per launch of the workload's dominant kernel from the committed capture, scaled to
     this launch's entries; None without a capture or once the kernel's sources have changed."""
     cap = NCU_CAPTURES.get(wl.worker_q.op)
-    if cap is None or cap[3] != csrc_digest(wl.worker_q.op):
+    whole = wl.worker_q.op == "sign1" and wl.worker_q.chunk == 0     # other kernels than the captured ones
+    if cap is None or whole or not wl.compensate or cap[3] != csrc_digest(wl.worker_q.op):
         return None
     return int(cap[1] * (wl.n * wl.d) / cap[2])
 
@@ -211,10 +216,10 @@ def time_oracle(wl, steps: int, warmup: int, seconds_per_step: float) -> dict:
     wq, sq = oracle.qspec_from(swl.worker_q), oracle.qspec_from(swl.server_q)
     gs = [make_gradients(swl, t, device="cpu").numpy() for t in range(2)]
     for t in range(warmup):
-        oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, t)
+        oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, t, compensate=swl.compensate)
     t0 = time.perf_counter()
     for t in range(steps):
-        oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, warmup + t)
+        oracle.step(st, gs[t % 2], wq, sq, swl.gamma, swl.seed, warmup + t, compensate=swl.compensate)
     dt = time.perf_counter() - t0
     assert np.isfinite(st.x).all()
     return {"value": swl.n * swl.d * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -250,7 +255,7 @@ def workload_config(wl) -> dict:
                 **({"bits_cleared": s.bits} if s.op == "clip" else {}),
                 **({"keep_one_in": s.keep_one_in, "scaled": bool(s.scaled)} if s.op == "rsparse" else {})}
     return {"workload": wl.name, "n_workers": wl.n, "d": wl.d, "gradient_dist": wl.dist, "worker_q": q(wl.worker_q),
-            "server_q": q(wl.server_q), "gamma": wl.gamma,
+            "server_q": q(wl.server_q), "gamma": wl.gamma, "error_compensation": wl.compensate,
             "l2": "inputs larger than L2: g and delta_w are streamed once per step and exceed 126 MB"
                   if wl.n * wl.d * 8 > 2 * 126e6 else "L2 flushed between steps by writing a 256 MB buffer"}
 
@@ -289,11 +294,14 @@ def measure_workload(env: Env, wl, args, lib, want_e2e: bool) -> dict:
     dev, world, rank = env.dev, env.world, env.rank
     K, W = args.steps, max(args.warmup, 3)
     ds = DoubleSqueeze.for_workload(wl, dev)
-    # distinct g_t resident in HBM: a fresh draw for every step where 48 GB hold them, else a ring of
-    # as many as fit (a training run never sees the same gradient twice; a short ring makes the
-    # top-k threshold oscillate with the ring's period)
-    R = max(2, min(K + W, int(48e9 // (wl.n * wl.d * 4))))
+    # distinct g_t resident in HBM: a fresh draw for every step of a block where 100 GB hold them, else
+    # a ring of as many as fit.  A training run never sees the same gradient twice, and a replayed
+    # sequence makes the error feedback -- hence the top-k threshold -- follow the ring's period, so
+    # where a threshold history matters the ring is drawn afresh (untimed) before every block.
+    R = max(2, min(K + W, int(100e9 // (wl.n * wl.d * 4))))
     ring = [make_gradients(wl, t, device=dev) for t in range(R)]
+    redraw = "topk" in (wl.worker_q.op, wl.server_q.op)
+    drawn = R
     need_flush = wl.n * wl.d * 8 <= 2 * 126e6
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
     stream = torch.cuda.current_stream(dev)
@@ -341,6 +349,10 @@ def measure_workload(env: Env, wl, args, lib, want_e2e: bool) -> dict:
     (slowest,) = max_over_ranks([total], device=dev)
     more = min(args.max_blocks, math.ceil(args.min_seconds * 1e3 / max(slowest, 1e-3))) - 1
     for _ in range(max(0, more)):
+        if redraw:
+            for slot in range(R):
+                make_gradients(wl, drawn, device=dev, out=ring[slot])
+                drawn += 1
         total, steps = timed_block()
         blocks.append(total)
         steps_all += steps
@@ -428,7 +440,10 @@ def measure_workload(env: Env, wl, args, lib, want_e2e: bool) -> dict:
     traffic = captured_traffic(wl)
     ms_per_step = block_med_slowest / K
     step_gbs = ab["total"] / (ms_per_step * 1e-3) / 1e9
-    roof = {"bound": "hbm", "kernel": DOMINANT[wl.worker_q.op], "achieved": achieved, "peak": peak, "unit": "GB/s",
+    dominant = DOMINANT[wl.worker_q.op]
+    if wl.worker_q.op == "sign1" and wl.worker_q.chunk == 0:
+        dominant = "k_whole_reduce / k_whole_sign <WORKER>"
+    roof = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": traffic,
             "algorithmic_bytes_per_launch": ab["worker"], "ms_per_launch": wk_ms,
             "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
@@ -563,7 +578,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", type=int, default=0,
                     help="0 (default): the five listed configurations in one run, headline = workload 5; 1..5 = one of them; "
-                         "6, 7, 8 = shape of 2 with the l2-magnitude 1-bit scale / 16-bit clipping / randomised sparsification")
+                         "6..12 = shape of 2 with the l2-magnitude 1-bit scale / 16-bit clipping / randomised sparsification / "
+                         "ternary quantiser / 1-bit with one factor per vector / the two methods without compensation")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--mode", default="replicas", choices=["replicas", "sharded"],
                     help="replicas (default): the listed single-GPU configuration on every GPU; sharded: one worker "

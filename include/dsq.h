@@ -107,10 +107,27 @@ typedef enum {
  *                compensated error grows; offered for completeness).  norm = DS_RSPARSE_PLAIN:
  *                survivors keep their value (a contraction).
  *
+ * DS_Q_SIGN1 with chunk = 0: the 1-bit operator exactly as Section 3.2 and Section 5.1 state it, with ONE
+ *                factor for the whole vector: ||v||_1 / d, or ||v||_2 / sqrt(d) with norm = DS_NORM_L2.  The
+ *                factor needs a sum over all of v first, so a pass is three kernels and reads its inputs
+ *                twice (about 20 bytes per entry on a worker instead of 12).
+ *
+ * DS_Q_TERNARY   the "QSGD" of Section 5.1 ("Implementations and setups", item 2): with m the entry of
+ *                largest absolute value of the whole vector, an entry e becomes sign(e) with probability
+ *                |e| / |m| and 0 otherwise; one factor, the l1 magnitude of v over that of the ternary
+ *                vector (||v||_1 / number of non-zeros), multiplies it.  The sign of an entry is the bit
+ *                (v >= 0).  Randomness: Philox4x32-10, key = seed, counter = (j/4, 0xFFFFFFFE, worker
+ *                index or 0xFFFFFFFF on the server pass, step); entry j uses output word j%4, top 24 bits,
+ *                as a uniform u in [0,1), and survives iff u < |e| / |m| (so the largest entry always
+ *                does).  chunk must be 0.  Five kernels per pass, inputs read three times.
+ *
  * Chunk reductions (sum of |v| or of v*v) are pairwise sums in index order over the chunk padded
- * with zeros to `chunk` entries, so results do not depend on launch geometry.
+ * with zeros to `chunk` entries (whole vector: to the next power of two at or above d), so results do not
+ * depend on launch geometry.
  */
-typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3, DS_Q_CLIP = 4, DS_Q_RSPARSE = 5 } ds_op;
+typedef enum {
+  DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3, DS_Q_CLIP = 4, DS_Q_RSPARSE = 5, DS_Q_TERNARY = 6
+} ds_op;
 
 /* ds_qspec.norm for DS_Q_SIGN1 */
 #define DS_NORM_L1 0u /* s_c = ||v_c||_1 / len_c (also selected by 1) */
@@ -121,19 +138,31 @@ typedef enum { DS_Q_IDENTITY = 0, DS_Q_SIGN1 = 1, DS_Q_TOPK = 2, DS_Q_QSGD = 3, 
 
 typedef struct {
   int32_t op;        /* ds_op */
-  uint32_t chunk;    /* SIGN1, QSGD, RSPARSE: a power of two in [128, 8192]; else ignored */
+  uint32_t chunk;    /* SIGN1, QSGD, RSPARSE: a power of two in [128, 8192]; SIGN1 also 0 = one factor for the
+                        whole vector; TERNARY: 0; else ignored */
   uint64_t k;        /* TOPK: 0 <= k <= d; else ignored */
   uint32_t levels;   /* QSGD: 1 <= levels <= 255; CLIP: bits set to zero, 16 or 24;
                         RSPARSE: S, a power of two in [2, 128]; else ignored */
   uint32_t norm;     /* SIGN1: DS_NORM_L1 (0 or 1) or DS_NORM_L2 (2); RSPARSE: DS_RSPARSE_*; else must be 0 */
 } ds_qspec;
 
+/*
+ * ds_config.flags.  DS_NO_COMPENSATION: the methods of Section 5.1 that compress without keeping the error
+ * ("Top-k SGD", item 5; "QSGD", item 2, with DS_Q_TERNARY workers and an IDENTITY server): a worker sends
+ * Q[g_i], the server sends Q[(1/n) sum_i Q[g_i]], x = x - gamma * that.  No error is read and none is
+ * written: delta_w is not used at all (delta_w_bytes is 0, the pointer may be NULL) and the worker pass
+ * moves 4 bytes per entry plus the payload instead of 12.  delta_s is likewise unused, except that a TOPK
+ * server pass lays its vector out there (delta_s then is scratch: required, never read back by a later
+ * step); for every other server operator delta_s_bytes is 0.
+ */
+#define DS_NO_COMPENSATION 0x1u
+
 typedef struct {
   uint32_t n;        /* workers, 1 <= n <= 65535 */
   uint32_t reserved; /* must be 0 */
   uint64_t d;        /* model dimension, 1 <= d < 2^32 */
   float gamma;       /* learning rate, finite */
-  uint32_t reserved2;
+  uint32_t flags;    /* DS_NO_COMPENSATION or 0 */
   ds_qspec worker_q; /* Q of the worker pass */
   ds_qspec server_q; /* Q of the server pass */
   uint64_t seed;     /* Philox key for DS_Q_QSGD */
@@ -146,7 +175,8 @@ typedef struct {
  *   delta_s  float[d]        server error; the caller zero-fills
  *   worker_payload           n payloads at a fixed stride, see ds_get_layout()
  *   server_payload           one payload
- *   workspace                scratch of the top-k path; may be NULL when workspace_bytes is 0.
+ *   workspace                scratch of the top-k path and of the whole-vector operators; may be NULL when
+ *                            workspace_bytes is 0.
  *                            Zero-fill it once.  Between calls it holds only hints (the previous
  *                            steps' threshold bins); whatever it holds, results are the same
  *   dev_status uint32[4]     the caller zero-fills (flags and counters, see DS_DEV_*)
@@ -176,6 +206,9 @@ typedef struct {
  *             [2] float  step[ceil(d/chunk)] (the grid step q = N_c / levels that multiplies the
  *                 levels; 0 for a chunk sent as all zeros)
  *   CLIP      [0] uint16 hi[d] (levels = 16) or uint8 hi[d] (levels = 24): bits(v) >> levels
+ *   SIGN1, chunk = 0: as SIGN1 with one float in scale
+ *   TERNARY   [0] uint32 sgn[ceil(d/32)] (bit = v >= 0)  [1] uint32 nz[ceil(d/32)] (bit = entry is non-zero)
+ *             [2] float  scale[1]
  *   RSPARSE   [0] float  val[ceil(d/chunk) * chunk/S]  slot j/S = Q[v]_j of the survivor j, +0 where j >= d
  *             [1] uint32 off[ceil(d/chunk)]            the draw o of every chunk
  */
@@ -239,9 +272,9 @@ int ds_destroy(ds_handle h);
  *   one ds_server_aggregate_compress bit for bit.
  * ds_apply_update_slice: x = x - gamma Q[v] on lo .. hi-1 from that slice of the server payload.
  *
- * Operators that act per chunk or per entry (IDENTITY, SIGN1, QSGD, CLIP) are supported on both
- * passes; a global TOPK on either pass, and RSPARSE, are DS_ERR_UNSUPPORTED here (its threshold is a property of
- * the whole vector).  These calls do not take part in the worker -> server -> apply order check
+ * Operators that act per chunk or per entry (IDENTITY, SIGN1 with a chunk, QSGD, CLIP) are supported on both
+ * passes; the operators that need a quantity of the whole vector (TOPK, SIGN1 with chunk = 0, TERNARY) on
+ * either pass, and RSPARSE, are DS_ERR_UNSUPPORTED here.  These calls do not take part in the worker -> server -> apply order check
  * of the whole-vector calls: the caller sequences its slices.  Errors as for the whole-vector calls.
  */
 #define DS_SLICE_ALIGN 8192u

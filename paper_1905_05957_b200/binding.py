@@ -20,7 +20,8 @@ DS_ERR_INVALID_ARG, DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL = -1, -2, -3
 DS_ERR_STATE, DS_ERR_CUDA, DS_ERR_UNSUPPORTED = -4, -5, -6
 DS_FUSE_APPLY = 1
 DS_DEV_TOPK_INCONSISTENT = 1
-OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4, "rsparse": 5}
+OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4, "rsparse": 5, "ternary": 6}
+DS_NO_COMPENSATION = 1
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
            "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
            "ds_kernel_launches", "ds_topk_worker_static", "ds_worker_compress_rows",
@@ -35,7 +36,7 @@ class ds_qspec(C.Structure):
 
 class ds_config(C.Structure):
     _fields_ = [("n", C.c_uint32), ("reserved", C.c_uint32), ("d", C.c_uint64), ("gamma", C.c_float),
-                ("reserved2", C.c_uint32), ("worker_q", ds_qspec), ("server_q", ds_qspec), ("seed", C.c_uint64)]
+                ("flags", C.c_uint32), ("worker_q", ds_qspec), ("server_q", ds_qspec), ("seed", C.c_uint64)]
 
 
 class ds_buffers(C.Structure):
@@ -95,8 +96,8 @@ def _qspec(q: Q) -> ds_qspec:
     return ds_qspec(OPS[q.op], q.chunk, q.k, levels, norm)
 
 
-def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int) -> ds_config:
-    return ds_config(n, 0, d, gamma, 0, _qspec(worker_q), _qspec(server_q), seed)
+def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int, compensate: bool = True) -> ds_config:
+    return ds_config(n, 0, d, gamma, 0 if compensate else DS_NO_COMPENSATION, _qspec(worker_q), _qspec(server_q), seed)
 
 
 def get_layout(cfg: ds_config, which: int) -> ds_payload_layout:
@@ -113,6 +114,7 @@ _VIEW_DTYPES = {
     "topk": (("idx", torch.int32), ("val", torch.float32)),
     "qsgd": (("lvl", torch.uint8), ("sgn", torch.int32), ("step", torch.float32)),
     "rsparse": (("val", torch.float32), ("off", torch.int32)),
+    "ternary": (("sgn", torch.int32), ("nz", torch.int32), ("scale", torch.float32)),
     "clip": (("hi", torch.int16),),      # 8-bit entries when 24 bits are cleared, see payload_views
 }
 
@@ -159,8 +161,10 @@ class DoubleSqueeze:
 
     def __init__(self, n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int = 0,
                  device: str | torch.device = "cuda", x0: torch.Tensor | None = None, guard: bool = False,
-                 payload_fill: int = 0):
-        """guard=True surrounds every buffer handed to the library with GUARD_BYTES sentinel bytes
+                 payload_fill: int = 0, compensate: bool = True):
+        """compensate=False: the methods of Section 5.1 that keep no error (DS_NO_COMPENSATION): delta_w
+        and delta_s are then empty tensors unless the library asks for delta_s as scratch.
+        guard=True surrounds every buffer handed to the library with GUARD_BYTES sentinel bytes
         (check_guards() tells whether any was overwritten): a debugging aid for out-of-bounds writes.
         payload_fill: byte the payload buffers start out with (the library must overwrite every byte
         it defines whatever they held)."""
@@ -170,7 +174,8 @@ class DoubleSqueeze:
         self.device = torch.device(device)
         self.n, self.d, self.gamma, self.seed = n, d, gamma, seed
         self.worker_q, self.server_q = worker_q, server_q
-        self.cfg = make_config(n, d, gamma, worker_q, server_q, seed)
+        self.compensate = compensate
+        self.cfg = make_config(n, d, gamma, worker_q, server_q, seed, compensate)
         bufs = ds_buffers()
         rc = self.lib.ds_create(C.byref(self.cfg), C.byref(bufs), None)
         if rc != DS_NEED_BUFFERS:
@@ -192,13 +197,15 @@ class DoubleSqueeze:
         self.x = alloc(d * 4).view(torch.float32)
         if x0 is not None:
             self.x.copy_(x0.to(device=dev, dtype=torch.float32).reshape(-1))
-        self.delta_w = alloc(n * d * 4).view(torch.float32).view(n, d)
-        self.delta_s = alloc(d * 4).view(torch.float32)
+        self.delta_w = alloc(bufs.delta_w_bytes).view(torch.float32).view(n, bufs.delta_w_bytes // (4 * n))
+        self.delta_s = alloc(bufs.delta_s_bytes).view(torch.float32)
         self.worker_payload = alloc(bufs.worker_payload_bytes, payload_fill)
         self.server_payload = alloc(bufs.server_payload_bytes, payload_fill)
         self.workspace = alloc(max(bufs.workspace_bytes, 16))
         self.dev_status = alloc(16).view(torch.int32)
-        bufs.x, bufs.delta_w, bufs.delta_s = self.x.data_ptr(), self.delta_w.data_ptr(), self.delta_s.data_ptr()
+        bufs.x = self.x.data_ptr()
+        bufs.delta_w = self.delta_w.data_ptr() if bufs.delta_w_bytes else None
+        bufs.delta_s = self.delta_s.data_ptr() if bufs.delta_s_bytes else None
         bufs.worker_payload, bufs.server_payload = self.worker_payload.data_ptr(), self.server_payload.data_ptr()
         bufs.workspace, bufs.dev_status = self.workspace.data_ptr(), self.dev_status.data_ptr()
         self.bufs = bufs
@@ -221,7 +228,7 @@ class DoubleSqueeze:
 
     @classmethod
     def for_workload(cls, wl: Workload, device="cuda") -> "DoubleSqueeze":
-        return cls(wl.n, wl.d, wl.gamma, wl.worker_q, wl.server_q, wl.seed, device)
+        return cls(wl.n, wl.d, wl.gamma, wl.worker_q, wl.server_q, wl.seed, device, compensate=wl.compensate)
 
     # -- the three calls of one iteration -----------------------------------------------------
     def _stream(self, stream) -> int:

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(CSRC, "libdsq.so")
 SOURCES = ["dsq_api.cu", "dsq_chunked.cu", "dsq_chunked_sign.cu", "dsq_chunked_sign_l2.cu", "dsq_chunked_qsgd.cu", "dsq_chunked_qsgd_window.cu",
-           "dsq_elementwise.cu", "dsq_topk.cu", "dsq_static.cu"]
+           "dsq_elementwise.cu", "dsq_topk.cu", "dsq_static.cu", "dsq_whole.cu"]
 HEADERS = ["dsq_common.cuh", "dsq_chunked.cuh", "dsq_internal.h", os.path.join("..", "..", "include", "dsq.h")]
 
 NVCC_FLAGS = [

@@ -35,7 +35,8 @@ bool qspec_ok(const ds_qspec& q, uint64_t d) {
     return false;
   switch (q.op) {
     case DS_Q_IDENTITY: return true;
-    case DS_Q_SIGN1: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192;
+    case DS_Q_SIGN1: return q.chunk == 0 || (is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192);
+    case DS_Q_TERNARY: return q.chunk == 0;
     case DS_Q_QSGD: return is_pow2(q.chunk) && q.chunk >= 128 && q.chunk <= 8192 && q.levels >= 1 && q.levels <= 255;
     case DS_Q_TOPK: return q.k <= d;
     case DS_Q_CLIP: return q.levels == 16 || q.levels == 24;
@@ -47,11 +48,16 @@ bool qspec_ok(const ds_qspec& q, uint64_t d) {
 
 bool config_ok(const ds_config* c) {
   if (!c) return false;
-  if (c->n < 1 || c->n > 65535 || c->reserved != 0) return false;
+  if (c->n < 1 || c->n > 65535 || c->reserved != 0 || (c->flags & ~DS_NO_COMPENSATION)) return false;
   if (c->d < 1 || c->d >= (1ull << 32)) return false;
   if (!std::isfinite(c->gamma)) return false;
   return qspec_ok(c->worker_q, c->d) && qspec_ok(c->server_q, c->d);
 }
+
+// Operators whose scaling factor belongs to the whole vector (several kernels per pass, not sliceable).
+bool whole_vector(const ds_qspec& q) { return (q.op == DS_Q_SIGN1 && q.chunk == 0) || q.op == DS_Q_TERNARY; }
+
+bool no_compensation(const ds_config& c) { return (c.flags & DS_NO_COMPENSATION) != 0; }
 
 void layout_of(const ds_qspec& q, uint64_t d, ds_payload_layout* L) {
   memset(L, 0, sizeof *L);
@@ -64,7 +70,8 @@ void layout_of(const ds_qspec& q, uint64_t d, ds_payload_layout* L) {
   };
   switch (q.op) {
     case DS_Q_IDENTITY: put(0, d, 4); break;
-    case DS_Q_SIGN1: put(0, nw, 4); put(1, (d + q.chunk - 1) / q.chunk, 4); break;
+    case DS_Q_SIGN1: put(0, nw, 4); put(1, q.chunk ? (d + q.chunk - 1) / q.chunk : 1, 4); break;
+    case DS_Q_TERNARY: put(0, nw, 4); put(1, nw, 4); put(2, 1, 4); break;
     case DS_Q_TOPK: put(0, q.k, 4); put(1, q.k, 4); break;
     case DS_Q_QSGD: put(0, d, 1); put(1, nw, 4); put(2, (d + q.chunk - 1) / q.chunk, 4); break;
     case DS_Q_CLIP: put(0, d, (32 - q.levels) / 8); break;
@@ -82,6 +89,7 @@ struct ds_ctx {
   TopkPlan wplan, splan;  // workspace carving of the top-k path (worker rows / server row)
   float* acc;             // dense accumulator for sparse worker payloads (inside workspace), or NULL
   uint32_t* acc_offsets;  // span offsets of the sparse payloads (inside workspace), or NULL
+  void* whole;            // scratch of the operators with one factor per vector (inside workspace), or NULL
   int phase;              // 0: step complete, 1: worker pass done, 2: unfused server pass done
 };
 
@@ -121,6 +129,12 @@ uint64_t plan_workspace(ds_ctx* c) {
     c->splan.pred = ws ? reinterpret_cast<TopkPred*>(ws + total) : nullptr;
     total += round16(sizeof(TopkPred));
   }
+  // tile sums of the operators with one factor per vector (the two passes run one after the other)
+  uint64_t whole_bytes = 0;
+  if (whole_vector(cfg.worker_q)) whole_bytes = whole_workspace_bytes(cfg.d, cfg.n);
+  if (whole_vector(cfg.server_q) && whole_workspace_bytes(cfg.d, 1) > whole_bytes) whole_bytes = whole_workspace_bytes(cfg.d, 1);
+  c->whole = (whole_bytes && ws) ? ws + total : nullptr;
+  total += round16(whole_bytes);
   return total;
 }
 
@@ -128,7 +142,7 @@ SrcParams worker_src(const ds_ctx* c, const float* g) {
   SrcParams s;
   memset(&s, 0, sizeof s);
   s.g = g;
-  s.delta = c->buf.delta_w;
+  s.delta = no_compensation(c->cfg) ? nullptr : c->buf.delta_w;
   s.d = c->cfg.d;
   s.n = c->cfg.n;
   s.vec = (c->cfg.d % 4 == 0) && aligned16(g);
@@ -139,7 +153,7 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
   SrcParams s;
   memset(&s, 0, sizeof s);
   const ds_qspec& wq = c->cfg.worker_q;
-  s.delta = c->buf.delta_s;
+  s.delta = no_compensation(c->cfg) ? nullptr : c->buf.delta_s;   // NULL: v is the plain mean
   s.d = c->cfg.d;
   s.n = c->cfg.n;
   s.inv_n = 1.0f / (float)c->cfg.n;
@@ -147,6 +161,7 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
   s.wp_stride = c->wl.stride;
   for (int i = 0; i < 3; ++i) s.wp_off[i] = c->wl.off[i];
   s.w_log2_chunk = (wq.op == DS_Q_SIGN1 || wq.op == DS_Q_QSGD || wq.op == DS_Q_RSPARSE) ? log2u(wq.chunk) : 0;
+  if (whole_vector(wq)) s.w_log2_chunk = 32;   // every entry (d < 2^32) reads factor number 0
   s.w_log2_keep = wq.op == DS_Q_RSPARSE ? log2u(wq.levels) : 0;
   s.w_levels = (float)wq.levels;
   s.w_clip_bits = wq.op == DS_Q_CLIP ? wq.levels : 0;
@@ -158,6 +173,7 @@ SrcParams server_src(const ds_ctx* c, int* kind) {
     case DS_Q_TOPK: *kind = SRC_SRV_TOPK; break;
     case DS_Q_CLIP: *kind = SRC_SRV_CLIP; break;
     case DS_Q_RSPARSE: *kind = SRC_SRV_RSPARSE; break;
+    case DS_Q_TERNARY: *kind = SRC_SRV_TERNARY; break;
     default: *kind = SRC_SRV_QSGD; break;
   }
   return s;
@@ -185,7 +201,28 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       e = launch_identity(src_kind, src, reinterpret_cast<float*>(payload + L.off[0]) + lo, L.stride / 4, delta, row_stride,
                           x_fused, c->cfg.gamma, rows, st);
       break;
+    case DS_Q_TERNARY:
     case DS_Q_SIGN1:
+      if (whole_vector(q)) {
+        if (win) return DS_ERR_UNSUPPORTED;
+        WholeParams wp;
+        memset(&wp, 0, sizeof wp);
+        wp.out_sgn = reinterpret_cast<uint32_t*>(payload + L.off[0]);
+        wp.out_nz = q.op == DS_Q_TERNARY ? reinterpret_cast<uint32_t*>(payload + L.off[1]) : nullptr;
+        wp.out_scale = reinterpret_cast<float*>(payload + L.off[q.op == DS_Q_TERNARY ? 2 : 1]);
+        wp.word_stride = L.stride / 4;
+        wp.delta_out = delta;
+        wp.delta_row_stride = row_stride;
+        wp.x = x_fused;
+        wp.gamma = c->cfg.gamma;
+        wp.keys = philox_key_schedule((uint32_t)(c->cfg.seed & 0xFFFFFFFFu), (uint32_t)(c->cfg.seed >> 32));
+        wp.step = step;
+        wp.server_pass = server ? 1u : 0u;
+        wp.l2 = (q.op == DS_Q_SIGN1 && q.norm == DS_NORM_L2) ? 1u : 0u;
+        e = launch_whole(q.op, src_kind, src, wp, c->whole, rows, st);
+        break;
+      }
+      // fall through: the 1-bit operator with a factor per chunk
     case DS_Q_QSGD: {
       ChunkParams p;
       memset(&p, 0, sizeof p);
@@ -222,6 +259,13 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       io.val = reinterpret_cast<float*>(payload + L.off[1]);
       io.payload_stride = L.stride;
       io.v_inout = delta;  // v is written over delta, then the kept entries are zeroed: delta = v - Q[v]
+      io.keep_error = 1;
+      if (src_kind == SRC_WORKER_PLAIN) {
+        // no error is kept: v is the gradient itself, selected where it lies and never written
+        if (q.k == 0) return DS_OK;  // nothing to send, nothing to keep
+        io.v_inout = const_cast<float*>(src.g);
+        io.keep_error = 0;
+      }
       io.x = x_fused;
       io.gamma = c->cfg.gamma;
       io.dev_status = c->buf.dev_status;
@@ -278,7 +322,11 @@ int ds_create(const ds_config* cfg, ds_buffers* bufs, ds_handle* out) {
   tmp.buf = *bufs;
   layout_of(cfg->worker_q, cfg->d, &tmp.wl);
   layout_of(cfg->server_q, cfg->d, &tmp.sl);
-  const uint64_t need_x = cfg->d * 4, need_dw = (uint64_t)cfg->n * cfg->d * 4, need_ds = cfg->d * 4;
+  // without compensation no error is carried: delta_w is not needed at all, delta_s only as the place
+  // where a top-k server pass lays out its vector
+  const bool nocomp = no_compensation(*cfg);
+  const uint64_t need_x = cfg->d * 4, need_dw = nocomp ? 0 : (uint64_t)cfg->n * cfg->d * 4;
+  const uint64_t need_ds = (nocomp && cfg->server_q.op != DS_Q_TOPK) ? 0 : cfg->d * 4;
   const uint64_t need_wp = (uint64_t)cfg->n * tmp.wl.stride, need_sp = tmp.sl.stride;
   const uint64_t need_ws = plan_workspace(&tmp);
   if (bufs->x == nullptr) {  // query mode
@@ -291,7 +339,8 @@ int ds_create(const ds_config* cfg, ds_buffers* bufs, ds_handle* out) {
     return DS_NEED_BUFFERS;
   }
   if (!out) return DS_ERR_INVALID_ARG;
-  if (!bufs->delta_w || !bufs->delta_s || !bufs->worker_payload || !bufs->server_payload || !bufs->dev_status)
+  if ((need_dw && !bufs->delta_w) || (need_ds && !bufs->delta_s) || !bufs->worker_payload || !bufs->server_payload ||
+      !bufs->dev_status)
     return DS_ERR_INVALID_ARG;
   if (need_ws && !bufs->workspace) return DS_ERR_INVALID_ARG;
   const void* ptrs[] = {bufs->x, bufs->delta_w, bufs->delta_s, bufs->worker_payload, bufs->server_payload, bufs->workspace};
@@ -315,8 +364,10 @@ int ds_worker_compress(ds_handle h, const float* g, uint32_t step, void* cuda_st
   if (h->phase != 0) return DS_ERR_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const SrcParams src = worker_src(h, g);
-  const int rc = run_pass(h, SRC_WORKER, src, h->cfg.worker_q, h->wl, static_cast<uint8_t*>(h->buf.worker_payload),
-                          h->buf.delta_w, h->cfg.n, false, nullptr, step, st);
+  const bool nocomp = no_compensation(h->cfg);
+  const int rc = run_pass(h, nocomp ? SRC_WORKER_PLAIN : SRC_WORKER, src, h->cfg.worker_q, h->wl,
+                          static_cast<uint8_t*>(h->buf.worker_payload), nocomp ? nullptr : h->buf.delta_w, h->cfg.n, false,
+                          nullptr, step, st);
   if (rc == DS_OK) h->phase = 1;
   return rc;
 }
@@ -335,8 +386,11 @@ int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, voi
     if (e != cudaSuccess) return cuda_fail(e, "sparse accumulate");
   }
   const bool fuse = (flags & DS_FUSE_APPLY) != 0;
-  const int rc = run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload),
-                          h->buf.delta_s, 1, true, fuse ? h->buf.x : nullptr, step, st);
+  // without compensation the residual has no destination -- except that a top-k pass still lays its
+  // vector out in delta_s (which is then scratch: never read back)
+  float* ds_out = (no_compensation(h->cfg) && h->cfg.server_q.op != DS_Q_TOPK) ? nullptr : h->buf.delta_s;
+  const int rc = run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload), ds_out, 1, true,
+                          fuse ? h->buf.x : nullptr, step, st);
   if (rc == DS_OK) h->phase = fuse ? 0 : 2;
   return rc;
 }
@@ -351,6 +405,7 @@ int ds_apply_update(ds_handle h, void* cuda_stream) {
   pv.base = static_cast<const uint8_t*>(h->buf.server_payload);
   for (int i = 0; i < 3; ++i) pv.off[i] = h->sl.off[i];
   pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD || q.op == DS_Q_RSPARSE) ? log2u(q.chunk) : 0;
+  if (whole_vector(q)) pv.log2_chunk = 32;   // one factor: every entry reads number 0
   pv.levels_f = (float)q.levels;
   pv.clip_bits = q.op == DS_Q_CLIP ? q.levels : 0;
   pv.log2_keep = q.op == DS_Q_RSPARSE ? log2u(q.levels) : 0;
@@ -368,7 +423,7 @@ bool slice_ok(const ds_ctx* h, uint64_t lo, uint64_t hi) {
   return lo < hi && hi <= d && lo % DS_SLICE_ALIGN == 0 && (hi == d || hi % DS_SLICE_ALIGN == 0);
 }
 
-bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK && q.op != DS_Q_RSPARSE; }
+bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK && q.op != DS_Q_RSPARSE && !whole_vector(q); }
 
 }  // namespace
 
@@ -378,12 +433,14 @@ int ds_worker_compress_rows(ds_handle h, const float* g, uint32_t row0, uint32_t
   if (!sliceable(h->cfg.worker_q)) return DS_ERR_UNSUPPORTED;
   const uint64_t d = h->cfg.d;
   SrcParams src = worker_src(h, g);
-  src.delta = h->buf.delta_w + (uint64_t)row0 * d;
+  const bool nocomp = no_compensation(h->cfg);
+  float* delta_rows = nocomp ? nullptr : h->buf.delta_w + (uint64_t)row0 * d;
+  src.delta = delta_rows;
   src.vec = (d % 4 == 0) && aligned16(g);
   const PassWindow win{d, 0, row0};
-  return run_pass(h, SRC_WORKER, src, h->cfg.worker_q, h->wl,
-                  static_cast<uint8_t*>(h->buf.worker_payload) + (uint64_t)row0 * h->wl.stride,
-                  h->buf.delta_w + (uint64_t)row0 * d, nrows, false, nullptr, step, static_cast<cudaStream_t>(cuda_stream), &win);
+  return run_pass(h, nocomp ? SRC_WORKER_PLAIN : SRC_WORKER, src, h->cfg.worker_q, h->wl,
+                  static_cast<uint8_t*>(h->buf.worker_payload) + (uint64_t)row0 * h->wl.stride, delta_rows, nrows, false, nullptr,
+                  step, static_cast<cudaStream_t>(cuda_stream), &win);
 }
 
 int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flags, uint64_t lo, uint64_t hi,
@@ -395,7 +452,8 @@ int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flag
   const ds_qspec& wq = h->cfg.worker_q;
   // the slice of every worker payload: shift each sub-array to entry lo
   src.d = hi - lo;
-  src.delta = h->buf.delta_s + lo;
+  float* ds_slice = no_compensation(h->cfg) ? nullptr : h->buf.delta_s + lo;
+  src.delta = ds_slice;
   switch (wq.op) {
     case DS_Q_IDENTITY: src.wp_off[0] += lo * 4; break;
     case DS_Q_SIGN1: src.wp_off[0] += lo / 8; src.wp_off[1] += lo / wq.chunk * 4; break;
@@ -405,7 +463,7 @@ int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flag
   }
   const PassWindow win{hi - lo, lo, 0};
   const bool fuse = (flags & DS_FUSE_APPLY) != 0;
-  return run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload), h->buf.delta_s + lo, 1,
+  return run_pass(h, kind, src, h->cfg.server_q, h->sl, static_cast<uint8_t*>(h->buf.server_payload), ds_slice, 1,
                   true, fuse ? h->buf.x + lo : nullptr, step, static_cast<cudaStream_t>(cuda_stream), &win);
 }
 

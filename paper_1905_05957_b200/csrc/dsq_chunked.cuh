@@ -86,11 +86,39 @@ __device__ __forceinline__ uint32_t octet_sign_words(const uint32_t (&nib)[V], u
   return x;
 }
 
+// Pairwise sum over a chunk: part[j] is the calling thread's sum over its float4 number j (entries
+// (j*G + t)*4 .. +3 of the chunk, already added as (a+b)+(c+d)).  Every thread of the chunk returns the
+// chunk total.  Called by all threads of the CTA (one barrier when the chunk spans several warps).
+template <int V, int LOG2G>
+__device__ __forceinline__ float chunk_total(float (&part)[V], float* s_red) {
+  constexpr uint32_t G = 1u << LOG2G;
+  constexpr uint32_t NG = (V * G) >> 5;   // 128-entry groups per chunk
+  const uint32_t tid = threadIdx.x, lane = tid & 31u;
+  const uint32_t sub = tid >> LOG2G, t = tid & (G - 1u);
+  float total = warp_rows_sum<V>(part, lane);  // lane holds the 128-entry group sum of row lane % V
+  if constexpr (NG > 1) {
+    // group index inside the chunk: row j = lane, warp (t >> 5) of the row
+    if (lane < (uint32_t)V) s_red[sub * NG + lane * (G >> 5) + (t >> 5)] = total;
+    __syncthreads();
+    float x;
+    if constexpr (NG <= 32) {
+      x = lane < NG ? s_red[sub * NG + lane] : 0.f;
+#pragma unroll
+      for (uint32_t o = 1; o < NG; o <<= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
+    } else {  // NG == 64
+      x = __fadd_rn(s_red[sub * 64 + 2 * lane], s_red[sub * 64 + 2 * lane + 1]);
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
+    }
+    total = __shfl_sync(0xffffffffu, x, 0);
+  }
+  return total;
+}
+
 template <int OP, int SRC, int V, int LOG2G, bool FULL>
 __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkParams& p, float* s_red, float* s_scal) {
   constexpr uint32_t G = 1u << LOG2G;
   constexpr uint32_t L = (uint32_t)V * G * 4u;
-  constexpr uint32_t NG = (V * G) >> 5;   // 128-entry groups per chunk
   constexpr uint32_t CPC = kThreads / G;  // chunks per CTA
   const uint32_t tid = threadIdx.x, lane = tid & 31u;
   const uint32_t sub = tid >> LOG2G, t = tid & (G - 1u);
@@ -126,7 +154,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
   }
 
   // fused model update (server pass): fetch x now so that its latency hides behind the reduction
-  constexpr bool kServer = SRC != SRC_WORKER;  // only a server pass can carry the update
+  constexpr bool kServer = !is_worker_src(SRC);  // only a server pass can carry the update
   float4 xv[kServer ? V : 1];
   if (kServer && p.x) {
 #pragma unroll
@@ -147,23 +175,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
     }
     part[j] = __fadd_rn(__fadd_rn(m0, m1), __fadd_rn(m2, m3));
   }
-  float total = warp_rows_sum<V>(part, lane);  // lane holds the 128-entry group sum of row lane % V
-  if constexpr (NG > 1) {
-    // group index inside the chunk: row j = lane, warp (t >> 5) of the row
-    if (lane < (uint32_t)V) s_red[sub * NG + lane * (G >> 5) + (t >> 5)] = total;
-    __syncthreads();
-    float x;
-    if constexpr (NG <= 32) {
-      x = lane < NG ? s_red[sub * NG + lane] : 0.f;
-#pragma unroll
-      for (uint32_t o = 1; o < NG; o <<= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
-    } else {  // NG == 64
-      x = __fadd_rn(s_red[sub * 64 + 2 * lane], s_red[sub * 64 + 2 * lane + 1]);
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
-    }
-    total = __shfl_sync(0xffffffffu, x, 0);
-  }
+  const float total = chunk_total<V, LOG2G>(part, s_red);
 
   // ---- per-chunk quantities
   const uint32_t len = FULL ? L : (chunk_live ? (uint32_t)min((uint64_t)L, d - base) : 1u);
@@ -255,11 +267,15 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
     if constexpr (!FULL) nib[j] &= (1u << cnt[j]) - 1u;  // pad bits are 0
 
     if (cnt[j]) {
-      const float4 dl = sub4_rn(v[j], C);
-      if constexpr (FULL) {
-        st_stream4(delta_chunk + tq * 4u, dl);
-      } else {
-        store_row4(delta_chunk, (uint64_t)tq * 4u, cnt[j], src.vec, dl);
+      // the residual (Eq. 3 / Eq. 4) -- unless no error is carried: a plain worker never keeps one, a
+      // server pass without compensation has no destination for it
+      if (SRC != SRC_WORKER_PLAIN && (SRC == SRC_WORKER || p.delta_out)) {
+        const float4 dl = sub4_rn(v[j], C);
+        if constexpr (FULL) {
+          st_stream4(delta_chunk + tq * 4u, dl);
+        } else {
+          store_row4(delta_chunk, (uint64_t)tq * 4u, cnt[j], src.vec, dl);
+        }
       }
       if (kServer && p.x) {  // fused model update (server pass only): x = x - gamma * Q[v]
         const float4 xo = xv[kServer ? j : 0];
@@ -285,7 +301,7 @@ __device__ __forceinline__ void chunk_body(const SrcParams& src, const ChunkPara
 // registers, what the whole-vector kernel gets by itself; with 48 it measured 8 % slower).  Server
 // passes see kServerCtasPerSm.
 constexpr int chunk_ctas(int op, int src, int v) {
-  if (src == SRC_WORKER) return (op == kOpQsgdWindow && v <= 2) ? 6 : 0;
+  if (is_worker_src(src)) return (op == kOpQsgdWindow && v <= 2) ? 6 : 0;
   return v >= 8 ? 2 : kServerCtasPerSm;
 }
 
@@ -333,6 +349,8 @@ cudaError_t launch_src(int srck, const SrcParams& src, const ChunkParams& p, uin
     case SRC_SRV_QSGD: return launch_v<OP, SRC_SRV_QSGD>(src, p, rows, chunk, st);
     case SRC_SRV_CLIP: return launch_v<OP, SRC_SRV_CLIP>(src, p, rows, chunk, st);
     case SRC_SRV_RSPARSE: return launch_v<OP, SRC_SRV_RSPARSE>(src, p, rows, chunk, st);
+    case SRC_WORKER_PLAIN: return launch_v<OP, SRC_WORKER_PLAIN>(src, p, rows, chunk, st);
+    case SRC_SRV_TERNARY: return launch_v<OP, SRC_SRV_TERNARY>(src, p, rows, chunk, st);
   }
   return cudaErrorInvalidValue;
 }

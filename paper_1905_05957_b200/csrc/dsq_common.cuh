@@ -31,12 +31,16 @@ enum Src : int {
   SRC_SRV_QSGD = 4,
   SRC_SRV_CLIP = 5,      // payload = the high bits of every entry
   SRC_SRV_RSPARSE = 6,   // payload = the survivors of every chunk and the chunk's draw
+  SRC_WORKER_PLAIN = 7,  // v = g[row]: a worker that keeps no error (no compensation)
+  SRC_SRV_TERNARY = 8,   // payload = sign words, non-zero words and one factor per worker
 };
+
+__host__ __device__ constexpr bool is_worker_src(int src) { return src == SRC_WORKER || src == SRC_WORKER_PLAIN; }
 
 // Where v comes from.  Worker payload sub-arrays follow the documented payload layout.
 struct SrcParams {
   const float* g;          // worker: gradients [n, d]
-  const float* delta;      // worker: delta_w [n, d]; server: delta_s [d]
+  const float* delta;      // worker: delta_w [n, d]; server: delta_s [d], or NULL: no error is carried (v is the plain mean)
   uint64_t d;
   uint32_t n;              // server: number of payloads to average
   float inv_n;             // server: 1/n rounded once
@@ -142,13 +146,17 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
 #pragma unroll
     for (int j = 0; j < V; ++j)
       v[j] = add4_rn(a[j], b[j]);
+  } else if constexpr (SRC == SRC_WORKER_PLAIN) {
+    const uint64_t off = (uint64_t)row * p.d;
+#pragma unroll
+    for (int j = 0; j < V; ++j) v[j] = load_row4(p.g + off, e[j], cnt[j], p.vec);
   } else {
     const uint32_t lane = threadIdx.x & 31u;
     float4 acc[V], ds[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) {
       acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      ds[j] = load_row4(p.delta, e[j], cnt[j], p.vec);
+      ds[j] = p.delta ? load_row4(p.delta, e[j], cnt[j], p.vec) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if constexpr (SRC == SRC_SRV_IDENTITY) {
       for (uint32_t i = 0; i < p.n; ++i) {
@@ -161,13 +169,14 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
           acc[j] = add4_rn(acc[j], ci[j]);
         }
       }
-    } else if constexpr (SRC == SRC_SRV_SIGN1 || SRC == SRC_SRV_QSGD) {
-      constexpr int kSgn = SRC == SRC_SRV_SIGN1 ? 0 : 1;    // payload sub-array of the sign words
-      constexpr int kScl = SRC == SRC_SRV_SIGN1 ? 1 : 2;    // ... of the per-chunk scale / grid step
+    } else if constexpr (SRC == SRC_SRV_SIGN1 || SRC == SRC_SRV_QSGD || SRC == SRC_SRV_TERNARY) {
+      constexpr int kSgn = SRC == SRC_SRV_QSGD ? 1 : 0;     // payload sub-array of the sign words
+      constexpr int kScl = SRC == SRC_SRV_SIGN1 ? 1 : 2;    // ... of the per-chunk scale / grid step / factor
       const uint64_t nw = (p.d + 31) >> 5;
       const uint32_t sh = (lane & 7u) * 4u;                 // this lane's nibble inside its word
       for (uint32_t i0 = 0; i0 < p.n; i0 += 8) {
         uint32_t wreg[V];
+        uint32_t zreg[SRC == SRC_SRV_TERNARY ? V : 1];      // ternary: words of the non-zero plane
         float sreg[V];
         uint32_t lv[SRC == SRC_SRV_QSGD ? V : 1][SRC == SRC_SRV_QSGD ? 8 : 1];
 #pragma unroll
@@ -180,6 +189,11 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
           sreg[j] = 0.f;
           if (wi < p.n && word < nw)
             wreg[j] = __ldg(reinterpret_cast<const uint32_t*>(p.wp + wi * p.wp_stride + p.wp_off[kSgn]) + word);
+          if constexpr (SRC == SRC_SRV_TERNARY) {
+            zreg[j] = 0;
+            if (wi < p.n && word < nw)
+              zreg[j] = __ldg(reinterpret_cast<const uint32_t*>(p.wp + wi * p.wp_stride + p.wp_off[1]) + word);
+          }
           if (lane < 8 && i0 + lane < p.n && e0 < p.d)
             sreg[j] = __ldg(reinterpret_cast<const float*>(p.wp + (i0 + lane) * p.wp_stride + p.wp_off[kScl]) +
                             (e0 >> p.w_log2_chunk));
@@ -202,6 +216,11 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
               if constexpr (SRC == SRC_SRV_SIGN1) {
                 acc[j] = add4_rn(acc[j], make_float4(signed_by_bit(sc, ww, 0), signed_by_bit(sc, ww, 1),
                                                      signed_by_bit(sc, ww, 2), signed_by_bit(sc, ww, 3)));
+              } else if constexpr (SRC == SRC_SRV_TERNARY) {
+                // +-factor where the entry's non-zero bit is set, +0 elsewhere
+                const uint32_t zz = __shfl_sync(0xffffffffu, zreg[j], u * 4 + (lane >> 3)) >> sh;
+                acc[j] = add4_rn(acc[j], make_float4((zz & 1u) ? signed_by_bit(sc, ww, 0) : 0.f, (zz & 2u) ? signed_by_bit(sc, ww, 1) : 0.f,
+                                                     (zz & 4u) ? signed_by_bit(sc, ww, 2) : 0.f, (zz & 8u) ? signed_by_bit(sc, ww, 3) : 0.f));
               } else {
                 const uint32_t l4 = lv[j][u];
                 const float4 mag = mul4_rn(make_float4(byte_to_float(l4, 0), byte_to_float(l4, 1), byte_to_float(l4, 2),
@@ -300,8 +319,13 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
 #pragma unroll
     for (int j = 0; j < V; ++j) {
       // scalar on purpose: a packed multiply feeding a packed add was seen to come out fused
-      v[j].x = __fadd_rn(__fmul_rn(acc[j].x, p.inv_n), ds[j].x); v[j].y = __fadd_rn(__fmul_rn(acc[j].y, p.inv_n), ds[j].y);
-      v[j].z = __fadd_rn(__fmul_rn(acc[j].z, p.inv_n), ds[j].z); v[j].w = __fadd_rn(__fmul_rn(acc[j].w, p.inv_n), ds[j].w);
+      if (p.delta) {
+        v[j].x = __fadd_rn(__fmul_rn(acc[j].x, p.inv_n), ds[j].x); v[j].y = __fadd_rn(__fmul_rn(acc[j].y, p.inv_n), ds[j].y);
+        v[j].z = __fadd_rn(__fmul_rn(acc[j].z, p.inv_n), ds[j].z); v[j].w = __fadd_rn(__fmul_rn(acc[j].w, p.inv_n), ds[j].w);
+      } else {  // no error is carried: the plain mean, with no addition at all
+        v[j].x = __fmul_rn(acc[j].x, p.inv_n); v[j].y = __fmul_rn(acc[j].y, p.inv_n);
+        v[j].z = __fmul_rn(acc[j].z, p.inv_n); v[j].w = __fmul_rn(acc[j].w, p.inv_n);
+      }
       // entries past the end must read as +0 whatever the payload padding holds
       if (cnt[j] < 4) {
 #pragma unroll

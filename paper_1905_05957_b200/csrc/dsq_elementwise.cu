@@ -6,6 +6,13 @@
 
 namespace dsq {
 
+// Whether a pass writes a residual: a worker with error feedback always does, a worker without
+// compensation never, a server pass when it was given a destination.
+template <int SRC>
+__device__ __forceinline__ bool keeps_error(const float* delta_out) {
+  return SRC != SRC_WORKER_PLAIN && (SRC == SRC_WORKER || delta_out != nullptr);
+}
+
 template <int SRC>
 __global__ void __launch_bounds__(kThreads) k_identity(const SrcParams src, float* out_c, uint64_t c_row_stride,
                                                        float* delta_out, uint64_t delta_row_stride, float* x,
@@ -24,7 +31,7 @@ __global__ void __launch_bounds__(kThreads) k_identity(const SrcParams src, floa
     const float4 v = vv[0];
     if (!cnt) continue;
     store_row4(out_c + (uint64_t)row * c_row_stride, e, cnt, 1, v);  // Q[v] = v
-    store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, make_float4(0.f, 0.f, 0.f, 0.f));
+    if (keeps_error<SRC>(delta_out)) store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, make_float4(0.f, 0.f, 0.f, 0.f));
     if (x) {
       float4 xv = load_row4(x, e, cnt, 1);
       xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, v.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, v.y));
@@ -44,16 +51,7 @@ cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64
                             uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st) {
   dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
 #define DSQ_ID(S) launch_pdl(k_identity<S>, grid, kThreads, st, src, out_c, c_row_stride, delta_out, delta_row_stride, x, gamma)
-  switch (srck) {
-    case SRC_WORKER: DSQ_ID(SRC_WORKER); break;
-    case SRC_SRV_IDENTITY: DSQ_ID(SRC_SRV_IDENTITY); break;
-    case SRC_SRV_SIGN1: DSQ_ID(SRC_SRV_SIGN1); break;
-    case SRC_SRV_TOPK: DSQ_ID(SRC_SRV_TOPK); break;
-    case SRC_SRV_QSGD: DSQ_ID(SRC_SRV_QSGD); break;
-    case SRC_SRV_CLIP: DSQ_ID(SRC_SRV_CLIP); break;
-    case SRC_SRV_RSPARSE: DSQ_ID(SRC_SRV_RSPARSE); break;
-    default: return cudaErrorInvalidValue;
-  }
+  DSQ_SWITCH_SRC(srck, DSQ_ID)
 #undef DSQ_ID
   count_launches(1);
   return cudaGetLastError();
@@ -62,7 +60,7 @@ cudaError_t launch_identity(int srck, const SrcParams& src, float* out_c, uint64
 // Q = clipping (Section 3.2): the low BITS bits of every number are set to zero; the payload is what
 // is left, bits(v) >> BITS, as 16- or 8-bit entries.  The residual v - Q[v] is exact.
 template <int SRC, int BITS>
-__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : kServerCtasPerSm)
+__global__ void __launch_bounds__(kThreads, is_worker_src(SRC) ? 0 : kServerCtasPerSm)
 k_clip(const SrcParams src, uint8_t* out_hi, uint64_t hi_row_stride, float* delta_out, uint64_t delta_row_stride, float* x,
        float gamma) {
   pdl_prologue();
@@ -99,7 +97,7 @@ k_clip(const SrcParams src, uint8_t* out_hi, uint64_t hi_row_stride, float* delt
         }
       }
     }
-    store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
+    if (keeps_error<SRC>(delta_out)) store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
     if (x) {
       float4 xv = load_row4(x, e, cnt, 1);
       xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
@@ -114,16 +112,7 @@ static cudaError_t launch_clip_bits(int srck, const SrcParams& src, uint8_t* out
                                     uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st) {
   dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
 #define DSQ_CL(S) launch_pdl(k_clip<S, BITS>, grid, kThreads, st, src, out_hi, hi_row_stride, delta_out, delta_row_stride, x, gamma)
-  switch (srck) {
-    case SRC_WORKER: DSQ_CL(SRC_WORKER); break;
-    case SRC_SRV_IDENTITY: DSQ_CL(SRC_SRV_IDENTITY); break;
-    case SRC_SRV_SIGN1: DSQ_CL(SRC_SRV_SIGN1); break;
-    case SRC_SRV_TOPK: DSQ_CL(SRC_SRV_TOPK); break;
-    case SRC_SRV_QSGD: DSQ_CL(SRC_SRV_QSGD); break;
-    case SRC_SRV_CLIP: DSQ_CL(SRC_SRV_CLIP); break;
-    case SRC_SRV_RSPARSE: DSQ_CL(SRC_SRV_RSPARSE); break;
-    default: return cudaErrorInvalidValue;
-  }
+  DSQ_SWITCH_SRC(srck, DSQ_CL)
 #undef DSQ_CL
   count_launches(1);
   return cudaGetLastError();
@@ -159,7 +148,7 @@ __global__ void __launch_bounds__(kThreads) k_rsparse_draw(const RsparseParams r
 // Q = randomised sparsification (Section 3.2): the entries of a chunk share one draw o in 0..S-1 and
 // the entry at offset t survives iff t mod S == o; survivors go to slot j / S of the payload.
 template <int SRC>
-__global__ void __launch_bounds__(kThreads, SRC == SRC_WORKER ? 0 : kServerCtasPerSm)
+__global__ void __launch_bounds__(kThreads, is_worker_src(SRC) ? 0 : kServerCtasPerSm)
 k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_t delta_row_stride, float* x, float gamma) {
   pdl_prologue();
   const uint32_t row = blockIdx.y;
@@ -195,7 +184,7 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
       const uint64_t group = (src.d - 1) >> rp.log2_keep;
       if ((group << rp.log2_keep) + o >= src.d) val[group] = 0.f;
     }
-    store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
+    if (keeps_error<SRC>(delta_out)) store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
     if (x) {
       float4 xv = load_row4(x, e, cnt, 1);
       xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
@@ -212,16 +201,7 @@ cudaError_t launch_rsparse(int srck, const SrcParams& src, const RsparseParams& 
   count_launches(1);
   dim3 grid(grid_for((src.d + 3) / 4), rows, 1);
 #define DSQ_RS(S) launch_pdl(k_rsparse<S>, grid, kThreads, st, src, rp, delta_out, delta_row_stride, x, gamma)
-  switch (srck) {
-    case SRC_WORKER: DSQ_RS(SRC_WORKER); break;
-    case SRC_SRV_IDENTITY: DSQ_RS(SRC_SRV_IDENTITY); break;
-    case SRC_SRV_SIGN1: DSQ_RS(SRC_SRV_SIGN1); break;
-    case SRC_SRV_TOPK: DSQ_RS(SRC_SRV_TOPK); break;
-    case SRC_SRV_QSGD: DSQ_RS(SRC_SRV_QSGD); break;
-    case SRC_SRV_CLIP: DSQ_RS(SRC_SRV_CLIP); break;
-    case SRC_SRV_RSPARSE: DSQ_RS(SRC_SRV_RSPARSE); break;
-    default: return cudaErrorInvalidValue;
-  }
+  DSQ_SWITCH_SRC(srck, DSQ_RS)
 #undef DSQ_RS
   count_launches(1);
   return cudaGetLastError();
@@ -241,6 +221,12 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(const PayloadView pv, 
       const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]) + (e >> 5)) >> (uint32_t)(e & 31);
       const float s = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
       C = make_float4(signed_by_bit(s, w, 0), signed_by_bit(s, w, 1), signed_by_bit(s, w, 2), signed_by_bit(s, w, 3));
+    } else if (pv.op == DS_Q_TERNARY) {
+      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[0]) + (e >> 5)) >> (uint32_t)(e & 31);
+      const uint32_t z = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[1]) + (e >> 5)) >> (uint32_t)(e & 31);
+      const float s = __ldg(reinterpret_cast<const float*>(pv.base + pv.off[2]));
+      C = make_float4((z & 1u) ? signed_by_bit(s, w, 0) : 0.f, (z & 2u) ? signed_by_bit(s, w, 1) : 0.f,
+                      (z & 4u) ? signed_by_bit(s, w, 2) : 0.f, (z & 8u) ? signed_by_bit(s, w, 3) : 0.f);
     } else if (pv.op == DS_Q_RSPARSE) {
       const uint32_t o = __ldg(reinterpret_cast<const uint32_t*>(pv.base + pv.off[1]) + (e >> pv.log2_chunk));
       const float* val = reinterpret_cast<const float*>(pv.base + pv.off[0]);

@@ -17,6 +17,22 @@ inline void count_launches(uint64_t n) { g_kernel_launches.fetch_add(n, std::mem
 // Records the text of a CUDA error for ds_last_error() (kept per host thread) and returns DS_ERR_CUDA.
 int cuda_fail(cudaError_t e, const char* where);
 
+// Runs X(S) for the source kind `srck` with S a compile-time constant; returns
+// cudaErrorInvalidValue from the enclosing function for an unknown kind.
+#define DSQ_SWITCH_SRC(srck, X)                          \
+  switch (srck) {                                        \
+    case SRC_WORKER: X(SRC_WORKER); break;               \
+    case SRC_SRV_IDENTITY: X(SRC_SRV_IDENTITY); break;   \
+    case SRC_SRV_SIGN1: X(SRC_SRV_SIGN1); break;         \
+    case SRC_SRV_TOPK: X(SRC_SRV_TOPK); break;           \
+    case SRC_SRV_QSGD: X(SRC_SRV_QSGD); break;           \
+    case SRC_SRV_CLIP: X(SRC_SRV_CLIP); break;           \
+    case SRC_SRV_RSPARSE: X(SRC_SRV_RSPARSE); break;     \
+    case SRC_WORKER_PLAIN: X(SRC_WORKER_PLAIN); break;   \
+    case SRC_SRV_TERNARY: X(SRC_SRV_TERNARY); break;     \
+    default: return cudaErrorInvalidValue;               \
+  }
+
 // kernel<<<grid, block, 0, st>>>(args...) with programmatic stream serialization allowed (the
 // kernel begins with pdl_prologue()).  A failed launch shows in cudaGetLastError().
 template <typename... P, typename... A>
@@ -25,6 +41,24 @@ inline void launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, cudaStream_t
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
+// The same with `smem` bytes of dynamic shared memory (beyond the 48 KB a kernel gets by default the
+// limit is raised first; that call only sets a number on the host).
+template <typename... P, typename... A>
+inline void launch_pdl_smem(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args) {
+  if (smem > 48 * 1024) (void)cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr{};
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -102,7 +136,9 @@ struct TopkIO {
   uint32_t* idx;            // payload sub-arrays of row 0; rows are payload_stride bytes apart
   float* val;
   uint64_t payload_stride;
-  float* v_inout;           // [rows, d]: receives v, then has the kept entries zeroed (the residual)
+  float* v_inout;           // [rows, d]: receives v, then has the kept entries zeroed (the residual).  With
+                            // keep_error = 0 (source SRC_WORKER_PLAIN): where v already lies (the gradient); only read
+  int keep_error;
   float* x;                 // non-NULL: fused model update at the kept entries (server pass)
   float gamma;
   uint32_t* dev_status;
@@ -134,6 +170,28 @@ struct RsparseParams {
 };
 cudaError_t launch_rsparse(int src_kind, const SrcParams& src, const RsparseParams& rp, float* delta_out,
                            uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);
+
+// Operators with ONE factor for the whole vector: the 1-bit operator as Section 3.2 / Section 5.1 state
+// it (chunk = 0) and the ternary quantiser of Section 5.1, item 2.  The factor depends on a sum (and,
+// ternary, on the largest magnitude and the number of survivors) over all d entries, so a pass is
+// several kernels: tile sums, their pairwise combination, then the encoding.  v is recomputed from its
+// source in every kernel instead of being stored.
+struct WholeParams {
+  uint32_t* out_sgn;         // sign words (bit = v >= 0), row stride word_stride (in words)
+  uint32_t* out_nz;          // ternary: words of the non-zero plane
+  float* out_scale;          // one factor per row, row stride word_stride (floats)
+  uint64_t word_stride;
+  float* delta_out;          // residual destination, or NULL: no error is kept
+  uint64_t delta_row_stride;
+  float* x;                  // non-NULL: fused model update (server pass)
+  float gamma;
+  PhiloxKeys keys;
+  uint32_t step, server_pass;
+  uint32_t l2;               // SIGN1: 1 = l2 magnitudes
+};
+uint64_t whole_workspace_bytes(uint64_t d, uint32_t rows);
+cudaError_t launch_whole(int op, int src_kind, const SrcParams& src, const WholeParams& p, void* workspace, uint32_t rows,
+                         cudaStream_t st);
 
 // x = x - gamma * decode(payload)
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);

@@ -38,8 +38,8 @@ assert len(RESNET18_SLICES) == 62 and sum(RESNET18_SLICES) == 11_689_512
 
 @dataclass(frozen=True)
 class Q:
-    op: str = "identity"     # identity | sign1 | topk | qsgd | clip | rsparse
-    chunk: int = 0
+    op: str = "identity"     # identity | sign1 | topk | qsgd | clip | rsparse | ternary
+    chunk: int = 0           # sign1 / qsgd / rsparse: entries per chunk; sign1 with 0: one factor for the whole vector
     k: int = 0
     levels: int = 0
     norm: int = 1            # sign1: scale from l1 (1) or l2 (2) magnitudes
@@ -50,7 +50,7 @@ class Q:
 
 @dataclass(frozen=True)
 class Workload:
-    wid: int                 # 1..5, index into the benchmark list
+    wid: int                 # 1..5 = the listed configurations; 6.. = added ones
     name: str
     n: int
     d: int
@@ -60,6 +60,7 @@ class Workload:
     server_q: Q
     gamma: float = 0.1
     seed: int = BASE_SEED    # Philox seed handed to the randomised Q
+    compensate: bool = True  # False: the compressed methods of Section 5.1 that keep no error
 
     def scaled(self, d: int, n: int | None = None, steps: int | None = None) -> "Workload":
         """Same recipe at another size; top-k keeps its fraction of d."""
@@ -90,6 +91,16 @@ def _wl() -> dict[int, Workload]:
         # ... and with randomised sparsification (one entry in 32 survives, unscaled) on both passes
         8: Workload(8, "rsparse32_n8_resnet18", 8, 11_689_512, 20, "layered",
                     Q("rsparse", chunk=4096, keep_one_in=32), Q("rsparse", chunk=4096, keep_one_in=32)),
+        # ... with the ternary quantiser of Section 5.1 (item 2) on both passes, error-compensated
+        9: Workload(9, "ternary_n8_resnet18", 8, 11_689_512, 20, "layered", Q("ternary"), Q("ternary")),
+        # ... with the 1-bit operator carrying ONE factor per vector, as Section 3.2 / 5.1 state it
+        10: Workload(10, "sign1whole_n8_resnet18", 8, 11_689_512, 20, "layered", Q("sign1", chunk=0), Q("sign1", chunk=0)),
+        # the two compressed methods of Section 5.1 that keep no error: "QSGD" (item 2: ternary workers, the
+        # server sends the plain mean) and "Top-k SGD" (item 5), here with the paper's k = 300000
+        11: Workload(11, "qsgd_baseline_n8_resnet18", 8, 11_689_512, 20, "layered", Q("ternary"), Q("identity"),
+                     compensate=False),
+        12: Workload(12, "topk_sgd_n8_resnet18", 8, 11_689_512, 20, "layered", Q("topk", k=300_000), Q("identity"),
+                     compensate=False),
     }
 
 

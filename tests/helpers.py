@@ -59,6 +59,10 @@ def compare_payload(name: str, op: str, gpu_views: dict, ora: dict):
     elif op == "rsparse":
         assert_bits_match(f"{name}.off", u32(gpu_views["off"]), ora["off"])
         assert_bits_match(f"{name}.val", u32(gpu_views["val"].view(dtype=__import__("torch").int32)), ora["val"].view(np.uint32))
+    elif op == "ternary":
+        assert_bits_match(f"{name}.sgn", u32(gpu_views["sgn"]), ora["sgn"])
+        assert_bits_match(f"{name}.nz", u32(gpu_views["nz"]), ora["nz"])
+        assert_float_match(f"{name}.scale", gpu_views["scale"].cpu().numpy(), ora["scale"])
     elif op == "clip":
         assert_bits_match(f"{name}.hi", u32(gpu_views["hi"]), ora["hi"])
     else:
@@ -73,7 +77,8 @@ def compare_state(ds, st: oracle.State, g_host: np.ndarray, tag: str = ""):
     compare_payload(f"{tag}server", sq, ds.server_views(), st.server_payload)
     # delta = v - Q[v] is a difference: relative to |v| + |Q[v]|, bounded here by |g| + |delta| scale
     mag = float(np.abs(g_host).max()) + float(np.abs(st.delta_w).max()) + 1e-30
-    assert_float_match(f"{tag}delta_w", ds.delta_w.cpu().numpy(), st.delta_w, scale=mag)
-    assert_float_match(f"{tag}delta_s", ds.delta_s.cpu().numpy(), st.delta_s, scale=mag)
+    if ds.compensate:   # without compensation there are no errors (delta_s may exist as scratch: not compared)
+        assert_float_match(f"{tag}delta_w", ds.delta_w.cpu().numpy(), st.delta_w, scale=mag)
+        assert_float_match(f"{tag}delta_s", ds.delta_s.cpu().numpy(), st.delta_s, scale=mag)
     assert_float_match(f"{tag}x", ds.x.cpu().numpy(), st.x, scale=np.abs(st.x).astype(np.float64) + ds.gamma * mag)
     assert ds.device_status() == 0, f"{tag}device status {ds.device_status():#x}"

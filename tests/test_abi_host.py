@@ -64,6 +64,38 @@ def test_layouts(lib):
     assert (a.stride, list(a.off), list(a.count)) == (l2.stride, list(l2.off), list(l2.count))
 
 
+def test_layouts_of_the_whole_vector_operators_and_sizes_without_compensation(lib):
+    d, n = 100_003, 4
+    nw = (d + 31) // 32
+    cfg = b.make_config(n, d, 0.1, Q("sign1", chunk=0), Q("ternary"), 1)
+    w, s = b.get_layout(cfg, 0), b.get_layout(cfg, 1)
+    assert list(w.count)[:2] == [nw, 1] and w.off[1] == (4 * nw + 15) // 16 * 16 and w.stride == w.off[1] + 16
+    assert list(s.count) == [nw, nw, 1] and s.off[1] == w.off[1] and s.off[2] == 2 * w.off[1] and s.stride == s.off[2] + 16
+    bufs = b.ds_buffers()
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_NEED_BUFFERS
+    ntile = (d + 4095) // 4096
+    assert bufs.workspace_bytes >= 2 * n * ntile * 4 + 16 * n        # tile sums, tile maxima / counts, per-vector results
+    assert bufs.delta_w_bytes == 4 * n * d and bufs.delta_s_bytes == 4 * d
+    # without compensation no error buffer is asked for, except delta_s as the top-k server's scratch
+    cfg = b.make_config(n, d, 0.1, Q("topk", k=10), Q("identity"), 1, compensate=False)
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_NEED_BUFFERS
+    assert bufs.delta_w_bytes == 0 and bufs.delta_s_bytes == 0
+    cfg = b.make_config(n, d, 0.1, Q("ternary"), Q("topk", k=10), 1, compensate=False)
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_NEED_BUFFERS
+    assert bufs.delta_w_bytes == 0 and bufs.delta_s_bytes == 4 * d
+    # a handle without error buffers
+    cfg = b.make_config(2, 1000, 0.1, Q("sign1", chunk=128), Q("identity"), 0, compensate=False)
+    bufs = b.ds_buffers()
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_NEED_BUFFERS
+    bufs.x, bufs.worker_payload, bufs.server_payload, bufs.dev_status = 0x10000, 0x20000, 0x30000, 0x40000
+    h = C.c_void_p()
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), C.byref(h)) == b.DS_OK
+    assert lib.ds_destroy(h) == b.DS_OK
+    # unknown flag bits are refused
+    cfg.flags = 2
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_ERR_INVALID_ARG
+
+
 def test_query_mode_reports_sizes(lib):
     cfg = b.make_config(16, 25_557_032, 0.1, Q("topk", k=255_570), Q("topk", k=255_570), 1)
     bufs = b.ds_buffers()
@@ -85,6 +117,7 @@ def test_query_mode_reports_sizes(lib):
     dict(worker_q=Q("clip", bits=32)),
     dict(worker_q=Q("rsparse", chunk=4096, keep_one_in=3)), dict(server_q=Q("rsparse", chunk=4096, keep_one_in=256)),
     dict(server_q=Q("rsparse", chunk=100, keep_one_in=4)), dict(worker_q=Q("rsparse", chunk=4096, keep_one_in=4, scaled=2)),
+    dict(worker_q=Q("ternary", chunk=4096)), dict(worker_q=Q("qsgd", chunk=0, levels=255)),
 ])
 def test_bad_configs_are_rejected(lib, kw):
     args = dict(n=4, d=1000, gamma=0.1, worker_q=Q("identity"), server_q=Q("identity"), seed=0)

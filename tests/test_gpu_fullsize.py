@@ -12,7 +12,7 @@ from tests.helpers import compare_state, to_oracle_q
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12])
 def test_full_size_step_matches_oracle(wid):
     wl = WORKLOADS[wid]
     need = 4 * wl.n * wl.d * 4 + (2 << 30)
@@ -23,15 +23,18 @@ def test_full_size_step_matches_oracle(wid):
     gen = torch.Generator(device=dev).manual_seed(1000 + wid)
     g = make_gradients(wl, 3, device=dev)
     scale = float(g[0, :100_000].abs().mean())
-    ds.delta_w.normal_(0.0, 0.5 * scale, generator=gen)
-    ds.delta_s.normal_(0.0, 0.25 * scale, generator=gen)
     ds.x.normal_(0.0, 1.0, generator=gen)
-    st = oracle.State(ds.x.cpu().numpy().copy(), ds.delta_w.cpu().numpy().copy(), ds.delta_s.cpu().numpy().copy())
+    if wl.compensate:
+        ds.delta_w.normal_(0.0, 0.5 * scale, generator=gen)
+        ds.delta_s.normal_(0.0, 0.25 * scale, generator=gen)
+        st = oracle.State(ds.x.cpu().numpy().copy(), ds.delta_w.cpu().numpy().copy(), ds.delta_s.cpu().numpy().copy())
+    else:
+        st = oracle.State.zeros(wl.n, wl.d, ds.x.cpu().numpy())
     ds.step(g, 3, fuse_apply=True)
     torch.cuda.synchronize()
     g_host = g.cpu().numpy()
     del g
-    oracle.step(st, g_host, to_oracle_q(wl.worker_q), to_oracle_q(wl.server_q), wl.gamma, wl.seed, 3)
+    oracle.step(st, g_host, to_oracle_q(wl.worker_q), to_oracle_q(wl.server_q), wl.gamma, wl.seed, 3, compensate=wl.compensate)
     compare_state(ds, st, g_host, tag=f"workload {wid}: ")
     ds.close()
 

@@ -16,14 +16,17 @@ TOPK = lambda k: Q("topk", k=k)
 IDENT = Q("identity")
 CLIP = lambda b=16: Q("clip", bits=b)
 RSP = lambda S=4, L=4096, scaled=0: Q("rsparse", chunk=L, keep_one_in=S, scaled=scaled)
+SIGN_WHOLE = lambda norm=1: Q("sign1", chunk=0, norm=norm)      # one factor for the whole vector
+TERN = Q("ternary")
 
 
-def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None, scribble=False):
+def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None, state0=None, scribble=False,
+                 compensate=True):
     """Free-running: both sides start from the same state and see the same gradients; after every
     step every output must agree."""
     # every buffer sits between sentinel bytes and the payloads start out as 0xFF: a write outside a
     # buffer, or a payload byte the library leaves to chance, fails the comparison
-    ds = DoubleSqueeze(n, d, gamma, wq, sq, seed, x0=x0, guard=True, payload_fill=0xFF)
+    ds = DoubleSqueeze(n, d, gamma, wq, sq, seed, x0=x0, guard=True, payload_fill=0xFF, compensate=compensate)
     st = oracle.State.zeros(n, d, None if x0 is None else x0.cpu().numpy())
     if state0 is not None:
         dw, dsv = state0
@@ -38,7 +41,7 @@ def run_lockstep(n, d, wq, sq, gs, gamma=0.1, seed=190505957, fuse=True, x0=None
         ds.step(g_dev, t, fuse_apply=fuse)
         torch.cuda.synchronize()
         g_host = g.cpu().numpy()
-        oracle.step(st, g_host, to_oracle_q(wq), to_oracle_q(sq), gamma, seed, t)
+        oracle.step(st, g_host, to_oracle_q(wq), to_oracle_q(sq), gamma, seed, t, compensate=compensate)
         compare_state(ds, st, g_host, tag=f"step {t}: ")
         assert ds.check_guards(), f"step {t}: bytes outside a buffer were overwritten"
     ds.close()
@@ -117,6 +120,67 @@ def test_rsparse_mixed_with_other_operators_unaligned_rows_and_unfused_update():
     run_lockstep(37, 9000, RSP(4, 128), RSP(4, 128), randn_steps(37, 9000, 2, seed=50))
 
 
+# ------------------------------------------------------------------ one factor for the whole vector
+
+@pytest.mark.parametrize("d", [1, 33, 4096, 10_000, 65_536 + 4 * 37, 5 * 4096 * 1024 // 16 + 12])
+@pytest.mark.parametrize("norm", [1, 2])
+def test_sign1_whole_vector_both_passes(d, norm):
+    run_lockstep(3, d, SIGN_WHOLE(norm), SIGN_WHOLE(norm), randn_steps(3, d, 3, seed=d + norm))
+
+
+def test_sign1_whole_vector_many_tiles_exercises_the_block_sums():
+    # more than 1024 tiles per vector: every thread of the combining kernel sums a block of tile sums
+    d = 4096 * 2500 + 777
+    run_lockstep(2, d, SIGN_WHOLE(1), SIGN_WHOLE(2), randn_steps(2, d, 2, seed=3))
+
+
+@pytest.mark.parametrize("d", [1, 5, 33, 4096, 10_000, 65_536 + 4 * 37, 300_001])
+def test_ternary_both_passes(d):
+    run_lockstep(3, d, TERN, TERN, randn_steps(3, d, 3, seed=d, scale=1e-2))
+
+
+def test_whole_vector_operators_mixed_unaligned_unfused_and_degenerate():
+    d = 50_000 + 13
+    for wq, sq in [(TERN, IDENT), (TERN, TOPK(500)), (TERN, SIGN(2048)), (SIGN_WHOLE(), TERN), (QSGD(1024, 31), TERN),
+                   (TOPK(700), SIGN_WHOLE(2)), (SIGN_WHOLE(2), QSGD(2048)), (CLIP(16), TERN), (TERN, RSP(8)),
+                   (RSP(4), SIGN_WHOLE()), (IDENT, TERN), (SIGN_WHOLE(), CLIP(24))]:
+        run_lockstep(5, d, wq, sq, randn_steps(5, d, 2, seed=51))
+    run_lockstep(3, 30_000, TERN, TERN, randn_steps(3, 30_000, 3, seed=52), fuse=False)
+    run_lockstep(3, 30_001, SIGN_WHOLE(), SIGN_WHOLE(2), randn_steps(3, 30_001, 3, seed=53), fuse=False)
+    run_lockstep(37, 9000, TERN, SIGN_WHOLE(), randn_steps(37, 9000, 2, seed=54))
+    n, dd = 2, 3 * 4096
+    g = torch.randn(n, dd) * 1e-3
+    g[:, :4096] = 0.0
+    g[:, 4096:4096 + 64] = -0.0
+    g[:, 5000:5100] = 1e-41
+    for wq in (TERN, SIGN_WHOLE(1), SIGN_WHOLE(2)):
+        run_lockstep(n, dd, wq, wq, [g, g.clone(), -g, torch.zeros(n, dd)])
+
+
+# ------------------------------------------------------------------ without error compensation
+
+@pytest.mark.parametrize("wq,sq", [
+    (TOPK(500), IDENT), (TERN, IDENT), (SIGN(4096), SIGN(4096)), (QSGD(2048), QSGD(2048)), (TOPK(700), TOPK(300)),
+    (SIGN(1024), TOPK(200)), (CLIP(16), RSP(8)), (RSP(4), CLIP(24)), (IDENT, IDENT), (SIGN_WHOLE(), TERN),
+    (TOPK(0), SIGN(128)), (SIGN_L2(512), SIGN_WHOLE(2)),
+])
+def test_without_compensation_matches_the_oracle(wq, sq):
+    d = 50_000 + 12
+    run_lockstep(5, d, wq, sq, randn_steps(5, d, 3, seed=61), compensate=False)
+    run_lockstep(3, 30_001, wq, sq, randn_steps(3, 30_001, 2, seed=62), compensate=False, fuse=False)
+
+
+def test_without_compensation_top_k_on_predicted_bands_and_after_jumps():
+    n, d, k = 3, 120_000, 1200
+    gen = torch.Generator().manual_seed(9)
+    scales = [1, 1, 1, 1, 1.02, 8.0, 8.0, 0.01, 0.01, 1]
+    gs = [torch.randn(n, d, generator=gen) * s for s in scales]
+    ds, _ = run_lockstep(n, d, TOPK(k), TOPK(k), gs, compensate=False)
+    predicted, full = ds.topk_routes()
+    assert predicted >= 3 * (n + 1) and full >= 3 * (n + 1)
+    assert ds.delta_w.numel() == 0          # no worker error exists at all
+
+
 def test_identity_is_parallel_sgd():
     run_lockstep(4, 10_001, IDENT, IDENT, randn_steps(4, 10_001, 3))
 
@@ -186,8 +250,10 @@ def test_topk_threshold_prediction_hits_misses_and_garbage():
     ds, _ = run_lockstep(n, d, TOPK(k), TOPK(k), gs)
     predicted, full = ds.topk_routes()
     assert predicted + full == (n + 1) * len(gs)
-    assert full >= 3 * (n + 1)          # the first step and the two jumps by 8x and 800x cannot be predicted
-    assert predicted >= 4 * (n + 1)     # the steady stretches are
+    # the first step and the jump by 8x cannot be predicted (after the jump down the errors still carry
+    # the large magnitudes, so the threshold comes down slowly); the steady stretches are
+    assert full >= 2 * (n + 1)
+    assert predicted >= 4 * (n + 1)
     run_lockstep(n, d, SIGN(4096), TOPK(k // 2), gs[:6])
     run_lockstep(n, d, TOPK(k), TOPK(k), gs[:5], scribble=True)
 
@@ -212,15 +278,15 @@ def test_many_workers_and_one_worker():
 
 # ------------------------------------------------------------------ the five workloads, scaled down
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12])
 def test_workload_recipes_scaled(wid):
     wl = WORKLOADS[wid]
     wl = wl if wid == 1 else wl.scaled(d=200_000 + 40, n=min(wl.n, 8), steps=4)
     gs = [make_gradients(wl, t, device="cpu") for t in range(min(wl.steps, 4))]
-    run_lockstep(wl.n, wl.d, wl.worker_q, wl.server_q, gs, gamma=wl.gamma, seed=wl.seed)
+    run_lockstep(wl.n, wl.d, wl.worker_q, wl.server_q, gs, gamma=wl.gamma, seed=wl.seed, compensate=wl.compensate)
 
 
-@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10])
 def test_telescoping_identity_free_running_on_the_gpu(wid):
     """Eq. 5-6 on the GPU alone, with no oracle in the loop: after T steps of any Q,
     x_T - gamma (delta_T + mean_i delta_T^(i)) = x_0 - gamma sum_t mean_i g_t^(i), up to fp32 rounding."""
