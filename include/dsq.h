@@ -53,6 +53,8 @@ typedef enum {
 
 /* dev_status is four words.  Word 0 holds flags: */
 #define DS_DEV_TOPK_INCONSISTENT 0x1u /* top-k selection counted a number of entries other than k */
+#define DS_DEV_TAIL_TIMEOUT 0x2u      /* a bounded wait between the thread blocks of the top-k selection kernel
+                                         ran out; the kernel left early and this step's results are not valid */
 /* Words 1 and 2 count top-k selections (one per vector and pass) by the route they took: with the
  * threshold band predicted from the previous steps ("predicted": v is read once), or through the
  * full histogram after a missing or wrong prediction ("full": v is read three times).  Both routes

@@ -20,6 +20,7 @@ DS_ERR_INVALID_ARG, DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL = -1, -2, -3
 DS_ERR_STATE, DS_ERR_CUDA, DS_ERR_UNSUPPORTED = -4, -5, -6
 DS_FUSE_APPLY = 1
 DS_DEV_TOPK_INCONSISTENT = 1
+DS_DEV_TAIL_TIMEOUT = 2
 OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4, "rsparse": 5, "ternary": 6}
 DS_NO_COMPENSATION = 1
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",

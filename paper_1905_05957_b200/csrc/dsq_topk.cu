@@ -110,17 +110,14 @@ __device__ __forceinline__ uint32_t octet_words4(const uint32_t (&nib)[4], uint3
 // is "listed": its (value bits, index) goes to the tile's own region of the list (kTile slots,
 // enough for the whole tile, so CTAs never share a region), in index order.  Listed entries with
 // key > hi are certain to be kept; they are counted and already zeroed in the residual (their
-// value survives in the list).  The keys of the other listed entries -- the candidates, inside the
-// band -- also go to the tile's candidate region `cand` (kTile slots).  info receives
-// (listed, above hi, 0, 0); the two zeros are the counters the selection fills.  out_row = NULL: nothing is zeroed.  s_tot: one uint4 per warp, free for reuse after the call's barrier
-// has been passed by all threads a second time; s_cand: one word.  Called by all threads of the CTA.
+// value survives in the list).  info receives (listed, above hi, 0, 0); the two zeros are the
+// counters classify fills.  out_row = NULL: nothing is zeroed.  s_tot: one uint4 per warp, free for reuse after the call's barrier
+// has been passed by all threads a second time.  Called by all threads of the CTA.
 template <bool FULL>
 __device__ __forceinline__ void mark_tile(const float4 (&v)[4], const uint32_t (&cnt)[4], uint64_t base, uint32_t key_lo,
-                                          uint32_t key_hi, float* out_row, uint2* region, uint32_t* cand, uint4* info,
-                                          uint4* s_tot, uint32_t* s_cand) {
+                                          uint32_t key_hi, float* out_row, uint2* region, uint4* info, uint4* s_tot) {
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5;
   uint32_t sel[4], kept = 0;
-  if (tid == 0) *s_cand = 0;  // ordered before its first use by the barrier below
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     sel[j] = 0;
@@ -147,8 +144,6 @@ __device__ __forceinline__ void mark_tile(const float4 (&v)[4], const uint32_t (
       }
     }
   }
-  // candidates of this thread: listed, not above the band
-  const uint32_t nc = __popc(sel[0]) + __popc(sel[1]) + __popc(sel[2]) + __popc(sel[3]) - kept;
   // index order is (j, thread, k): per-j counts, packed two to a word, scanned over the warp
   const uint32_t ca = __popc(sel[0]) | (__popc(sel[1]) << 16), cb = __popc(sel[2]) | (__popc(sel[3]) << 16);
   uint32_t ia = ca, ib = cb;
@@ -171,9 +166,6 @@ __device__ __forceinline__ void mark_tile(const float4 (&v)[4], const uint32_t (
   const uint32_t t0 = sa & 0xFFFFu, t1 = sa >> 16, t2 = sb & 0xFFFFu, t3 = sb >> 16;
   const uint32_t ea = pa + ia - ca, eb = pb + ib - cb;
   uint32_t pos[4] = {ea & 0xFFFFu, t0 + (ea >> 16), t0 + t1 + (eb & 0xFFFFu), t0 + t1 + t2 + (eb >> 16)};
-  // the candidates' keys alone, in any order, also go to the tile's candidate region (the selection
-  // only counts them); their slots come from a counter in shared memory
-  uint32_t at = nc ? atomicAdd(s_cand, nc) : 0u;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     if (sel[j]) {
@@ -181,13 +173,8 @@ __device__ __forceinline__ void mark_tile(const float4 (&v)[4], const uint32_t (
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if ((sel[j] >> k) & 1u) {
-          const uint32_t bits = __float_as_uint(compc(v[j], k));
-          if (pos[j] < kTile) region[pos[j]] = make_uint2(bits, i0 + k);
+          if (pos[j] < kTile) region[pos[j]] = make_uint2(__float_as_uint(compc(v[j], k)), i0 + k);
           ++pos[j];
-          if ((bits & 0x7fffffffu) <= key_hi) {
-            if (at < kTile) cand[at] = bits & 0x7fffffffu;
-            ++at;
-          }
         }
     }
   }
@@ -199,8 +186,7 @@ __device__ __forceinline__ void mark_tile(const float4 (&v)[4], const uint32_t (
 // marked while v is still in registers.
 template <int SRC, bool FULL>
 __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, uint64_t base, float* out_row, bool marking,
-                                           uint32_t key_lo, uint32_t key_hi, uint2* region, uint32_t* cand, uint4* info,
-                                           uint4* s_tot, uint32_t* s_cand) {
+                                           uint32_t key_lo, uint32_t key_hi, uint2* region, uint4* info, uint4* s_tot) {
   const uint32_t tid = threadIdx.x;
   const uint64_t d = src.d;
   float4 v[4];
@@ -248,15 +234,14 @@ __device__ __forceinline__ void pass1_tile(const SrcParams& src, uint32_t row, u
       }
     }
   }
-  if (marking) mark_tile<FULL>(v, cnt, base, key_lo, key_hi, SRC == SRC_WORKER_PLAIN ? nullptr : out_row, region, cand, info, s_tot, s_cand);
+  if (marking) mark_tile<FULL>(v, cnt, base, key_lo, key_hi, SRC == SRC_WORKER_PLAIN ? nullptr : out_row, region, info, s_tot);
 }
 
 template <int SRC>
 __global__ void __launch_bounds__(kThreads, is_worker_src(SRC) || SRC == SRC_SRV_TOPK ? 5 : kServerCtasPerSm) k_topk_pass1(const SrcParams src, float* v_out, const TopkPred* pred, uint2* list,
-                                                         uint32_t* cand_keys, uint64_t cap, uint4* tile_info, uint64_t ntile) {
+                                                         uint64_t cap, uint4* tile_info, uint64_t ntile) {
   pdl_prologue();
   __shared__ uint4 s_tot[kThreads / 32];
-  __shared__ uint32_t s_cand;
   const uint32_t row = blockIdx.y;
   const uint64_t tile = blockIdx.x, base = tile * kTile;
   const uint64_t d = src.d;
@@ -264,12 +249,11 @@ __global__ void __launch_bounds__(kThreads, is_worker_src(SRC) || SRC == SRC_SRV
   const bool marking = predicted_band(pred, row, &key_lo, &key_hi);
   float* out_row = v_out + (uint64_t)row * d;
   uint2* region = list + (uint64_t)row * cap + base;
-  uint32_t* cand = cand_keys + (uint64_t)row * cap + base;
   uint4* info = tile_info + (uint64_t)row * ntile + tile;
   if (src.vec && base + kTile <= d) {
-    pass1_tile<SRC, true>(src, row, base, out_row, marking, key_lo, key_hi, region, cand, info, s_tot, &s_cand);
+    pass1_tile<SRC, true>(src, row, base, out_row, marking, key_lo, key_hi, region, info, s_tot);
   } else {
-    pass1_tile<SRC, false>(src, row, base, out_row, marking, key_lo, key_hi, region, cand, info, s_tot, &s_cand);
+    pass1_tile<SRC, false>(src, row, base, out_row, marking, key_lo, key_hi, region, info, s_tot);
   }
 }
 
@@ -395,11 +379,9 @@ __global__ void __launch_bounds__(kThreads) k_topk_hist(float* v_io, uint64_t d,
 // Rebuilds the tile regions for the exact threshold bin: entries in bins above it are kept (and
 // zeroed), entries inside it are the candidates.  A small grid strides over the tiles.
 __global__ void __launch_bounds__(kThreads) k_topk_mark(float* v_io, uint64_t d, int vec, int keep_error, const TopkState* state,
-                                                        uint2* list, uint32_t* cand_keys, uint64_t cap, uint4* tile_info,
-                                                        uint64_t ntile) {
+                                                        uint2* list, uint64_t cap, uint4* tile_info, uint64_t ntile) {
   pdl_prologue();
   __shared__ uint4 s_tot[kThreads / 32];
-  __shared__ uint32_t s_cand;
   const uint32_t tid = threadIdx.x, row = blockIdx.y;
   if (!state[row].need_mark) return;
   const uint32_t lo = state[row].tb1 << 19, hi = lo | 0x7FFFFu;
@@ -426,15 +408,14 @@ __global__ void __launch_bounds__(kThreads) k_topk_mark(float* v_io, uint64_t d,
     }
     uint2* region = list + (uint64_t)row * cap + base;
     uint4* info = tile_info + (uint64_t)row * ntile + tile;
-    uint32_t* cand = cand_keys + (uint64_t)row * cap + base;
     float* zero_in = keep_error ? vrow : nullptr;
-    if (full) mark_tile<true>(v, cnt, base, lo, hi, zero_in, region, cand, info, s_tot, &s_cand);
-    else mark_tile<false>(v, cnt, base, lo, hi, zero_in, region, cand, info, s_tot, &s_cand);
+    if (full) mark_tile<true>(v, cnt, base, lo, hi, zero_in, region, info, s_tot);
+    else mark_tile<false>(v, cnt, base, lo, hi, zero_in, region, info, s_tot);
     __syncthreads();  // s_tot is written again for the next tile
   }
 }
 
-// ---------------------------------------------------------------- selection from the candidates
+// ---------------------------------------------------------------- tile regions -> dense list
 // Exclusive prefix of one value per thread over the CTA (blockDim a multiple of 32, at most 1024).
 // s_warp: 33 words.  *total = sum over the CTA.  Ends with a barrier; s_warp may be reused after
 // the next barrier the caller passes.
@@ -464,264 +445,257 @@ __device__ __forceinline__ uint32_t cta_excl_scan(uint32_t val, uint32_t* s_warp
   return s_warp[wrp] + incl - val;
 }
 
+// One batch of up to 64 region entries, two neighbours per lane (q.x, q.y = first entry, q.z, q.w =
+// second): those not above the band (key <= fhi) are the candidates; they go to the dense list as
+// (key, index) from slot `run` on, in entry order.
+template <bool HIST>
+__device__ __forceinline__ void put_candidates(uint4 q, bool valid0, bool valid1, uint32_t fhi, uint32_t& run, uint2* drow,
+                                               uint64_t cap, uint32_t* s_hist, uint32_t lane) {
+  const uint32_t key0 = q.x & 0x7fffffffu, key1 = q.z & 0x7fffffffu;
+  const bool is0 = valid0 && key0 <= fhi, is1 = valid1 && key1 <= fhi;
+  const uint32_t b0 = __ballot_sync(0xffffffffu, is0), b1 = __ballot_sync(0xffffffffu, is1);
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t pos = run + __popc(b0 & lt) + __popc(b1 & lt);
+  if (is0) {
+    if (pos < cap) drow[pos] = make_uint2(key0, q.y);
+    if (HIST) atomicAdd(&s_hist[key0 >> 19], 1u);
+    ++pos;
+  }
+  if (is1) {
+    if (pos < cap) drow[pos] = make_uint2(key1, q.w);
+    if (HIST) atomicAdd(&s_hist[key1 >> 19], 1u);
+  }
+  run += __popc(b0) + __popc(b1);
+}
+
 // The first / a later 64-entry batch of a region of n entries (regions are 16-byte aligned).
 __device__ __forceinline__ uint4 region_batch(const uint2* region, uint32_t i0, uint32_t n, uint32_t lane) {
   return i0 + 2u * lane < n ? reinterpret_cast<const uint4*>(region)[(i0 >> 1) + lane] : make_uint4(0u, 0u, 0u, 0u);
 }
 
-
-// Exclusive prefix over the `count` (kept, ties) pairs of one vector, by one 1024-thread CTA.  get(i)
-// returns pair i; pre receives the prefixes; the grand total is returned to every thread.  A round
-// takes 4096 pairs: loaded and stored with neighbouring threads on neighbouring pairs, scanned
-// with four consecutive pairs per thread; shared memory turns one order into the other.
-// s_item: 4096 pairs, s_warp: 32 pairs, s_carry: one pair.
-template <typename Get>
-__device__ __forceinline__ uint2 cta_scan_pairs(uint64_t count, Get get, uint2* pre, uint2* s_item, uint2* s_warp, uint2* s_carry) {
-  constexpr int ITEMS = 4;
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5;
-  if (tid == 0) *s_carry = make_uint2(0, 0);
-  for (uint64_t base = 0; base < count; base += 1024 * ITEMS) {
-#pragma unroll
-    for (int u = 0; u < ITEMS; ++u) {
-      const uint64_t i = base + (uint64_t)u * 1024 + tid;
-      s_item[u * 1024 + tid] = i < count ? get(i) : make_uint2(0, 0);
-    }
+// Copies the candidates out of the tile regions into one dense list per vector; a tile's
+// candidates stay together and in index order, the tiles of a CTA follow one another.  Each CTA
+// takes a contiguous run of tiles; the tile_info counts say how many candidates each region
+// holds, so one prefix sum per CTA and ONE reservation in the dense list place them all (the
+// counters of all vectors share a cache line, and atomics on one line are served one after the
+// other).  With HIST the top-12-bit histogram of the keys is counted on the way.  Returns this
+// thread's share of the "entries above the band" counts.  s_n, s_off: blockDim words each;
+// s_warp: 34 words.  Called by whole CTAs.
+template <bool HIST>
+__device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint4* info, uint64_t ntile, uint2* drow,
+                                                 uint64_t cap, uint32_t* dense_count, uint32_t fhi, uint32_t* s_hist,
+                                                 uint32_t* s_n, uint32_t* s_off, uint32_t* s_warp) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, nthr = blockDim.x, warps = nthr >> 5;
+  const uint64_t per = (ntile + gridDim.x - 1) / gridDim.x;
+  const uint64_t c0 = (uint64_t)blockIdx.x * per, c1 = min(ntile, c0 + per);
+  uint32_t kept = 0;
+  for (uint64_t r0 = c0; r0 < c1; r0 += nthr) {
+    uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+    if (r0 + tid < c1) mine = info[r0 + tid];
+    const uint32_t n = min(mine.x, (uint32_t)kTile), above = min(mine.y, n);
+    kept += above;
+    uint32_t total;
+    const uint32_t excl = cta_excl_scan(n - above, s_warp, &total);
+    s_n[tid] = n;
+    s_off[tid] = excl;
+    if (tid == 0) s_warp[33] = total ? atomicAdd(dense_count, total) : 0u;
     __syncthreads();
-    uint2 mine[ITEMS];
-    uint2 sum = make_uint2(0, 0);
+    const uint32_t base = s_warp[33];
+    const uint32_t ntl = (uint32_t)min((uint64_t)nthr, c1 - r0);
+    // a warp takes four tiles at a time and has the first 64 entries of each in flight at once
+    for (uint32_t i = wrp; i < ntl; i += 4 * warps) {
+      uint32_t nn[4];
+      uint4 q[4];
 #pragma unroll
-    for (int u = 0; u < ITEMS; ++u) {
-      mine[u] = s_item[tid * ITEMS + u];
-      sum.x += mine[u].x;
-      sum.y += mine[u].y;
-    }
-    uint2 incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t yx = __shfl_up_sync(0xffffffffu, incl.x, o), yy = __shfl_up_sync(0xffffffffu, incl.y, o);
-      if (lane >= (uint32_t)o) { incl.x += yx; incl.y += yy; }
-    }
-    if (lane == 31) s_warp[wrp] = incl;
-    __syncthreads();
-    if (wrp == 0) {
-      const uint2 w = s_warp[lane];
-      uint2 wi = w;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t yx = __shfl_up_sync(0xffffffffu, wi.x, o), yy = __shfl_up_sync(0xffffffffu, wi.y, o);
-        if (lane >= (uint32_t)o) { wi.x += yx; wi.y += yy; }
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t iu = i + u * warps;
+        nn[u] = iu < ntl ? s_n[iu] : 0u;
+        q[u] = region_batch(lrow + (r0 + iu) * kTile, 0, nn[u], lane);  // no read where nn[u] == 0
       }
-      s_warp[lane] = make_uint2(wi.x - w.x, wi.y - w.y);
-    }
-    __syncthreads();
-    const uint2 carry = *s_carry;
-    uint2 excl = make_uint2(carry.x + s_warp[wrp].x + incl.x - sum.x, carry.y + s_warp[wrp].y + incl.y - sum.y);
 #pragma unroll
-    for (int u = 0; u < ITEMS; ++u) {
-      s_item[tid * ITEMS + u] = excl;
-      excl.x += mine[u].x;
-      excl.y += mine[u].y;
+      for (int u = 0; u < 4; ++u) {
+        if (nn[u] == 0) continue;
+        const uint32_t iu = i + u * warps;
+        const uint2* reg = lrow + (r0 + iu) * kTile;
+        uint32_t run = base + s_off[iu];
+        put_candidates<HIST>(q[u], 2u * lane < nn[u], 2u * lane + 1u < nn[u], fhi, run, drow, cap, s_hist, lane);
+        for (uint32_t i0 = 64; i0 < nn[u]; i0 += 64)
+          put_candidates<HIST>(region_batch(reg, i0, nn[u], lane), i0 + 2u * lane < nn[u], i0 + 2u * lane + 1u < nn[u], fhi,
+                               run, drow, cap, s_hist, lane);
+      }
     }
-    __syncthreads();
-    if (tid == 1023) *s_carry = excl;  // the prefix after this round's last pair
-#pragma unroll
-    for (int u = 0; u < ITEMS; ++u) {
-      const uint64_t i = base + (uint64_t)u * 1024 + tid;
-      if (i < count) pre[i] = s_item[u * 1024 + tid];
-    }
-    __syncthreads();
+    __syncthreads();  // s_n, s_off and s_warp are rewritten by the next round
   }
-  __syncthreads();
-  return *s_carry;
+  return kept;
 }
 
-// Everything between pass1 (or mark, after a miss) and emit for one vector, by ONE 1024-thread CTA:
-// the verdict on the predicted band, the three radix digits of the threshold from the candidates'
-// keys, the per-tile counts of candidates at or above the threshold, and their exclusive prefix
-// over the tiles.  The candidates are few once the band has settled (a fraction of a percent of d),
-// so a single CTA per vector does in one launch what would otherwise be a chain of small kernels,
-// each waiting for the one before it.
-//
-// A thread owns the tiles tid, tid + 1024, ...; it walks the candidate region of each.  The first
-// walk also copies the keys into shared memory (kKeyCache of them; the later digits then run from
-// there; with more candidates they walk the regions again).
-//   PHASE 0, after pass1: needs a band to have been predicted and the k-th entry to be one of the
-//            candidates (above < k <= above + candidates); else the vector is flagged for the full
-//            route (hist, pick1, mark) and PHASE 1 finishes it.
-//   PHASE 1, after mark: the regions were rebuilt for the exact first digit; two digits remain.
-constexpr uint32_t kKeyCache = 32768;
-
-template <int PHASE>
-__global__ void __launch_bounds__(1024) k_topk_select(const uint32_t* cand_keys, uint64_t cap, uint4* tile_info, uint2* tile_pre,
-                                                      uint64_t ntile, TopkState* state, TopkPred* pred, uint32_t k,
-                                                      uint32_t* dev_status) {
+// After a miss: the candidates of the regions that mark rebuilt, made dense.
+__global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, uint64_t cap, const uint4* tile_info,
+                                                           uint64_t ntile, uint2* dense, uint32_t* dense_count,
+                                                           const TopkState* state) {
   pdl_prologue();
-  extern __shared__ uint32_t s_keys[];          // kKeyCache keys
-  __shared__ uint2 s_buf[4096];                 // histogram (as 4096 words), later the scan's items
-  __shared__ uint2 s_pair[32], s_carry;
+  __shared__ uint32_t s_n[kThreads], s_off[kThreads], s_warp[34];
+  const uint32_t row = blockIdx.y;
+  if (!state[row].need_mark) return;
+  gather_tiles<false>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile, dense + (uint64_t)row * cap, cap,
+                      &dense_count[row], (state[row].tb1 << 19) | 0x7FFFFu, nullptr, s_n, s_off, s_warp);
+}
+
+// ---------------------------------------------------------------- list histogram + pick
+// One radix digit from the candidate list: LEVEL 1 = key bits 30..19 (and the verdict on the
+// prediction), LEVEL 2 = bits 18..7, LEVEL 3 = bits 6..0 (tau and r complete; tau is remembered
+// for the next step's prediction).  Several CTAs per vector histogram slices of the list into the
+// vector's global histogram; the CTA that finishes last (a ticket counter, no waiting) picks the
+// digit and clears histogram and ticket.
+template <int LEVEL>
+__global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t cap, const uint4* tile_info, uint64_t ntile,
+                                                     uint2* dense, uint32_t* dense_count, uint32_t* kept_count,
+                                                     TopkState* state, uint32_t* hist, uint32_t* done, uint32_t k,
+                                                     TopkPred* pred, uint32_t* dev_status) {
+  pdl_prologue();
+  __shared__ uint32_t s_hist[kBins1];
   __shared__ uint32_t s_warp[34], s_out[3];
-  uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_buf);
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.x;
+  __shared__ uint32_t s_last, s_kept;
+  constexpr uint32_t NB = LEVEL == 3 ? 128u : 4096u;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   TopkState* st = state + row;
-  uint4* info = tile_info + (uint64_t)row * ntile;
-  const uint32_t* crow = cand_keys + (uint64_t)row * cap;
   uint32_t band_lo = 1, band_hi = 0;
-  if (PHASE == 0) {
-    if (!predicted_band(pred, row, &band_lo, &band_hi)) {   // pass1 had no band: nothing was listed
-      if (tid == 0) {
-        st->need_full = 1;
-        st->need_mark = 1;
-        atomicAdd(&dev_status[DS_DEV_WORD_TOPK_FULL], 1u);
-      }
-      return;
-    }
-  } else if (!st->need_mark) {
-    return;
-  }
-  // how many entries lie above the band and how many candidates there are
-  uint32_t above = 0, mine = 0;
-  for (uint64_t t = tid; t < ntile; t += 1024) {
-    const uint4 i4 = info[t];
-    const uint32_t listed = min(i4.x, (uint32_t)kTile), ab = min(i4.y, listed);
-    above += ab;
-    mine += listed - ab;
-  }
-  uint32_t n;
-  const uint32_t my_off = cta_excl_scan(mine, s_warp, &n);   // where this thread's keys start in the cache
-  above = __reduce_add_sync(0xffffffffu, above);
-  __syncthreads();                                           // s_warp is reused
-  if (lane == 0) s_warp[tid >> 5] = above;
+  // LEVEL 1 reads what pass1 wrote, which exists only if pass1 had a band to work with
+  const bool readable = LEVEL != 1 || predicted_band(pred, row, &band_lo, &band_hi);
+  const uint32_t tb1 = st->tb1, top24 = (st->tb1 << 12) | st->tb2;
+  for (uint32_t b = tid; b < NB; b += 1024) s_hist[b] = 0;
+  if (tid == 0) s_kept = 0;
   __syncthreads();
-  above = 0;
+  if constexpr (LEVEL == 1) {
+    __shared__ uint32_t s_n[1024], s_off[1024];
+    uint32_t kept = 0;
+    if (readable)
+      kept = gather_tiles<true>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile,
+                                dense + (uint64_t)row * cap, cap, &dense_count[row], band_hi, s_hist, s_n, s_off, s_warp);
+    kept = __reduce_add_sync(0xffffffffu, kept);
+    if (lane == 0 && kept) atomicAdd(&s_kept, kept);
+  } else {
+    const uint2* drow = dense + (uint64_t)row * cap;
+    const uint64_t n = min((uint64_t)dense_count[row], cap);
+    const uint64_t step = (uint64_t)gridDim.x * 8 * 1024;
+    for (uint64_t i0 = (uint64_t)blockIdx.x * 8 * 1024; i0 < n; i0 += step) {
+      uint32_t key[8];
 #pragma unroll
-  for (int w = 0; w < 32; ++w) above += s_warp[w];
-  __syncthreads();
-  uint32_t want, tb1 = 0;
-  if (PHASE == 0) {
-    // the prediction holds iff the k-th largest entry is one of the candidates
-    if (!(above < k && k - above <= n)) {
-      if (tid == 0) {
-        st->need_full = 1;   // hist, pick1 and mark rebuild the regions for the exact first digit
-        st->need_mark = 1;
-        atomicAdd(&dev_status[DS_DEV_WORD_TOPK_FULL], 1u);
+      for (int u = 0; u < 8; ++u) {
+        const uint64_t i = i0 + (uint64_t)u * 1024 + tid;
+        key[u] = i < n ? drow[i].x : 0xFFFFFFFFu;  // bit 31 set: matches no bin and no prefix
       }
-      return;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (LEVEL == 2) {
+          if ((key[u] >> 19) == tb1) atomicAdd(&s_hist[(key[u] >> 7) & 0xFFFu], 1u);
+        } else {
+          if ((key[u] >> 7) == top24) atomicAdd(&s_hist[key[u] & 0x7Fu], 1u);
+        }
+      }
     }
-    want = k - above;
-  } else {
-    want = st->k_rem;
-    tb1 = st->tb1;
   }
-  const bool cached = n <= kKeyCache;
-
-  // one radix digit: histogram of digit(key) over the candidates that pass `keep`, then the pick
-  auto walk_regions = [&](auto&& f) {
-    for (uint64_t t = tid; t < ntile; t += 1024) {
-      const uint4 i4 = info[t];
-      const uint32_t listed = min(i4.x, (uint32_t)kTile), c = listed - min(i4.y, listed);
-      const uint32_t* ck = crow + t * kTile;
-      for (uint32_t i = 0; i < c; ++i) f(ck[i]);
-    }
-  };
-  auto walk_cache = [&](auto&& f) {
-    for (uint32_t i = tid; i < n; i += 1024) f(s_keys[i]);
-  };
-  auto clear_hist = [&]() {
-    for (uint32_t b = tid; b < kBins1; b += 1024) s_hist[b] = 0;
-    if (tid == 0) { s_out[0] = 0; s_out[1] = 0; s_out[2] = 0; }
-    __syncthreads();
-  };
-
-  bool have_cache = false;
-  if (PHASE == 0) {
-    clear_hist();
-    uint32_t at = my_off;
-    walk_regions([&](uint32_t key) {
-      if (cached) s_keys[at++] = key;
-      atomicAdd(&s_hist[key >> 19], 1u);
-    });
-    have_cache = cached;
-    __syncthreads();
-    cta_pick(s_hist, want, s_warp, s_out);
-    tb1 = s_out[0];
-    want = s_out[1];
-    __syncthreads();
+  __syncthreads();
+  uint32_t* h = hist + (uint64_t)row * kBins1;
+  for (uint32_t b = tid; b < NB; b += 1024) {
+    const uint32_t c = s_hist[b];
+    if (c) atomicAdd(&h[b], c);
   }
-  // second digit: key bits 18..7 of the candidates inside the first digit's bin
-  clear_hist();
-  if (have_cache) {
-    walk_cache([&](uint32_t key) { if ((key >> 19) == tb1) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u); });
-  } else {
-    uint32_t at = my_off;
-    walk_regions([&](uint32_t key) {
-      if (cached) s_keys[at++] = key;
-      if ((key >> 19) == tb1) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
-    });
-    have_cache = cached;
+  if (LEVEL == 1 && tid == 0 && s_kept) atomicAdd(&kept_count[row], s_kept);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&done[row], 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // every CTA of this vector has flushed: read the complete histogram past L1, pick, clear
+  for (uint32_t b = tid; b < kBins1; b += 1024) {
+    s_hist[b] = b < NB ? __ldcg(&h[b]) : 0u;
+    if (b < NB) h[b] = 0;
   }
+  uint32_t want = st->k_rem;
+  if (LEVEL == 1) {
+    const uint32_t kept = __ldcg(&kept_count[row]);
+    want = kept < k ? k - kept : 0u;  // 0: the threshold lies above the band
+  }
+  if (tid == 0) { s_out[0] = 0; s_out[1] = 0; s_out[2] = 0; done[row] = 0; }
   __syncthreads();
   cta_pick(s_hist, want, s_warp, s_out);
-  const uint32_t top24 = (tb1 << 12) | s_out[0];
-  want = s_out[1];
-  __syncthreads();
-  // third digit: key bits 6..0
-  clear_hist();
-  if (have_cache) walk_cache([&](uint32_t key) { if ((key >> 7) == top24) atomicAdd(&s_hist[key & 0x7Fu], 1u); });
-  else walk_regions([&](uint32_t key) { if ((key >> 7) == top24) atomicAdd(&s_hist[key & 0x7Fu], 1u); });
-  __syncthreads();
-  cta_pick(s_hist, want, s_warp, s_out);
-  const uint32_t tau = (top24 << 7) | s_out[0], r = s_out[1];
-  __syncthreads();
-
-  // per tile: candidates above tau (.z) and equal to it (.w), beside the tile's counts
-  for (uint64_t t = tid; t < ntile; t += 1024) {
-    const uint4 i4 = info[t];
-    const uint32_t listed = min(i4.x, (uint32_t)kTile), c = listed - min(i4.y, listed);
-    const uint32_t* ck = crow + t * kTile;
-    uint32_t gt = 0, eq = 0;
-    for (uint32_t i = 0; i < c; ++i) {
-      const uint32_t key = ck[i];
-      gt += key > tau ? 1u : 0u;
-      eq += key == tau ? 1u : 0u;
-    }
-    info[t] = make_uint4(i4.x, i4.y, gt, eq);
-  }
-  __syncthreads();   // the scan below reads what other threads of this CTA just wrote
-  const uint2 tot = cta_scan_pairs(ntile, [&](uint64_t i) {
-    const uint4 t4 = info[i];
-    return make_uint2(min(t4.y, min(t4.x, (uint32_t)kTile)) + t4.z, t4.w);  // above the band + candidates above tau; ties
-  }, tile_pre + (uint64_t)row * ntile, s_buf, s_pair, &s_carry);
   if (tid != 0) return;
-  st->tb1 = tb1;
-  st->tb2 = top24 & 0xFFFu;
-  st->tau = tau;
-  st->r = r;
-  st->k_rem = r;
-  st->total_gt = tot.x;
-  st->total_tie = tot.y;
-  if (tot.x + min(tot.y, r) != k) atomicOr(&dev_status[DS_DEV_WORD_FLAGS], DS_DEV_TOPK_INCONSISTENT);
-  if (PHASE == 0) {
-    st->need_full = 0;
-    st->need_mark = 0;
-    st->zeroed_above = band_hi;
-    atomicAdd(&dev_status[DS_DEV_WORD_TOPK_PREDICTED], 1u);
-  }
-  if (pred) {
-    // remember tau for the next step's band, and how far the extrapolation was off
-    uint32_t lo = 1, hi = 0, centre = 0;
-    const bool had = predicted_band(pred, row, &lo, &hi, &centre);
-    TopkPred np;
-    np.magic = kPredMagic;
-    np.tau_prev = had ? pred[row].tau_last : tau;
-    np.tau_last = tau;
-    if (had) {
-      const uint32_t e = tau > centre ? tau - centre : centre - tau;
-      const uint32_t old = min(pred[row].err, kMaxErr);
-      np.err = min(kMaxErr, max(old - (old >> 2), e));
+  if (LEVEL == 1) {
+    // the prediction holds iff the k-th largest entry is one of the listed candidates
+    const bool hit = readable && want >= 1 && want <= s_out[2];
+    atomicAdd(&dev_status[hit ? DS_DEV_WORD_TOPK_PREDICTED : DS_DEV_WORD_TOPK_FULL], 1u);  // one per selection
+    if (hit) {
+      st->tb1 = s_out[0];
+      st->k_rem = s_out[1];
+      st->need_full = 0;
+      st->need_mark = 0;
+      st->zeroed_above = band_hi;
     } else {
-      np.err = kFirstErr;
+      st->need_full = 1;  // hist, pick, mark and compact rebuild the regions and the list for the exact bin
+      st->need_mark = 1;
+      dense_count[row] = 0;
     }
-    pred[row] = np;
+  } else if (LEVEL == 2) {
+    st->tb2 = s_out[0];
+    st->k_rem = s_out[1];
+  } else {
+    const uint32_t tau = (top24 << 7) | s_out[0];
+    st->tau = tau;
+    st->r = s_out[1];
+    st->k_rem = s_out[1];
+    if (pred) {
+      uint32_t lo = 1, hi = 0, centre = 0;
+      const bool had = predicted_band(pred, row, &lo, &hi, &centre);
+      TopkPred np;
+      np.magic = kPredMagic;
+      np.tau_prev = had ? pred[row].tau_last : tau;
+      np.tau_last = tau;
+      if (had) {
+        const uint32_t e = tau > centre ? tau - centre : centre - tau;
+        const uint32_t old = min(pred[row].err, kMaxErr);
+        np.err = min(kMaxErr, max(old - (old >> 2), e));
+      } else {
+        np.err = kFirstErr;
+      }
+      pred[row] = np;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- classify
+// Per tile, how many of its candidates lie above tau (z) and how many equal it (w): the counters
+// pass1 / mark left at zero beside the tile's counts.  A tile's candidates are neighbours in the
+// dense list, so the lanes of a warp that count for the same counter send one atomic between
+// them.  Integer atomics: order-free.
+__global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* dense, const uint32_t* dense_count, uint64_t cap,
+                                                            const TopkState* state, uint4* tile_info, uint64_t ntile) {
+  pdl_prologue();
+  const uint32_t row = blockIdx.y, lane = threadIdx.x & 31u;
+  const uint2* drow = dense + (uint64_t)row * cap;
+  const uint64_t n = min((uint64_t)dense_count[row], cap);
+  const uint32_t tau = state[row].tau;
+  uint32_t* counters = reinterpret_cast<uint32_t*>(tile_info + (uint64_t)row * ntile);
+  const uint64_t step = (uint64_t)gridDim.x * kThreads * 4;
+  // the loop bound is the same for all lanes of a warp (i0 - threadIdx.x is), as match needs
+  for (uint64_t c0 = (uint64_t)blockIdx.x * kThreads * 4; c0 < n; c0 += step) {
+    const uint64_t i0 = c0 + threadIdx.x;
+    uint2 e[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = i0 + (uint64_t)u * kThreads;
+      e[u] = i < n ? drow[i] : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t t = e[u].y >> 12;
+      const bool live = i0 + (uint64_t)u * kThreads < n && t < ntile && e[u].x >= tau;
+      // word index of the counter inside the vector's tile_info: .z for "above", .w for "equal"
+      const uint32_t word = live ? (uint32_t)t * 4u + (e[u].x > tau ? 2u : 3u) : 0xFFFFFFFFu;
+      const uint32_t peers = __match_any_sync(0xffffffffu, word);
+      if (live && lane == (uint32_t)__ffs(peers) - 1u) atomicAdd(&counters[word], (uint32_t)__popc(peers));
+    }
   }
 }
 
@@ -1009,18 +983,84 @@ __global__ void __launch_bounds__(kThreads) k_topk_finalize(const float* v_in, u
 
 // ================================================================ shared tail
 
-// Exclusive prefix of the per-segment counts of one vector (in place); checks that exactly k entries
-// will be emitted.
-__global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, uint64_t nseg, TopkState* state, uint32_t k,
-                                                    uint32_t* dev_status) {
+// Exclusive prefix of the per-segment counts of one vector (in place), or with TILES of the
+// per-tile counts in tile_info (written to seg_cnt); checks that exactly k entries will be emitted.
+template <bool TILES>
+__global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4* tile_info, uint64_t nseg, TopkState* state,
+                                                    uint32_t k, uint32_t* dev_status) {
   pdl_prologue();
-  __shared__ uint2 s_item[4096];
+  // A round takes 4096 counts: loaded and stored with neighbouring threads on neighbouring counts,
+  // scanned with four consecutive counts per thread; shared memory turns one order into the other.
+  constexpr int ITEMS = 4;
+  __shared__ uint2 s_item[1024 * ITEMS];
   __shared__ uint2 s_warp[32];
   __shared__ uint2 s_carry;
-  const uint32_t row = blockIdx.x;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.x;
   uint2* c = seg_cnt + (uint64_t)row * nseg;
-  const uint2 tot = cta_scan_pairs(nseg, [&](uint64_t i) { return c[i]; }, c, s_item, s_warp, &s_carry);
-  if (threadIdx.x == 0) {
+  if (tid == 0) s_carry = make_uint2(0, 0);
+  for (uint64_t base = 0; base < nseg; base += 1024 * ITEMS) {
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      const uint64_t i = base + (uint64_t)u * 1024 + tid;
+      uint2 item = make_uint2(0, 0);
+      if (i < nseg) {
+        if (TILES) {
+          const uint4 t = tile_info[(uint64_t)row * nseg + i];
+          item = make_uint2(t.y + t.z, t.w);  // above the band + candidates above tau; candidates equal to tau
+        } else {
+          item = c[i];
+        }
+      }
+      s_item[u * 1024 + tid] = item;
+    }
+    __syncthreads();
+    uint2 mine[ITEMS];
+    uint2 sum = make_uint2(0, 0);
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      mine[u] = s_item[tid * ITEMS + u];
+      sum.x += mine[u].x;
+      sum.y += mine[u].y;
+    }
+    uint2 incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t yx = __shfl_up_sync(0xffffffffu, incl.x, o), yy = __shfl_up_sync(0xffffffffu, incl.y, o);
+      if (lane >= (uint32_t)o) { incl.x += yx; incl.y += yy; }
+    }
+    if (lane == 31) s_warp[wrp] = incl;
+    __syncthreads();
+    if (wrp == 0) {
+      const uint2 w = s_warp[lane];
+      uint2 wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t yx = __shfl_up_sync(0xffffffffu, wi.x, o), yy = __shfl_up_sync(0xffffffffu, wi.y, o);
+        if (lane >= (uint32_t)o) { wi.x += yx; wi.y += yy; }
+      }
+      s_warp[lane] = make_uint2(wi.x - w.x, wi.y - w.y);
+    }
+    __syncthreads();
+    const uint2 carry = s_carry;
+    uint2 excl = make_uint2(carry.x + s_warp[wrp].x + incl.x - sum.x, carry.y + s_warp[wrp].y + incl.y - sum.y);
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      s_item[tid * ITEMS + u] = excl;
+      excl.x += mine[u].x;
+      excl.y += mine[u].y;
+    }
+    __syncthreads();
+    if (tid == 1023) s_carry = excl;  // the prefix after this round's last count
+#pragma unroll
+    for (int u = 0; u < ITEMS; ++u) {
+      const uint64_t i = base + (uint64_t)u * 1024 + tid;
+      if (i < nseg) c[i] = s_item[u * 1024 + tid];
+    }
+    __syncthreads();
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const uint2 tot = s_carry;
     const uint32_t r = state[row].r;
     state[row].total_gt = tot.x;
     state[row].total_tie = tot.y;
@@ -1150,7 +1190,7 @@ void topk_plan(uint64_t d, uint32_t rows, uint64_t k, bool with_list, TopkPlan* 
   p->off_seg = pos;        pos = round16(pos + (uint64_t)rows * (with_list ? p->ntile : p->nseg) * sizeof(uint2));
   p->off_list = pos;       pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint2));
   p->off_tile_info = pos;  pos = round16(pos + (with_list ? (uint64_t)rows * p->ntile * sizeof(uint4) : 0));
-  p->off_dense = pos;      pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint32_t));
+  p->off_dense = pos;      pos = round16(pos + (uint64_t)rows * p->list_cap * sizeof(uint2));
   p->bytes = pos;
   p->pred = nullptr;
 }
@@ -1166,7 +1206,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   uint2* seg = reinterpret_cast<uint2*>(ws + pl.off_seg);
   uint2* list = pl.list_cap ? reinterpret_cast<uint2*>(ws + pl.off_list) : nullptr;
   uint4* tile_info = reinterpret_cast<uint4*>(ws + pl.off_tile_info);
-  uint32_t* cand_keys = reinterpret_cast<uint32_t*>(ws + pl.off_dense);  // candidate keys, one region of kTile per tile
+  uint2* dense = reinterpret_cast<uint2*>(ws + pl.off_dense);
   const uint64_t d = src.d, cap = pl.list_cap;
   const uint64_t padded = pl.nseg * (uint64_t)kSegElems;
   uint32_t* done = list_count + rows;        // ticket counters of the list histograms
@@ -1192,22 +1232,31 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
 
   if (list && k) {
     TopkPred* pred = pl.pred;
-#define DSQ_P1(S) launch_pdl(k_topk_pass1<S>, g1, kThreads, st, src, io.v_inout, pred, list, cand_keys, cap, tile_info, pl.ntile)
+#define DSQ_P1(S) launch_pdl(k_topk_pass1<S>, g1, kThreads, st, src, io.v_inout, pred, list, cap, tile_info, pl.ntile)
     DSQ_SWITCH_SRC(srck, DSQ_P1)
 #undef DSQ_P1
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    launch_pdl_smem(k_topk_select<0>, rows, 1024, kKeyCache * 4, st, cand_keys, cap, tile_info, seg, pl.ntile, state, pred, k32,
-                    io.dev_status);
+    // level 1 keeps a whole SM per CTA (registers), so its grid is one wave; levels 2 and 3 fit two per SM
+    dim3 gl1((unsigned)(148ull / rows ? 148ull / rows : 1), rows, 1);
+    dim3 gl((unsigned)(148ull * 2ull / rows ? 148ull * 2ull / rows : 1), rows, 1);
+    launch_pdl(k_topk_lhist<1>, gl1, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+                                         k32, pred, io.dev_status);
     launch_pdl(k_topk_hist, gm, kThreads, st, io.v_inout, d, src.vec, io.keep_error, state, pred, list, cap, tile_info, hist);
     launch_pdl(k_topk_pick1, rows, 1024, st, hist, state, k32);
-    launch_pdl(k_topk_mark, gm, kThreads, st, io.v_inout, d, src.vec, io.keep_error, state, list, cand_keys, cap, tile_info, pl.ntile);
-    launch_pdl_smem(k_topk_select<1>, rows, 1024, kKeyCache * 4, st, cand_keys, cap, tile_info, seg, pl.ntile, state, pred, k32,
-                    io.dev_status);
+    launch_pdl(k_topk_mark, gm, kThreads, st, io.v_inout, d, src.vec, io.keep_error, state, list, cap, tile_info, pl.ntile);
+    launch_pdl(k_topk_compact, gm, kThreads, st, list, cap, tile_info, pl.ntile, dense, list_count, state);
+    launch_pdl(k_topk_lhist<2>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+                                         k32, pred, io.dev_status);
+    launch_pdl(k_topk_lhist<3>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
+                                         k32, pred, io.dev_status);
+    dim3 gc((unsigned)(148ull * 8ull / rows ? 148ull * 8ull / rows : 1), rows, 1);
+    launch_pdl(k_topk_classify, gc, kThreads, st, dense, list_count, cap, state, tile_info, pl.ntile);
+    launch_pdl(k_topk_scan<true>, rows, 1024, st, seg, tile_info, pl.ntile, state, k32, io.dev_status);
     dim3 ge((unsigned)((pl.ntile + kThreads / 32 - 1) / (kThreads / 32)), rows, 1);
     launch_pdl(k_topk_emit_list, ge, kThreads, st, io.v_inout, d, state, list, cap, tile_info, seg, pl.ntile,
                                               reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x,
                                               io.gamma, io.keep_error);
-    count_launches(7);
+    count_launches(11);
     return cudaGetLastError();
   } else {
 #define DSQ_P1(S) launch_pdl(k_topk_pass1_basic<S>, g1b, kThreads, st, src, io.v_inout, hist, span)
@@ -1225,7 +1274,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     launch_pdl(k_topk_finalize, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
     count_launches(7);
   }
-  launch_pdl(k_topk_scan, rows, 1024, st, seg, pl.nseg, state, k32, io.dev_status);
+  launch_pdl(k_topk_scan<false>, rows, 1024, st, seg, nullptr, pl.nseg, state, k32, io.dev_status);
   launch_pdl(k_topk_emit, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg,
                                        reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x, io.gamma);
   count_launches(2);
