@@ -243,7 +243,8 @@ int ds_worker_compress(ds_handle h, const float* g, uint32_t step, void* cuda_st
  * Algorithm 1, "On parameter server" (Eq. 4): decode the n worker payloads, average in worker
  * order, add delta_s, compress, keep the residual.  Writes server_payload and delta_s; with
  * DS_FUSE_APPLY also updates x and completes the step.  DS_ERR_STATE unless ds_worker_compress
- * was the previous call.
+ * was the previous call.  worker_payload and workspace are read as that call left them (a TOPK worker pass
+ * leaves an index of its payloads in the workspace): do not modify either between the two calls.
  */
 int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, void* cuda_stream);
 

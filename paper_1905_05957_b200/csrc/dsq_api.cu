@@ -91,6 +91,7 @@ struct ds_ctx {
   uint32_t* acc_offsets;  // span offsets of the sparse payloads (inside workspace), or NULL
   void* whole;            // scratch of the operators with one factor per vector (inside workspace), or NULL
   int phase;              // 0: step complete, 1: worker pass done, 2: unfused server pass done
+  bool offsets_ready;     // the worker pass that just ran left the span table of its sparse payloads in acc_offsets
 };
 
 namespace {
@@ -260,6 +261,8 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
       io.payload_stride = L.stride;
       io.v_inout = delta;  // v is written over delta, then the kept entries are zeroed: delta = v - Q[v]
       io.keep_error = 1;
+      // the whole-vector worker pass hands the server the span table of its index lists
+      io.span_off = (!server && !win && q.k > 0) ? c->acc_offsets : nullptr;
       if (src_kind == SRC_WORKER_PLAIN) {
         // no error is kept: v is the gradient itself, selected where it lies and never written
         if (q.k == 0) return DS_OK;  // nothing to send, nothing to keep
@@ -368,7 +371,10 @@ int ds_worker_compress(ds_handle h, const float* g, uint32_t step, void* cuda_st
   const int rc = run_pass(h, nocomp ? SRC_WORKER_PLAIN : SRC_WORKER, src, h->cfg.worker_q, h->wl,
                           static_cast<uint8_t*>(h->buf.worker_payload), nocomp ? nullptr : h->buf.delta_w, h->cfg.n, false,
                           nullptr, step, st);
-  if (rc == DS_OK) h->phase = 1;
+  if (rc == DS_OK) {
+    h->phase = 1;
+    h->offsets_ready = h->cfg.worker_q.op == DS_Q_TOPK && h->cfg.worker_q.k > 0;
+  }
   return rc;
 }
 
@@ -382,7 +388,8 @@ int ds_server_aggregate_compress(ds_handle h, uint32_t step, uint32_t flags, voi
     // (1/n) sum_i Q[v_i] for sparse payloads: dense accumulator, workers added in order 0..n-1
     const cudaError_t e = launch_sparse_accumulate(static_cast<const uint8_t*>(h->buf.worker_payload), h->wl.stride,
                                                    h->wl.off[0], h->wl.off[1], h->cfg.n, h->cfg.worker_q.k, h->cfg.d,
-                                                   h->acc_offsets, h->acc, st);
+                                                   h->acc_offsets, h->offsets_ready, h->acc, st);
+    h->offsets_ready = false;
     if (e != cudaSuccess) return cuda_fail(e, "sparse accumulate");
   }
   const bool fuse = (flags & DS_FUSE_APPLY) != 0;

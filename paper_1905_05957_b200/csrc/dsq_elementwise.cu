@@ -289,7 +289,7 @@ cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamm
 // entries of eight workers are fetched at once, then added worker by worker with a barrier in
 // between (indices inside one payload are distinct, so one worker's additions never collide), and
 // the finished slice is written out whole -- the accumulator needs no clearing beforehand.
-constexpr uint32_t kAccSpan = 8192;
+constexpr uint32_t kAccSpan = kSparseSpan;
 
 __global__ void __launch_bounds__(kThreads) k_sparse_offsets(const uint8_t* __restrict__ wp, uint64_t stride, uint64_t off_idx,
                                                              uint64_t k, uint64_t nspan, uint32_t* off) {
@@ -369,13 +369,16 @@ __global__ void __launch_bounds__(kThreads) k_sparse_accumulate(const uint8_t* _
 uint64_t sparse_offsets_bytes(uint32_t n, uint64_t d) { return (uint64_t)n * ((d + kAccSpan - 1) / kAccSpan + 1) * 4; }
 
 cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_t off_idx, uint64_t off_val, uint32_t n,
-                                     uint64_t k, uint64_t d, uint32_t* offsets, float* acc, cudaStream_t st) {
+                                     uint64_t k, uint64_t d, uint32_t* offsets, bool offsets_ready, float* acc, cudaStream_t st) {
   const uint64_t nspan = (d + kAccSpan - 1) / kAccSpan;
-  uint64_t ctas = (k + kThreads) / kThreads;
-  if (ctas > 148 * 8) ctas = 148 * 8;
-  launch_pdl(k_sparse_offsets, dim3((unsigned)ctas, n, 1), kThreads, st, wp, stride, off_idx, k, nspan, offsets);
+  if (!offsets_ready) {
+    uint64_t ctas = (k + kThreads) / kThreads;
+    if (ctas > 148 * 8) ctas = 148 * 8;
+    launch_pdl(k_sparse_offsets, dim3((unsigned)ctas, n, 1), kThreads, st, wp, stride, off_idx, k, nspan, offsets);
+    count_launches(1);
+  }
   launch_pdl(k_sparse_accumulate, (unsigned)nspan, kThreads, st, wp, stride, off_idx, off_val, n, d, nspan, offsets, acc);
-  count_launches(2);
+  count_launches(1);
   return cudaGetLastError();
 }
 

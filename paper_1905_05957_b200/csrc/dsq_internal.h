@@ -139,6 +139,8 @@ struct TopkIO {
   float* v_inout;           // [rows, d]: receives v, then has the kept entries zeroed (the residual).  With
                             // keep_error = 0 (source SRC_WORKER_PLAIN): where v already lies (the gradient); only read
   int keep_error;
+  uint32_t* span_off;       // non-NULL: also receives, per vector, where every span of kSparseSpan indices begins in
+                            // the emitted index list ([rows, nspan + 1]; the table launch_sparse_accumulate works from)
   float* x;                 // non-NULL: fused model update at the kept entries (server pass)
   float gamma;
   uint32_t* dev_status;
@@ -197,9 +199,11 @@ cudaError_t launch_whole(int op, int src_kind, const SrcParams& src, const Whole
 cudaError_t launch_apply(const PayloadView& pv, float* x, uint64_t d, float gamma, cudaStream_t st);
 
 // acc[j] = sum over workers i = 0..n-1, in that order, of the value worker i's sparse payload holds for j
-// (every entry of acc is written).  offsets: scratch of sparse_offsets_bytes(n, d) bytes.
+// (every entry of acc is written).  offsets: scratch of sparse_offsets_bytes(n, d) bytes; offsets_ready: the
+// table in it is already filled (by the top-k pass that wrote these payloads), else it is built first.
+constexpr uint32_t kSparseSpan = 8192;   // indices per span of the table
 uint64_t sparse_offsets_bytes(uint32_t n, uint64_t d);
 cudaError_t launch_sparse_accumulate(const uint8_t* wp, uint64_t stride, uint64_t off_idx, uint64_t off_val, uint32_t n,
-                                     uint64_t k, uint64_t d, uint32_t* offsets, float* acc, cudaStream_t st);
+                                     uint64_t k, uint64_t d, uint32_t* offsets, bool offsets_ready, float* acc, cudaStream_t st);
 
 }  // namespace dsq

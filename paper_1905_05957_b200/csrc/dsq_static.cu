@@ -70,6 +70,7 @@ extern "C" int ds_topk_worker_static(const float* g, float* delta, uint64_t d, u
   io.payload_stride = 0;  // a single vector
   io.v_inout = delta;
   io.keep_error = 1;
+  io.span_off = nullptr;
   io.x = nullptr;
   io.gamma = 0.f;
   io.dev_status = dev_status;

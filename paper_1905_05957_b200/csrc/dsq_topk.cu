@@ -664,41 +664,6 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
   }
 }
 
-// ---------------------------------------------------------------- classify
-// Per tile, how many of its candidates lie above tau (z) and how many equal it (w): the counters
-// pass1 / mark left at zero beside the tile's counts.  A tile's candidates are neighbours in the
-// dense list, so the lanes of a warp that count for the same counter send one atomic between
-// them.  Integer atomics: order-free.
-__global__ void __launch_bounds__(kThreads) k_topk_classify(const uint2* dense, const uint32_t* dense_count, uint64_t cap,
-                                                            const TopkState* state, uint4* tile_info, uint64_t ntile) {
-  pdl_prologue();
-  const uint32_t row = blockIdx.y, lane = threadIdx.x & 31u;
-  const uint2* drow = dense + (uint64_t)row * cap;
-  const uint64_t n = min((uint64_t)dense_count[row], cap);
-  const uint32_t tau = state[row].tau;
-  uint32_t* counters = reinterpret_cast<uint32_t*>(tile_info + (uint64_t)row * ntile);
-  const uint64_t step = (uint64_t)gridDim.x * kThreads * 4;
-  // the loop bound is the same for all lanes of a warp (i0 - threadIdx.x is), as match needs
-  for (uint64_t c0 = (uint64_t)blockIdx.x * kThreads * 4; c0 < n; c0 += step) {
-    const uint64_t i0 = c0 + threadIdx.x;
-    uint2 e[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint64_t i = i0 + (uint64_t)u * kThreads;
-      e[u] = i < n ? drow[i] : make_uint2(0u, 0u);
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint64_t t = e[u].y >> 12;
-      const bool live = i0 + (uint64_t)u * kThreads < n && t < ntile && e[u].x >= tau;
-      // word index of the counter inside the vector's tile_info: .z for "above", .w for "equal"
-      const uint32_t word = live ? (uint32_t)t * 4u + (e[u].x > tau ? 2u : 3u) : 0xFFFFFFFFu;
-      const uint32_t peers = __match_any_sync(0xffffffffu, word);
-      if (live && lane == (uint32_t)__ffs(peers) - 1u) atomicAdd(&counters[word], (uint32_t)__popc(peers));
-    }
-  }
-}
-
 // ---------------------------------------------------------------- emit from the tile regions
 // A warp per tile.  The region lists, in index order, every entry that can be kept; the scan gave
 // the tile its first output slot (and the number of ties before it), so a ballot per 32 entries
@@ -708,7 +673,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit_list(float* v_io, uint64
                                                              uint64_t cap, const uint4* tile_info, const uint2* tile_pre,
                                                              uint64_t ntile, uint8_t* payload, uint64_t payload_stride,
                                                              uint64_t off_idx, uint64_t off_val, uint32_t k, float* x,
-                                                             float gamma, int keep_error) {
+                                                             float gamma, int keep_error, uint32_t* span_off) {
   pdl_prologue();
   const uint32_t tid = threadIdx.x, lane = tid & 31u, row = blockIdx.y;
   const uint64_t tile = (uint64_t)blockIdx.x * (kThreads / 32) + (tid >> 5);
@@ -720,12 +685,21 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit_list(float* v_io, uint64
   const uint4 info = tile_info[(uint64_t)row * ntile + tile];
   const uint2 pre = tile_pre[(uint64_t)row * ntile + tile];
   const uint32_t n = min(info.x, (uint32_t)kTile);
-  if (n == 0) return;
   const uint32_t tau = state[row].tau, r = state[row].r, zeroed_above = state[row].zeroed_above;
   const bool ties = info.w != 0;  // the tile holds an entry equal to tau
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t ties_before = pre.y;
   uint32_t run = pre.x + min(pre.y, r);
+  if (span_off && lane == 0) {
+    // where every span of kSparseSpan indices begins in this vector's ascending index list: the table
+    // the ordered sum of sparse payloads works from (a span is a whole number of tiles)
+    constexpr uint64_t tps = kSparseSpan / kTile;
+    const uint64_t nspan = (ntile + tps - 1) / tps;
+    uint32_t* o = span_off + (uint64_t)row * (nspan + 1);
+    if (tile % tps == 0) o[tile / tps] = run;
+    if (tile == 0) o[nspan] = k;
+  }
+  if (n == 0) return;
   float* vrow = v_io + (uint64_t)row * d;
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(payload + (uint64_t)row * payload_stride + off_idx);
   float* out_val = reinterpret_cast<float*>(payload + (uint64_t)row * payload_stride + off_val);
@@ -985,17 +959,17 @@ __global__ void __launch_bounds__(kThreads) k_topk_finalize(const float* v_in, u
 
 // Exclusive prefix of the per-segment counts of one vector (in place), or with TILES of the
 // per-tile counts in tile_info (written to seg_cnt); checks that exactly k entries will be emitted.
+// Called by all 1024 threads of a CTA.
 template <bool TILES>
-__global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4* tile_info, uint64_t nseg, TopkState* state,
-                                                    uint32_t k, uint32_t* dev_status) {
-  pdl_prologue();
+__device__ __forceinline__ void cta_scan_counts(uint32_t row, uint2* seg_cnt, const uint4* tile_info, uint64_t nseg,
+                                                TopkState* state, uint32_t k, uint32_t* dev_status) {
   // A round takes 4096 counts: loaded and stored with neighbouring threads on neighbouring counts,
   // scanned with four consecutive counts per thread; shared memory turns one order into the other.
   constexpr int ITEMS = 4;
   __shared__ uint2 s_item[1024 * ITEMS];
   __shared__ uint2 s_warp[32];
   __shared__ uint2 s_carry;
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.x;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5;
   uint2* c = seg_cnt + (uint64_t)row * nseg;
   if (tid == 0) s_carry = make_uint2(0, 0);
   for (uint64_t base = 0; base < nseg; base += 1024 * ITEMS) {
@@ -1005,7 +979,7 @@ __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4*
       uint2 item = make_uint2(0, 0);
       if (i < nseg) {
         if (TILES) {
-          const uint4 t = tile_info[(uint64_t)row * nseg + i];
+          const uint4 t = __ldcg(&tile_info[(uint64_t)row * nseg + i]);   // other CTAs counted into it just now
           item = make_uint2(t.y + t.z, t.w);  // above the band + candidates above tau; candidates equal to tau
         } else {
           item = c[i];
@@ -1066,6 +1040,59 @@ __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, const uint4*
     state[row].total_tie = tot.y;
     if (tot.x + min(tot.y, r) != k) atomicOr(dev_status, DS_DEV_TOPK_INCONSISTENT);
   }
+}
+
+// Pipeline without a list: the prefix over the segment counts, one CTA per vector.
+__global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, uint64_t nseg, TopkState* state, uint32_t k,
+                                                    uint32_t* dev_status) {
+  pdl_prologue();
+  cta_scan_counts<false>(blockIdx.x, seg_cnt, nullptr, nseg, state, k, dev_status);
+}
+
+// ---------------------------------------------------------------- classify + prefix
+// Per tile, how many of its candidates lie above tau (z) and how many equal it (w): the counters
+// pass1 / mark left at zero beside the tile's counts.  A tile's candidates are neighbours in the
+// dense list, so the lanes of a warp that count for the same counter send one atomic between
+// them.  Integer atomics: order-free.  The CTA of a vector that finishes last (a ticket counter, no
+// waiting) then takes the exclusive prefix over the vector's tiles, which saves a launch.
+__global__ void __launch_bounds__(1024) k_topk_classify(const uint2* dense, const uint32_t* dense_count, uint64_t cap,
+                                                        TopkState* state, uint4* tile_info, uint2* tile_pre, uint64_t ntile,
+                                                        uint32_t* done, uint32_t k, uint32_t* dev_status) {
+  pdl_prologue();
+  __shared__ uint32_t s_last;
+  const uint32_t row = blockIdx.y, tid = threadIdx.x, lane = tid & 31u;
+  const uint2* drow = dense + (uint64_t)row * cap;
+  const uint64_t n = min((uint64_t)dense_count[row], cap);
+  const uint32_t tau = state[row].tau;
+  uint32_t* counters = reinterpret_cast<uint32_t*>(tile_info + (uint64_t)row * ntile);
+  const uint64_t step = (uint64_t)gridDim.x * 1024 * 4;
+  // the loop bound is the same for all lanes of a warp (i0 - threadIdx.x is), as match needs
+  for (uint64_t c0 = (uint64_t)blockIdx.x * 1024 * 4; c0 < n; c0 += step) {
+    const uint64_t i0 = c0 + tid;
+    uint2 e[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t i = i0 + (uint64_t)u * 1024;
+      e[u] = i < n ? drow[i] : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint64_t t = e[u].y >> 12;
+      const bool live = i0 + (uint64_t)u * 1024 < n && t < ntile && e[u].x >= tau;
+      // word index of the counter inside the vector's tile_info: .z for "above", .w for "equal"
+      const uint32_t word = live ? (uint32_t)t * 4u + (e[u].x > tau ? 2u : 3u) : 0xFFFFFFFFu;
+      const uint32_t peers = __match_any_sync(0xffffffffu, word);
+      if (live && lane == (uint32_t)__ffs(peers) - 1u) atomicAdd(&counters[word], (uint32_t)__popc(peers));
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&done[row], 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (tid == 0) done[row] = 0;
+  cta_scan_counts<true>(row, tile_pre, tile_info, ntile, state, k, dev_status);
 }
 
 // A scattered 4-byte read: ask L2 to fetch no more than 64 bytes around it.
@@ -1225,7 +1252,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   // itself and strides over the tiles, so that a single vector that missed is not left to a sliver
   // of the machine; the CTAs of the vectors that hit leave at once, so with many vectors the grid
   // per vector is halved to keep those empty launches short
-  uint64_t stride_ctas = rows >= 8 ? 148ull * 2ull : 148ull * 4ull;
+  uint64_t stride_ctas = rows >= 8 ? 148ull : 148ull * 4ull;
   if (stride_ctas > pl.ntile) stride_ctas = pl.ntile;
   dim3 gm((unsigned)stride_ctas, rows, 1);
   const uint64_t off_val = (uint64_t)(reinterpret_cast<uint8_t*>(io.val) - reinterpret_cast<uint8_t*>(io.idx));
@@ -1249,14 +1276,13 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
                                          k32, pred, io.dev_status);
     launch_pdl(k_topk_lhist<3>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred, io.dev_status);
-    dim3 gc((unsigned)(148ull * 8ull / rows ? 148ull * 8ull / rows : 1), rows, 1);
-    launch_pdl(k_topk_classify, gc, kThreads, st, dense, list_count, cap, state, tile_info, pl.ntile);
-    launch_pdl(k_topk_scan<true>, rows, 1024, st, seg, tile_info, pl.ntile, state, k32, io.dev_status);
+    dim3 gc((unsigned)(148ull / rows ? 148ull / rows : 1), rows, 1);   // one wave of 1024-thread CTAs
+    launch_pdl(k_topk_classify, gc, 1024, st, dense, list_count, cap, state, tile_info, seg, pl.ntile, done, k32, io.dev_status);
     dim3 ge((unsigned)((pl.ntile + kThreads / 32 - 1) / (kThreads / 32)), rows, 1);
     launch_pdl(k_topk_emit_list, ge, kThreads, st, io.v_inout, d, state, list, cap, tile_info, seg, pl.ntile,
                                               reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x,
-                                              io.gamma, io.keep_error);
-    count_launches(11);
+                                              io.gamma, io.keep_error, io.span_off);
+    count_launches(10);
     return cudaGetLastError();
   } else {
 #define DSQ_P1(S) launch_pdl(k_topk_pass1_basic<S>, g1b, kThreads, st, src, io.v_inout, hist, span)
@@ -1274,7 +1300,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     launch_pdl(k_topk_finalize, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg);
     count_launches(7);
   }
-  launch_pdl(k_topk_scan<false>, rows, 1024, st, seg, nullptr, pl.nseg, state, k32, io.dev_status);
+  launch_pdl(k_topk_scan, rows, 1024, st, seg, pl.nseg, state, k32, io.dev_status);
   launch_pdl(k_topk_emit, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg,
                                        reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x, io.gamma);
   count_launches(2);
