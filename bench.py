@@ -538,7 +538,9 @@ def run_sharded(args, wl):
     lib = load_library()
     K, W = args.steps, max(args.warmup, 3)
     swl = wl.scaled(d=wl.d, n=world)
-    ds = DoubleSqueeze(world, swl.d, swl.gamma, swl.worker_q, swl.server_q, swl.seed, device=dev)
+    # every rank keeps the error of its own worker only
+    ds = DoubleSqueeze(world, swl.d, swl.gamma, swl.worker_q, swl.server_q, swl.seed, device=dev,
+                       delta_w_rows=1 if world > 1 else 0)
     sh = ShardedDoubleSqueeze(ds, rank, world)
     tr = DistTransport()
     R = max(2, min(K + W, int(8e9 // (swl.d * 4))))

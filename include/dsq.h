@@ -53,8 +53,6 @@ typedef enum {
 
 /* dev_status is four words.  Word 0 holds flags: */
 #define DS_DEV_TOPK_INCONSISTENT 0x1u /* top-k selection counted a number of entries other than k */
-#define DS_DEV_TAIL_TIMEOUT 0x2u      /* a bounded wait between the thread blocks of the top-k selection kernel
-                                         ran out; the kernel left early and this step's results are not valid */
 /* Words 1 and 2 count top-k selections (one per vector and pass) by the route they took: with the
  * threshold band predicted from the previous steps ("predicted": v is read once), or through the
  * full histogram after a missing or wrong prediction ("full": v is read three times).  Both routes
@@ -161,7 +159,11 @@ typedef struct {
 
 typedef struct {
   uint32_t n;        /* workers, 1 <= n <= 65535 */
-  uint32_t reserved; /* must be 0 */
+  uint32_t delta_w_rows; /* 0 (or n): delta_w holds the errors of all n workers.  R < n: this instance is one rank of
+                        a deployment with one or a few workers per GPU and keeps the errors of R consecutive workers
+                        only (delta_w is float[R*d]; worker i uses row i mod R, and a ds_worker_compress_rows call
+                        must stay inside one block of R workers that starts at a multiple of R); ds_worker_compress
+                        for all n workers is then DS_ERR_UNSUPPORTED.  The payload buffers keep their n rows */
   uint64_t d;        /* model dimension, 1 <= d < 2^32 */
   float gamma;       /* learning rate, finite */
   uint32_t flags;    /* DS_NO_COMPENSATION or 0 */
@@ -173,7 +175,7 @@ typedef struct {
 /*
  * Caller-owned device buffers.  Layouts:
  *   x        float[d]        model; the caller sets x_0
- *   delta_w  float[n*d]      worker errors, row i = worker i; the caller zero-fills (delta = 0)
+ *   delta_w  float[n*d]      worker errors, row i = worker i (float[R*d] with delta_w_rows = R); the caller zero-fills (delta = 0)
  *   delta_s  float[d]        server error; the caller zero-fills
  *   worker_payload           n payloads at a fixed stride, see ds_get_layout()
  *   server_payload           one payload
@@ -275,9 +277,9 @@ int ds_destroy(ds_handle h);
  *   one ds_server_aggregate_compress bit for bit.
  * ds_apply_update_slice: x = x - gamma Q[v] on lo .. hi-1 from that slice of the server payload.
  *
- * Operators that act per chunk or per entry (IDENTITY, SIGN1 with a chunk, QSGD, CLIP) are supported on both
- * passes; the operators that need a quantity of the whole vector (TOPK, SIGN1 with chunk = 0, TERNARY) on
- * either pass, and RSPARSE, are DS_ERR_UNSUPPORTED here.  These calls do not take part in the worker -> server -> apply order check
+ * Operators that act per chunk or per entry (IDENTITY, SIGN1 with a chunk, QSGD, CLIP, RSPARSE) are supported on
+ * both passes; the operators that need a quantity of the whole vector (TOPK, SIGN1 with chunk = 0, TERNARY) on
+ * either pass are DS_ERR_UNSUPPORTED here.  These calls do not take part in the worker -> server -> apply order check
  * of the whole-vector calls: the caller sequences its slices.  Errors as for the whole-vector calls.
  */
 #define DS_SLICE_ALIGN 8192u

@@ -20,7 +20,6 @@ DS_ERR_INVALID_ARG, DS_ERR_ALIGN, DS_ERR_BUFFER_TOO_SMALL = -1, -2, -3
 DS_ERR_STATE, DS_ERR_CUDA, DS_ERR_UNSUPPORTED = -4, -5, -6
 DS_FUSE_APPLY = 1
 DS_DEV_TOPK_INCONSISTENT = 1
-DS_DEV_TAIL_TIMEOUT = 2
 OPS = {"identity": 0, "sign1": 1, "topk": 2, "qsgd": 3, "clip": 4, "rsparse": 5, "ternary": 6}
 DS_NO_COMPENSATION = 1
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
@@ -36,7 +35,7 @@ class ds_qspec(C.Structure):
 
 
 class ds_config(C.Structure):
-    _fields_ = [("n", C.c_uint32), ("reserved", C.c_uint32), ("d", C.c_uint64), ("gamma", C.c_float),
+    _fields_ = [("n", C.c_uint32), ("delta_w_rows", C.c_uint32), ("d", C.c_uint64), ("gamma", C.c_float),
                 ("flags", C.c_uint32), ("worker_q", ds_qspec), ("server_q", ds_qspec), ("seed", C.c_uint64)]
 
 
@@ -97,8 +96,9 @@ def _qspec(q: Q) -> ds_qspec:
     return ds_qspec(OPS[q.op], q.chunk, q.k, levels, norm)
 
 
-def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int, compensate: bool = True) -> ds_config:
-    return ds_config(n, 0, d, gamma, 0 if compensate else DS_NO_COMPENSATION, _qspec(worker_q), _qspec(server_q), seed)
+def make_config(n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int, compensate: bool = True,
+                delta_w_rows: int = 0) -> ds_config:
+    return ds_config(n, delta_w_rows, d, gamma, 0 if compensate else DS_NO_COMPENSATION, _qspec(worker_q), _qspec(server_q), seed)
 
 
 def get_layout(cfg: ds_config, which: int) -> ds_payload_layout:
@@ -162,8 +162,10 @@ class DoubleSqueeze:
 
     def __init__(self, n: int, d: int, gamma: float, worker_q: Q, server_q: Q, seed: int = 0,
                  device: str | torch.device = "cuda", x0: torch.Tensor | None = None, guard: bool = False,
-                 payload_fill: int = 0, compensate: bool = True):
-        """compensate=False: the methods of Section 5.1 that keep no error (DS_NO_COMPENSATION): delta_w
+                 payload_fill: int = 0, compensate: bool = True, delta_w_rows: int = 0):
+        """delta_w_rows = R < n: this instance is one rank of a deployment with R workers per GPU and keeps
+        only their errors (see ds_config.delta_w_rows).
+        compensate=False: the methods of Section 5.1 that keep no error (DS_NO_COMPENSATION): delta_w
         and delta_s are then empty tensors unless the library asks for delta_s as scratch.
         guard=True surrounds every buffer handed to the library with GUARD_BYTES sentinel bytes
         (check_guards() tells whether any was overwritten): a debugging aid for out-of-bounds writes.
@@ -176,7 +178,7 @@ class DoubleSqueeze:
         self.n, self.d, self.gamma, self.seed = n, d, gamma, seed
         self.worker_q, self.server_q = worker_q, server_q
         self.compensate = compensate
-        self.cfg = make_config(n, d, gamma, worker_q, server_q, seed, compensate)
+        self.cfg = make_config(n, d, gamma, worker_q, server_q, seed, compensate, delta_w_rows)
         bufs = ds_buffers()
         rc = self.lib.ds_create(C.byref(self.cfg), C.byref(bufs), None)
         if rc != DS_NEED_BUFFERS:
@@ -198,7 +200,7 @@ class DoubleSqueeze:
         self.x = alloc(d * 4).view(torch.float32)
         if x0 is not None:
             self.x.copy_(x0.to(device=dev, dtype=torch.float32).reshape(-1))
-        self.delta_w = alloc(bufs.delta_w_bytes).view(torch.float32).view(n, bufs.delta_w_bytes // (4 * n))
+        self.delta_w = alloc(bufs.delta_w_bytes).view(torch.float32).view(-1, d) if bufs.delta_w_bytes else alloc(0).view(torch.float32).view(n, 0)
         self.delta_s = alloc(bufs.delta_s_bytes).view(torch.float32)
         self.worker_payload = alloc(bufs.worker_payload_bytes, payload_fill)
         self.server_payload = alloc(bufs.server_payload_bytes, payload_fill)

@@ -48,7 +48,7 @@ bool qspec_ok(const ds_qspec& q, uint64_t d) {
 
 bool config_ok(const ds_config* c) {
   if (!c) return false;
-  if (c->n < 1 || c->n > 65535 || c->reserved != 0 || (c->flags & ~DS_NO_COMPENSATION)) return false;
+  if (c->n < 1 || c->n > 65535 || c->delta_w_rows > c->n || (c->flags & ~DS_NO_COMPENSATION)) return false;
   if (c->d < 1 || c->d >= (1ull << 32)) return false;
   if (!std::isfinite(c->gamma)) return false;
   return qspec_ok(c->worker_q, c->d) && qspec_ok(c->server_q, c->d);
@@ -58,6 +58,9 @@ bool config_ok(const ds_config* c) {
 bool whole_vector(const ds_qspec& q) { return (q.op == DS_Q_SIGN1 && q.chunk == 0) || q.op == DS_Q_TERNARY; }
 
 bool no_compensation(const ds_config& c) { return (c.flags & DS_NO_COMPENSATION) != 0; }
+
+// Rows of delta_w this instance holds: all n, or the R workers of its own block.
+uint32_t delta_rows(const ds_config& c) { return c.delta_w_rows ? c.delta_w_rows : c.n; }
 
 void layout_of(const ds_qspec& q, uint64_t d, ds_payload_layout* L) {
   memset(L, 0, sizeof *L);
@@ -280,11 +283,12 @@ int run_pass(ds_ctx* c, int src_kind, const SrcParams& src, const ds_qspec& q, c
                       x_fused, c->cfg.gamma, rows, st);
       break;
     case DS_Q_RSPARSE: {
-      if (win) return DS_ERR_UNSUPPORTED;
       RsparseParams rp;
       memset(&rp, 0, sizeof rp);
-      rp.out_val = reinterpret_cast<float*>(payload + L.off[0]);
-      rp.out_off = reinterpret_cast<uint32_t*>(payload + L.off[1]);
+      rp.out_val = reinterpret_cast<float*>(payload + L.off[0]) + lo / q.levels;     // slot j / S
+      rp.out_off = reinterpret_cast<uint32_t*>(payload + L.off[1]) + lo / q.chunk;
+      rp.chunk0 = (uint32_t)(lo / q.chunk);
+      rp.row0 = win ? win->row0 : 0;
       rp.val_stride = L.stride / 4;
       rp.off_stride = L.stride / 4;
       rp.log2_chunk = log2u(q.chunk);
@@ -328,7 +332,7 @@ int ds_create(const ds_config* cfg, ds_buffers* bufs, ds_handle* out) {
   // without compensation no error is carried: delta_w is not needed at all, delta_s only as the place
   // where a top-k server pass lays out its vector
   const bool nocomp = no_compensation(*cfg);
-  const uint64_t need_x = cfg->d * 4, need_dw = nocomp ? 0 : (uint64_t)cfg->n * cfg->d * 4;
+  const uint64_t need_x = cfg->d * 4, need_dw = nocomp ? 0 : (uint64_t)delta_rows(*cfg) * cfg->d * 4;
   const uint64_t need_ds = (nocomp && cfg->server_q.op != DS_Q_TOPK) ? 0 : cfg->d * 4;
   const uint64_t need_wp = (uint64_t)cfg->n * tmp.wl.stride, need_sp = tmp.sl.stride;
   const uint64_t need_ws = plan_workspace(&tmp);
@@ -365,6 +369,7 @@ int ds_worker_compress(ds_handle h, const float* g, uint32_t step, void* cuda_st
   if (!h || !g) return DS_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(g) & 3u) != 0) return DS_ERR_ALIGN;
   if (h->phase != 0) return DS_ERR_STATE;
+  if (delta_rows(h->cfg) != h->cfg.n) return DS_ERR_UNSUPPORTED;   // this instance holds the errors of one block of workers only
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const SrcParams src = worker_src(h, g);
   const bool nocomp = no_compensation(h->cfg);
@@ -430,7 +435,7 @@ bool slice_ok(const ds_ctx* h, uint64_t lo, uint64_t hi) {
   return lo < hi && hi <= d && lo % DS_SLICE_ALIGN == 0 && (hi == d || hi % DS_SLICE_ALIGN == 0);
 }
 
-bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK && q.op != DS_Q_RSPARSE && !whole_vector(q); }
+bool sliceable(const ds_qspec& q) { return q.op != DS_Q_TOPK && !whole_vector(q); }
 
 }  // namespace
 
@@ -441,12 +446,15 @@ int ds_worker_compress_rows(ds_handle h, const float* g, uint32_t row0, uint32_t
   const uint64_t d = h->cfg.d;
   SrcParams src = worker_src(h, g);
   const bool nocomp = no_compensation(h->cfg);
-  float* delta_rows = nocomp ? nullptr : h->buf.delta_w + (uint64_t)row0 * d;
-  src.delta = delta_rows;
+  // with the errors of one block of R workers only, worker i lives in row i mod R and a call stays inside a block
+  const uint32_t R = delta_rows(h->cfg);
+  if ((uint64_t)(row0 % R) + nrows > R) return DS_ERR_INVALID_ARG;
+  float* delta_blk = nocomp ? nullptr : h->buf.delta_w + (uint64_t)(row0 % R) * d;
+  src.delta = delta_blk;
   src.vec = (d % 4 == 0) && aligned16(g);
   const PassWindow win{d, 0, row0};
   return run_pass(h, nocomp ? SRC_WORKER_PLAIN : SRC_WORKER, src, h->cfg.worker_q, h->wl,
-                  static_cast<uint8_t*>(h->buf.worker_payload) + (uint64_t)row0 * h->wl.stride, delta_rows, nrows, false, nullptr,
+                  static_cast<uint8_t*>(h->buf.worker_payload) + (uint64_t)row0 * h->wl.stride, delta_blk, nrows, false, nullptr,
                   step, static_cast<cudaStream_t>(cuda_stream), &win);
 }
 
@@ -466,6 +474,7 @@ int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flag
     case DS_Q_SIGN1: src.wp_off[0] += lo / 8; src.wp_off[1] += lo / wq.chunk * 4; break;
     case DS_Q_QSGD: src.wp_off[0] += lo; src.wp_off[1] += lo / 8; src.wp_off[2] += lo / wq.chunk * 4; break;
     case DS_Q_CLIP: src.wp_off[0] += lo * ((32 - wq.levels) / 8); break;
+    case DS_Q_RSPARSE: src.wp_off[0] += lo / wq.levels * 4; src.wp_off[1] += lo / wq.chunk * 4; break;
     default: return DS_ERR_UNSUPPORTED;
   }
   const PassWindow win{hi - lo, lo, 0};
@@ -483,14 +492,16 @@ int ds_apply_update_slice(ds_handle h, uint64_t lo, uint64_t hi, void* cuda_stre
   pv.op = q.op;
   pv.base = static_cast<const uint8_t*>(h->buf.server_payload);
   for (int i = 0; i < 3; ++i) pv.off[i] = h->sl.off[i];
-  pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD) ? log2u(q.chunk) : 0;
+  pv.log2_chunk = (q.op == DS_Q_SIGN1 || q.op == DS_Q_QSGD || q.op == DS_Q_RSPARSE) ? log2u(q.chunk) : 0;
   pv.levels_f = (float)q.levels;
   pv.clip_bits = q.op == DS_Q_CLIP ? q.levels : 0;
+  pv.log2_keep = q.op == DS_Q_RSPARSE ? log2u(q.levels) : 0;
   switch (q.op) {
     case DS_Q_IDENTITY: pv.off[0] += lo * 4; break;
     case DS_Q_SIGN1: pv.off[0] += lo / 8; pv.off[1] += lo / q.chunk * 4; break;
     case DS_Q_QSGD: pv.off[0] += lo; pv.off[1] += lo / 8; pv.off[2] += lo / q.chunk * 4; break;
     case DS_Q_CLIP: pv.off[0] += lo * ((32 - q.levels) / 8); break;
+    case DS_Q_RSPARSE: pv.off[0] += lo / q.levels * 4; pv.off[1] += lo / q.chunk * 4; break;
     default: return DS_ERR_UNSUPPORTED;
   }
   const cudaError_t e = launch_apply(pv, h->buf.x + lo, hi - lo, h->cfg.gamma, static_cast<cudaStream_t>(cuda_stream));

@@ -135,7 +135,8 @@ __global__ void __launch_bounds__(kThreads) k_rsparse_draw(const RsparseParams r
   const uint32_t row = blockIdx.y;
   const uint64_t c = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
   if (c < nc) {
-    const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c, rp.server_pass ? 0xFFFFFFFFu : row, rp.step), rp.keys);
+    const uint4 rnd = philox4x32_10(make_uint4(0xFFFFFFFFu, (uint32_t)c + rp.chunk0, rp.server_pass ? 0xFFFFFFFFu : row + rp.row0, rp.step),
+                                    rp.keys);
     rp.out_off[(uint64_t)row * rp.off_stride + c] = rnd.x & ((1u << rp.log2_keep) - 1u);
   }
   if (blockIdx.x == gridDim.x - 1) {

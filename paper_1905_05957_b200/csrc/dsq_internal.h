@@ -169,6 +169,7 @@ struct RsparseParams {
   uint32_t log2_chunk, log2_keep, scaled;
   PhiloxKeys keys;
   uint32_t step, server_pass;
+  uint32_t chunk0, row0;     // a pass over a slice of d / some of the workers: index of its first chunk / worker
 };
 cudaError_t launch_rsparse(int src_kind, const SrcParams& src, const RsparseParams& rp, float* delta_out,
                            uint64_t delta_row_stride, float* x, float gamma, uint32_t rows, cudaStream_t st);

@@ -60,6 +60,11 @@ def payload_slice_ranges(q: Q, layout_off, lo: int, hi: int) -> list[tuple[int, 
         return [(layout_off[0] + b * lo, b * (hi - lo))]
     if q.op == "identity":
         return [(layout_off[0] + 4 * lo, 4 * (hi - lo))]
+    if q.op == "rsparse":
+        S, per = q.keep_one_in, q.chunk // q.keep_one_in
+        c_lo, c_hi = lo // q.chunk, -(-hi // q.chunk)          # whole chunks: a short last chunk still has `per` slots
+        return [(layout_off[0] + 4 * (lo // S), 4 * (c_hi * per - lo // S)),
+                (layout_off[1] + 4 * c_lo, 4 * (c_hi - c_lo))]
     raise ValueError(f"operator {q.op!r} has no slices along d")
 
 
@@ -128,10 +133,20 @@ class DistTransport:
         import torch.distributed as dist
         self.dist, self.group = dist, group
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
+        self._staging: dict = {}
+        self.bytes_sent = 0          # payload bytes this rank has put on the wire so far
+
+    def _recv_buffers(self, recv_sizes: list[int], device) -> list[torch.Tensor]:
+        """Receive staging, allocated once per shape of exchange and reused every iteration."""
+        key = (tuple(recv_sizes), str(device))
+        if key not in self._staging:
+            self._staging[key] = [torch.empty(n, dtype=torch.uint8, device=device) for n in recv_sizes]
+        return list(self._staging[key])
 
     def _exchange(self, send: list[torch.Tensor], recv_sizes: list[int]) -> list[torch.Tensor]:
         dist = self.dist
-        recv = [torch.empty(n, dtype=torch.uint8, device=send[0].device) for n in recv_sizes]
+        recv = self._recv_buffers(recv_sizes, send[0].device)
+        self.bytes_sent += sum(int(t.numel()) for q, t in enumerate(send) if q != self.rank)
         ops = []
         for q in range(self.world):
             if q == self.rank:
@@ -155,7 +170,8 @@ class DistTransport:
 
 class ShardedDoubleSqueeze:
     """One rank of the one-worker-per-GPU deployment (see the module text).  `ds` is this rank's
-    DoubleSqueeze instance, created with n = world; only row `rank` of its delta_w is used."""
+    DoubleSqueeze instance, created with n = world and, to hold the error of its own worker only,
+    delta_w_rows = 1 (an instance with all n rows works too and uses row `rank`)."""
 
     def __init__(self, ds, rank: int, world: int):
         if ds.n != world:

@@ -94,6 +94,13 @@ def test_layouts_of_the_whole_vector_operators_and_sizes_without_compensation(li
     # unknown flag bits are refused
     cfg.flags = 2
     assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_ERR_INVALID_ARG
+    # an instance that keeps the errors of one block of workers: delta_w shrinks, the payload buffers do not
+    bufs = b.ds_buffers()
+    cfg = b.make_config(8, d, 0.1, Q("sign1", chunk=4096), Q("sign1", chunk=4096), 1, delta_w_rows=2)
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_NEED_BUFFERS
+    assert bufs.delta_w_bytes == 2 * 4 * d and bufs.worker_payload_bytes == 8 * b.get_layout(cfg, 0).stride
+    cfg = b.make_config(8, d, 0.1, Q("sign1", chunk=4096), Q("sign1", chunk=4096), 1, delta_w_rows=9)
+    assert lib.ds_create(C.byref(cfg), C.byref(bufs), None) == b.DS_ERR_INVALID_ARG
 
 
 def test_query_mode_reports_sizes(lib):

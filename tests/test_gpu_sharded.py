@@ -15,7 +15,9 @@ pytestmark = pytest.mark.gpu
 SIGN = Q("sign1", chunk=4096)
 PAIRS = [(SIGN, SIGN), (Q("qsgd", chunk=2048, levels=255), Q("qsgd", chunk=2048, levels=255)),
          (Q("sign1", chunk=1024, norm=2), Q("clip", bits=16)), (Q("clip", bits=24), Q("qsgd", chunk=512, levels=7)),
-         (Q("identity"), SIGN), (Q("qsgd", chunk=8192, levels=31), Q("identity"))]
+         (Q("identity"), SIGN), (Q("qsgd", chunk=8192, levels=31), Q("identity")),
+         (Q("rsparse", chunk=4096, keep_one_in=32), Q("rsparse", chunk=4096, keep_one_in=32)),
+         (Q("rsparse", chunk=256, keep_one_in=4, scaled=1), SIGN), (Q("clip", bits=16), Q("rsparse", chunk=1024, keep_one_in=8))]
 
 
 def _bits(t):
@@ -30,7 +32,9 @@ def test_sharded_step_equals_whole_vector_step(wq, sq, world, d):
     gs = [torch.randn(world, d, generator=gen).cuda() for _ in range(T)]
     whole = DoubleSqueeze(world, d, gamma, wq, sq, seed)
     st = oracle.State.zeros(world, d)
-    ranks = [ShardedDoubleSqueeze(DoubleSqueeze(world, d, gamma, wq, sq, seed), r, world) for r in range(world)]
+    # every rank keeps the error of its own worker only (delta_w_rows = 1); rank 0 keeps all rows, which must work too
+    ranks = [ShardedDoubleSqueeze(DoubleSqueeze(world, d, gamma, wq, sq, seed, delta_w_rows=1 if r else 0), r, world)
+             for r in range(world)]
     bounds = slice_bounds(d, world)
     assert bounds[0][0] == 0 and bounds[-1][1] == d and all(a[1] == b[0] for a, b in zip(bounds, bounds[1:]))
     for t, g in enumerate(gs):
@@ -42,7 +46,9 @@ def test_sharded_step_equals_whole_vector_step(wq, sq, world, d):
         for r in ranks:
             lo, hi = bounds[r.rank]
             assert torch.equal(_bits(r.ds.x), _bits(whole.x)), f"x on rank {r.rank}, step {t}"
-            assert torch.equal(_bits(r.ds.delta_w[r.rank]), _bits(whole.delta_w[r.rank]))
+            own = r.ds.delta_w[r.rank] if r.ds.delta_w.shape[0] == world else r.ds.delta_w[0]
+            assert r.rank == 0 or r.ds.delta_w.shape[0] == 1      # one row of errors, not n
+            assert torch.equal(_bits(own), _bits(whole.delta_w[r.rank]))
             assert torch.equal(_bits(r.ds.delta_s[lo:hi]), _bits(whole.delta_s[lo:hi]))
             for name, view in r.ds.server_views().items():
                 assert torch.equal(_bits(view), _bits(whole.server_views()[name])), f"server payload {name} on rank {r.rank}"
@@ -64,6 +70,13 @@ def test_slices_reject_what_they_cannot_do():
         ds.server_aggregate_compress_slice(0, 0, 8000)            # end neither on the grid nor d
     with pytest.raises(Exception, match="-1"):
         ds.worker_compress_rows(g, 1, 0)                          # rows 1..2 of 2
+    one = DoubleSqueeze(4, 40_000, 0.1, SIGN, SIGN, delta_w_rows=2)
+    g4 = torch.randn(4, 40_000, device="cuda")
+    with pytest.raises(Exception, match="-6"):
+        one.worker_compress(g4, 0)                                # the errors of one block of workers only
+    with pytest.raises(Exception, match="-1"):
+        one.worker_compress_rows(g4[1:3].contiguous(), 1, 0)      # rows 1..2 straddle two blocks of 2
+    one.worker_compress_rows(g4[2:4].contiguous(), 2, 0)
     tk = DoubleSqueeze(2, 40_000, 0.1, Q("topk", k=10), SIGN)
     with pytest.raises(Exception, match="-6"):
         tk.worker_compress_rows(g[:1].contiguous(), 0, 0)

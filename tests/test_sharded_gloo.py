@@ -100,3 +100,102 @@ def test_slices_tile_the_vector_and_the_payload():
                     continue
                 sub = [(s, n) for s, n in covered if lay.off[j] <= s < lay.off[j] + max(1, lay.count[j] * 4)]
                 assert all(a[0] + a[1] <= b_[0] for a, b_ in zip(sub, sub[1:]))
+
+
+# ------------------------------------------------------------------ the whole iteration, phase by phase
+
+class _StandInInstance:
+    """What ShardedDoubleSqueeze needs of a DoubleSqueeze instance, on the CPU: the payload buffers and
+    layouts are the library's, the three passes write recognisable bytes and keep a log instead of
+    launching kernels.  The worker pass fills the rank's own payload row with a byte that names
+    (rank, step); the server pass fills this rank's slice of the server payload with the sum (mod 256)
+    of the first byte of that slice in every worker's row, so it can only come out right if hop 1
+    delivered every worker's slice before it ran; apply records which slices it was asked for."""
+
+    def __init__(self, rank, world):
+        self.n, self.d, self.worker_q, self.server_q = world, D, WQ, SQ
+        cfg = b.make_config(world, D, 0.1, WQ, SQ, 1)
+        self.worker_layout, self.server_layout = b.get_layout(cfg, 0), b.get_layout(cfg, 1)
+        self.worker_payload = torch.zeros(world * int(self.worker_layout.stride), dtype=torch.uint8)
+        self.server_payload = torch.zeros(int(self.server_layout.stride), dtype=torch.uint8)
+        self.rank, self.log = rank, []
+
+    def worker_compress_rows(self, g_rows, row0, t):
+        self.log.append(("worker", row0, t))
+        stride = int(self.worker_layout.stride)
+        self.worker_payload[row0 * stride:(row0 + 1) * stride] = (17 * row0 + 3 * t + 1) % 256
+
+    def server_aggregate_compress_slice(self, t, lo, hi, fuse_apply=False):
+        self.log.append(("server", lo, hi, t, fuse_apply))
+        stride = int(self.worker_layout.stride)
+        wr = payload_slice_ranges(WQ, tuple(self.worker_layout.off), lo, hi)
+        total = sum(int(self.worker_payload[i * stride + wr[0][0]]) for i in range(self.n)) % 256
+        for s_, n_ in payload_slice_ranges(SQ, tuple(self.server_layout.off), lo, hi):
+            self.server_payload[s_: s_ + n_] = total
+
+    def apply_update_slice(self, lo, hi):
+        self.log.append(("apply", lo, hi))
+
+
+def _step_main(rank: int, world: int, port: int, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_1905_05957_b200.sharded import ShardedDoubleSqueeze
+    inst = _StandInInstance(rank, world)
+    sh = ShardedDoubleSqueeze(inst, rank, world)
+    tr = DistTransport()
+    sent = []
+    for t in range(2):
+        before = tr.bytes_sent
+        sh.step(torch.zeros(D), t, tr)
+        sent.append(tr.bytes_sent - before)
+    staging = sum(len(v) for v in tr._staging.values())
+    dist.barrier()
+    out.put((rank, inst.log, inst.server_payload.numpy().tobytes(), sent, staging))
+    dist.destroy_process_group()
+
+
+def test_whole_iteration_over_gloo_runs_its_phases_in_order_and_moves_the_planned_bytes():
+    world, port = 3, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_step_main, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = {}
+    for _ in range(world):
+        r, log, sp, sent, staging = out.get(timeout=180)
+        got[r] = (log, torch.frombuffer(bytearray(sp), dtype=torch.uint8), sent, staging)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    bounds = slice_bounds(D, world)
+    cfg = b.make_config(world, D, 0.1, WQ, SQ, 1)
+    wl, sl = b.get_layout(cfg, 0), b.get_layout(cfg, 1)
+    # what the last step's server payload must be on EVERY rank: slice q filled by rank q from all workers' bytes
+    t = 1
+    want = torch.zeros(int(sl.stride), dtype=torch.uint8)
+    for q, (lo, hi) in enumerate(bounds):
+        total = sum((17 * i + 3 * t + 1) % 256 for i in range(world)) % 256
+        for s_, n_ in payload_slice_ranges(SQ, tuple(sl.off), lo, hi):
+            want[s_: s_ + n_] = total
+    for r in range(world):
+        log, sp, sent, staging = got[r]
+        lo, hi = bounds[r]
+        per_step = [("worker", r, None), ("server", lo, hi, None, True)] + \
+                   [("apply", *bounds[q]) for q in range(world) if q != r and bounds[q][1] > bounds[q][0]]
+        assert len(log) == 2 * len(per_step)
+        for t_ in range(2):
+            chunk = log[t_ * len(per_step):(t_ + 1) * len(per_step)]
+            assert chunk[0] == ("worker", r, t_) and chunk[1] == ("server", lo, hi, t_, True)
+            assert chunk[2:] == per_step[2:]
+        assert torch.equal(sp, want), f"server payload on rank {r}"
+        # bytes on the wire per step: slice q of the own payload to every other rank, the own server slice to every other rank
+        hop1 = sum(sum(n_ for _, n_ in payload_slice_ranges(WQ, tuple(wl.off), *bounds[q])) for q in range(world) if q != r)
+        hop2 = (world - 1) * sum(n_ for _, n_ in payload_slice_ranges(SQ, tuple(sl.off), lo, hi))
+        assert sent == [hop1 + hop2, hop1 + hop2]
+        assert staging == 2 * world        # one set of receive buffers per hop, reused by the second step
+    # the compressed hops move a small fraction of what the dense vector would: 9/32 and 1/32 of 4 bytes per entry here
+    dense = 4 * D
+    assert got[0][2][0] < 0.25 * dense
