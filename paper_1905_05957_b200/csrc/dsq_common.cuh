@@ -280,37 +280,76 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
         }
       }
     } else if constexpr (SRC == SRC_SRV_RSPARSE) {
-      // entry j of worker i survives iff (offset of j in its chunk) mod S equals the chunk's draw;
-      // its value sits in slot j / S.  Four workers at a time: their draws are fetched together,
-      // then their survivors, then they are added in worker order.
+      // entry j of worker i survives iff (offset of j in its chunk) mod S equals the chunk's draw o_i;
+      // its value sits in slot j / S.  With S >= 4 the four entries of a float4 lie in one group of S,
+      // so a worker has at most ONE survivor among them: it is there iff o_i agrees with the entries'
+      // offset in everything but the low two bits, it is component o_i % 4, and its slot is the
+      // group's.  Eight workers at a time: their draws are fetched together, then their survivors,
+      // then they are added in worker order.
       const uint32_t smask = (1u << p.w_log2_keep) - 1u;
-      for (uint32_t i0 = 0; i0 < p.n; i0 += 4) {
-        uint32_t o[V][4];
-        float4 c[V][4];
+      if (p.w_log2_keep >= 2) {
+        for (uint32_t i0 = 0; i0 < p.n; i0 += 8) {
+          uint32_t o[V][8];
+          float c[V][8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const uint32_t* off = reinterpret_cast<const uint32_t*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[1]);
+          for (int u = 0; u < 8; ++u) {
+            const uint32_t* off = reinterpret_cast<const uint32_t*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[1]);
 #pragma unroll
-          for (int j = 0; j < V; ++j) o[j][u] = (i0 + u < p.n && cnt[j]) ? __ldg(off + (e[j] >> p.w_log2_chunk)) : 0xFFFFFFFFu;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const float* val = reinterpret_cast<const float*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[0]);
-#pragma unroll
-          for (int j = 0; j < V; ++j) {
-            c[j][u] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              if ((uint32_t)k < cnt[j] && (((uint32_t)e[j] + k) & smask) == o[j][u])   // never true for the filler 0xFFFFFFFF
-                comp(c[j][u], k) = __ldg(val + ((e[j] + k) >> p.w_log2_keep));
+            for (int j = 0; j < V; ++j) o[j][u] = (i0 + u < p.n && cnt[j]) ? __ldg(off + (e[j] >> p.w_log2_chunk)) : 0xFFFFFFFFu;
           }
-        }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (i0 + u < p.n) {
+          for (int u = 0; u < 8; ++u) {
+            const float* val = reinterpret_cast<const float*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[0]);
 #pragma unroll
-            for (int j = 0; j < V; ++j) acc[j] = add4_rn(acc[j], c[j][u]);
+            for (int j = 0; j < V; ++j) {
+              // the filler 0xFFFFFFFF is no draw (draws are at most S - 1); a survivor past the end of a ragged
+              // last float4 reads its slot, which holds +0, and is dropped by the masking of v below anyway
+              const bool mine = o[j][u] <= smask && ((((uint32_t)e[j] ^ o[j][u]) & smask & ~3u) == 0u);
+              c[j][u] = mine ? __ldg(val + (e[j] >> p.w_log2_keep)) : 0.f;
+            }
           }
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            if (i0 + u < p.n) {
+#pragma unroll
+              for (int j = 0; j < V; ++j) {
+                const uint32_t k = o[j][u] & 3u;
+                // adding +0 to the other three components changes nothing: acc is never -0
+                acc[j] = add4_rn(acc[j], make_float4(k == 0u ? c[j][u] : 0.f, k == 1u ? c[j][u] : 0.f, k == 2u ? c[j][u] : 0.f,
+                                                     k == 3u ? c[j][u] : 0.f));
+              }
+            }
+        }
+      } else {
+        // S = 2: two survivors per float4; four workers at a time, entry by entry
+        for (uint32_t i0 = 0; i0 < p.n; i0 += 4) {
+          uint32_t o[V][4];
+          float4 c[V][4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t* off = reinterpret_cast<const uint32_t*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[1]);
+#pragma unroll
+            for (int j = 0; j < V; ++j) o[j][u] = (i0 + u < p.n && cnt[j]) ? __ldg(off + (e[j] >> p.w_log2_chunk)) : 0xFFFFFFFFu;
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float* val = reinterpret_cast<const float*>(p.wp + (uint64_t)(i0 + u) * p.wp_stride + p.wp_off[0]);
+#pragma unroll
+            for (int j = 0; j < V; ++j) {
+              c[j][u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                if ((uint32_t)k < cnt[j] && (((uint32_t)e[j] + k) & smask) == o[j][u])   // never true for the filler 0xFFFFFFFF
+                  comp(c[j][u], k) = __ldg(val + ((e[j] + k) >> p.w_log2_keep));
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (i0 + u < p.n) {
+#pragma unroll
+              for (int j = 0; j < V; ++j) acc[j] = add4_rn(acc[j], c[j][u]);
+            }
+        }
       }
     } else {  // SRC_SRV_TOPK: the sparse payloads were summed into p.acc (cleared before every use)
 #pragma unroll

@@ -158,39 +158,51 @@ k_rsparse(const SrcParams src, const RsparseParams rp, float* delta_out, uint64_
   const float factor = rp.scaled ? (float)(1u << rp.log2_keep) : 1.0f;
   float* val = rp.out_val + (uint64_t)row * rp.val_stride;
   const uint32_t* off = rp.out_off + (uint64_t)row * rp.off_stride;
+  // one float4 per thread and trip (two on the server passes measured slower: the decode of n payloads
+  // already fills the 64 registers that four resident CTAs allow)
+  constexpr int V = 1;
   // the loop bound is the same for all threads of the CTA: the source is read warp-cooperatively
-  for (uint64_t q0 = (uint64_t)blockIdx.x * kThreads; q0 < nq; q0 += (uint64_t)gridDim.x * kThreads) {
-    const uint64_t ee[1] = {(q0 + threadIdx.x) * 4};
-    const uint64_t e = ee[0];
-    const uint32_t cc[1] = {e < src.d ? (uint32_t)min((uint64_t)4, src.d - e) : 0u};
-    const uint32_t cnt = cc[0];
-    float4 vv[1];
-    src_load_tile<SRC, 1>(src, row, ee, cc, vv);
-    const float4 v = vv[0];
-    if (!cnt) continue;
-    const uint32_t o = __ldg(off + (e >> rp.log2_chunk));  // the chunk's draw, made by k_rsparse_draw
-    float4 C = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (uint64_t q0 = (uint64_t)blockIdx.x * kThreads * V; q0 < nq; q0 += (uint64_t)gridDim.x * kThreads * V) {
+    uint64_t ee[V];
+    uint32_t cc[V], oo[V];
+    float4 vv[V], xx[V];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if ((uint32_t)k < cnt && (((uint32_t)e + k) & smask) == o) {
-        const float kept = __fmul_rn(factor, compc(v, k));
-        comp(C, k) = kept;
-        val[(e + k) >> rp.log2_keep] = kept;
+    for (int j = 0; j < V; ++j) {
+      ee[j] = (q0 + (uint64_t)j * kThreads + threadIdx.x) * 4;
+      cc[j] = ee[j] < src.d ? (uint32_t)min((uint64_t)4, src.d - ee[j]) : 0u;
+      oo[j] = cc[j] ? __ldg(off + (ee[j] >> rp.log2_chunk)) : 0u;  // the chunk's draw, made by k_rsparse_draw
+      xx[j] = (x && cc[j]) ? load_row4(x, ee[j], cc[j], 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    src_load_tile<SRC, V>(src, row, ee, cc, vv);
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      const uint64_t e = ee[j];
+      const uint32_t cnt = cc[j], o = oo[j];
+      const float4 v = vv[j];
+      if (!cnt) continue;
+      float4 C = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if ((uint32_t)k < cnt && (((uint32_t)e + k) & smask) == o) {
+          const float kept = __fmul_rn(factor, compc(v, k));
+          comp(C, k) = kept;
+          val[(e + k) >> rp.log2_keep] = kept;
+        }
       }
-    }
-    // the group of S positions that holds the last entry: if its survivor lies past the end, its slot
-    // is sent as +0 (it may still hold a survivor of an earlier step); the slots of the groups
-    // wholly past the end are cleared by k_rsparse_draw
-    if (e + cnt == src.d) {
-      const uint64_t group = (src.d - 1) >> rp.log2_keep;
-      if ((group << rp.log2_keep) + o >= src.d) val[group] = 0.f;
-    }
-    if (keeps_error<SRC>(delta_out)) store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
-    if (x) {
-      float4 xv = load_row4(x, e, cnt, 1);
-      xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
-      xv.z = __fsub_rn(xv.z, __fmul_rn(gamma, C.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(gamma, C.w));
-      store_row4(x, e, cnt, 1, xv);
+      // the group of S positions that holds the last entry: if its survivor lies past the end, its slot
+      // is sent as +0 (it may still hold a survivor of an earlier step); the slots of the groups
+      // wholly past the end are cleared by k_rsparse_draw
+      if (e + cnt == src.d) {
+        const uint64_t group = (src.d - 1) >> rp.log2_keep;
+        if ((group << rp.log2_keep) + o >= src.d) val[group] = 0.f;
+      }
+      if (keeps_error<SRC>(delta_out)) store_row4(delta_out + (uint64_t)row * delta_row_stride, e, cnt, src.vec, sub4_rn(v, C));  // Eq. 3 / Eq. 4
+      if (x) {
+        float4 xv = xx[j];
+        xv.x = __fsub_rn(xv.x, __fmul_rn(gamma, C.x)); xv.y = __fsub_rn(xv.y, __fmul_rn(gamma, C.y));
+        xv.z = __fsub_rn(xv.z, __fmul_rn(gamma, C.z)); xv.w = __fsub_rn(xv.w, __fmul_rn(gamma, C.w));
+        store_row4(x, e, cnt, 1, xv);
+      }
     }
   }
 }
