@@ -279,7 +279,7 @@ int ds_destroy(ds_handle h);
  *
  * Operators that act per chunk or per entry (IDENTITY, SIGN1 with a chunk, QSGD, CLIP, RSPARSE) are supported on
  * both passes; the operators that need a quantity of the whole vector (TOPK, SIGN1 with chunk = 0, TERNARY) on
- * either pass are DS_ERR_UNSUPPORTED here.  These calls do not take part in the worker -> server -> apply order check
+ * either pass are DS_ERR_UNSUPPORTED here (a TOPK server pass over slices has calls of its own, below).  These calls do not take part in the worker -> server -> apply order check
  * of the whole-vector calls: the caller sequences its slices.  Errors as for the whole-vector calls.
  */
 #define DS_SLICE_ALIGN 8192u
@@ -287,6 +287,39 @@ int ds_worker_compress_rows(ds_handle h, const float* g, uint32_t row0, uint32_t
 int ds_server_aggregate_compress_slice(ds_handle h, uint32_t step, uint32_t flags, uint64_t lo, uint64_t hi,
                                        void* cuda_stream);
 int ds_apply_update_slice(ds_handle h, uint64_t lo, uint64_t hi, void* cuda_stream);
+
+/*
+ * Top-k on the server pass (Section 3.2, "Top-k sparsification": the k largest entries of the WHOLE vector) when the
+ * server's vector is spread over several GPUs, slice lo .. hi-1 on this one.  The threshold is a property of the whole
+ * vector, so the selection is cut into stages at the points where a histogram over all slices is needed; between the
+ * stages the caller adds the slices' histograms up across the GPUs (an all-reduce of 4096 words) and hands the sum to
+ * every slice.  Worker payloads must be of an operator that is laid out along d (everything but TOPK and the
+ * whole-vector operators).  The result equals ds_server_aggregate_compress on the whole vector bit for bit.
+ *
+ *  1. ds_server_topk_slice_begin   v = delta_s + (1/n) sum_i Q[v_i] on the slice (Eq. 4), written over that slice of
+ *                                  delta_s; hist[b] = how many of the slice's entries have (bits(v) & 0x7fffffff) >> 19 == b.
+ *  2. ds_server_topk_slice_digit   level 1, 2, 3: hist_sum = the sum over all slices of the previous stage's histogram
+ *                                  (the call consumes and clears it).  Picks this digit of the threshold (12, 12 and 7
+ *                                  key bits) and writes the next stage's histogram of this slice into hist_next.  After
+ *                                  level 3, hist_next[0..3] = (entries of this slice above the threshold tau, entries
+ *                                  equal to it, the number r of entries equal to tau that the whole vector keeps, tau).
+ *  3. ds_server_topk_slice_emit    ties go to lower indices first, so the caller gives slice q the quota
+ *                                  ties_to_keep = clamp(r - ties in the slices before q, 0, ties in q); the slice then
+ *                                  keeps count = above + ties_to_keep entries.  Writes them (GLOBAL indices ascending,
+ *                                  values) into slots first_slot .. first_slot+count-1 of the server payload's idx / val
+ *                                  arrays (first_slot = the counts of the slices before q, so the gathered payload is
+ *                                  the whole vector's), zeroes them in delta_s, and with DS_FUSE_APPLY updates x there.
+ *  4. ds_apply_update_sparse_range x = x - gamma Q[v] for the entries in slots first_slot .. +count-1 of the server
+ *                                  payload (the parts gathered from the other slices).
+ * hist, hist_sum, hist_next: device uint32[4096], 16-byte aligned, the caller's.  The stages keep their state in the
+ * workspace; one slice at a time per handle.  Errors as for the slice calls above.
+ */
+int ds_server_topk_slice_begin(ds_handle h, uint32_t step, uint64_t lo, uint64_t hi, uint32_t* hist, void* cuda_stream);
+int ds_server_topk_slice_digit(ds_handle h, int level, uint64_t lo, uint64_t hi, uint32_t* hist_sum, uint32_t* hist_next,
+                               void* cuda_stream);
+int ds_server_topk_slice_emit(ds_handle h, uint64_t lo, uint64_t hi, uint32_t ties_to_keep, uint32_t count, uint64_t first_slot,
+                              uint32_t flags, void* cuda_stream);
+int ds_apply_update_sparse_range(ds_handle h, uint64_t first_slot, uint64_t count, void* cuda_stream);
 
 /*
  * Convenience for callers that hold data in HOST memory: copies g_host (float[n*d], ideally

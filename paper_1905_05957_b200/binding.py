@@ -25,7 +25,8 @@ DS_NO_COMPENSATION = 1
 EXPORTS = ("ds_get_layout", "ds_create", "ds_worker_compress", "ds_server_aggregate_compress",
            "ds_apply_update", "ds_destroy", "ds_step_host", "ds_last_error", "ds_version",
            "ds_kernel_launches", "ds_topk_worker_static", "ds_worker_compress_rows",
-           "ds_server_aggregate_compress_slice", "ds_apply_update_slice")
+           "ds_server_aggregate_compress_slice", "ds_apply_update_slice", "ds_server_topk_slice_begin",
+           "ds_server_topk_slice_digit", "ds_server_topk_slice_emit", "ds_apply_update_sparse_range")
 DS_SLICE_ALIGN = 8192
 
 
@@ -82,6 +83,10 @@ def load_library() -> C.CDLL:
     L.ds_worker_compress_rows.argtypes = [vp, vp, u32, u32, u32, vp]
     L.ds_server_aggregate_compress_slice.argtypes = [vp, u32, u32, C.c_uint64, C.c_uint64, vp]
     L.ds_apply_update_slice.argtypes = [vp, C.c_uint64, C.c_uint64, vp]
+    L.ds_server_topk_slice_begin.argtypes = [vp, u32, C.c_uint64, C.c_uint64, vp, vp]
+    L.ds_server_topk_slice_digit.argtypes = [vp, C.c_int, C.c_uint64, C.c_uint64, vp, vp, vp]
+    L.ds_server_topk_slice_emit.argtypes = [vp, C.c_uint64, C.c_uint64, u32, u32, C.c_uint64, u32, vp]
+    L.ds_apply_update_sparse_range.argtypes = [vp, C.c_uint64, C.c_uint64, vp]
     for name in EXPORTS:
         getattr(L, name).restype = C.c_int
     L.ds_last_error.restype = C.c_char_p
@@ -266,6 +271,25 @@ class DoubleSqueeze:
 
     def apply_update_slice(self, lo: int, hi: int, stream=None):
         self._check(self.lib.ds_apply_update_slice(self.handle, lo, hi, self._stream(stream)), "ds_apply_update_slice")
+
+    # -- global top-k on the server pass over a slice (the stages between which histograms are summed across GPUs) ---
+    def server_topk_slice_begin(self, step: int, lo: int, hi: int, hist: torch.Tensor, stream=None):
+        self._check(self.lib.ds_server_topk_slice_begin(self.handle, step, lo, hi, hist.data_ptr(), self._stream(stream)),
+                    "ds_server_topk_slice_begin")
+
+    def server_topk_slice_digit(self, level: int, lo: int, hi: int, hist_sum: torch.Tensor, hist_next: torch.Tensor, stream=None):
+        self._check(self.lib.ds_server_topk_slice_digit(self.handle, level, lo, hi, hist_sum.data_ptr(), hist_next.data_ptr(),
+                                                        self._stream(stream)), "ds_server_topk_slice_digit")
+
+    def server_topk_slice_emit(self, lo: int, hi: int, ties_to_keep: int, count: int, first_slot: int, fuse_apply: bool = True,
+                               stream=None):
+        self._check(self.lib.ds_server_topk_slice_emit(self.handle, lo, hi, ties_to_keep, count, first_slot,
+                                                       DS_FUSE_APPLY if fuse_apply else 0, self._stream(stream)),
+                    "ds_server_topk_slice_emit")
+
+    def apply_update_sparse_range(self, first_slot: int, count: int, stream=None):
+        self._check(self.lib.ds_apply_update_sparse_range(self.handle, first_slot, count, self._stream(stream)),
+                    "ds_apply_update_sparse_range")
 
     def step(self, g: torch.Tensor, t: int, fuse_apply: bool = True, stream=None):
         self.worker_compress(g, t, stream)

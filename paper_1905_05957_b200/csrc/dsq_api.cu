@@ -508,6 +508,79 @@ int ds_apply_update_slice(ds_handle h, uint64_t lo, uint64_t hi, void* cuda_stre
   return e == cudaSuccess ? DS_OK : cuda_fail(e, "apply update");
 }
 
+// ---- global top-k on the server pass when the vector's slices live on different GPUs ----------
+
+namespace {
+bool topk_slice_ok(const ds_ctx* h, uint64_t lo, uint64_t hi) {
+  return h->cfg.server_q.op == DS_Q_TOPK && h->cfg.server_q.k > 0 && sliceable(h->cfg.worker_q) && slice_ok(h, lo, hi);
+}
+}  // namespace
+
+int ds_server_topk_slice_begin(ds_handle h, uint32_t step, uint64_t lo, uint64_t hi, uint32_t* hist, void* cuda_stream) {
+  (void)step;   // the selection draws nothing
+  if (!h || !hist || (reinterpret_cast<uintptr_t>(hist) & 15u)) return DS_ERR_INVALID_ARG;
+  if (h->cfg.server_q.op != DS_Q_TOPK || !sliceable(h->cfg.worker_q)) return DS_ERR_UNSUPPORTED;
+  if (!topk_slice_ok(h, lo, hi)) return DS_ERR_INVALID_ARG;
+  int kind = 0;
+  SrcParams src = server_src(h, &kind);
+  const ds_qspec& wq = h->cfg.worker_q;
+  src.d = hi - lo;
+  float* ds_slice = h->buf.delta_s + lo;   // v is laid out here; without compensation it is scratch
+  src.delta = no_compensation(h->cfg) ? nullptr : ds_slice;
+  switch (wq.op) {
+    case DS_Q_IDENTITY: src.wp_off[0] += lo * 4; break;
+    case DS_Q_SIGN1: src.wp_off[0] += lo / 8; src.wp_off[1] += lo / wq.chunk * 4; break;
+    case DS_Q_QSGD: src.wp_off[0] += lo; src.wp_off[1] += lo / 8; src.wp_off[2] += lo / wq.chunk * 4; break;
+    case DS_Q_CLIP: src.wp_off[0] += lo * ((32 - wq.levels) / 8); break;
+    case DS_Q_RSPARSE: src.wp_off[0] += lo / wq.levels * 4; src.wp_off[1] += lo / wq.chunk * 4; break;
+    default: return DS_ERR_UNSUPPORTED;
+  }
+  const cudaError_t e = launch_topk_slice_begin(kind, src, h->buf.workspace, ds_slice, h->cfg.server_q.k, hist,
+                                                static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "top-k over a slice, first histogram");
+}
+
+int ds_server_topk_slice_digit(ds_handle h, int level, uint64_t lo, uint64_t hi, uint32_t* hist_sum, uint32_t* hist_next,
+                               void* cuda_stream) {
+  if (!h || !hist_sum || !hist_next || level < 1 || level > 3) return DS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(hist_sum) | reinterpret_cast<uintptr_t>(hist_next)) & 15u) return DS_ERR_ALIGN;
+  if (h->cfg.server_q.op != DS_Q_TOPK) return DS_ERR_UNSUPPORTED;
+  if (!topk_slice_ok(h, lo, hi)) return DS_ERR_INVALID_ARG;
+  const cudaError_t e = launch_topk_slice_digit(level, h->buf.workspace, h->buf.delta_s + lo, hi - lo, 1, h->cfg.server_q.k, hist_sum,
+                                                hist_next, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "top-k over a slice, digit");
+}
+
+int ds_server_topk_slice_emit(ds_handle h, uint64_t lo, uint64_t hi, uint32_t ties_to_keep, uint32_t count, uint64_t first_slot,
+                              uint32_t flags, void* cuda_stream) {
+  if (!h || (flags & ~DS_FUSE_APPLY)) return DS_ERR_INVALID_ARG;
+  if (h->cfg.server_q.op != DS_Q_TOPK) return DS_ERR_UNSUPPORTED;
+  if (!topk_slice_ok(h, lo, hi) || first_slot + count > h->cfg.server_q.k) return DS_ERR_INVALID_ARG;
+  uint8_t* sp = static_cast<uint8_t*>(h->buf.server_payload);
+  uint32_t* idx = reinterpret_cast<uint32_t*>(sp + h->sl.off[0]) + first_slot;
+  float* val = reinterpret_cast<float*>(sp + h->sl.off[1]) + first_slot;
+  const cudaError_t e = launch_topk_slice_emit(h->buf.workspace, h->buf.delta_s + lo, hi - lo, h->cfg.server_q.k, ties_to_keep, count,
+                                               (uint32_t)lo, idx, val, (flags & DS_FUSE_APPLY) ? h->buf.x + lo : nullptr, h->cfg.gamma,
+                                               static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "top-k over a slice, emit");
+}
+
+int ds_apply_update_sparse_range(ds_handle h, uint64_t first_slot, uint64_t count, void* cuda_stream) {
+  if (!h) return DS_ERR_INVALID_ARG;
+  if (h->cfg.server_q.op != DS_Q_TOPK) return DS_ERR_UNSUPPORTED;
+  if (first_slot + count > h->cfg.server_q.k) return DS_ERR_INVALID_ARG;
+  if (count == 0) return DS_OK;
+  PayloadView pv;
+  memset(&pv, 0, sizeof pv);
+  pv.op = DS_Q_TOPK;
+  pv.base = static_cast<const uint8_t*>(h->buf.server_payload);
+  pv.off[0] = h->sl.off[0] + first_slot * 4;
+  pv.off[1] = h->sl.off[1] + first_slot * 4;
+  pv.k = count;
+  const cudaError_t e = launch_apply(pv, h->buf.x, h->cfg.d, h->cfg.gamma, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? DS_OK : cuda_fail(e, "apply update, part of a sparse payload");
+}
+
 int ds_step_host(ds_handle h, const float* g_host, float* g_dev, uint32_t step, void* server_payload_host, float* x_host,
                  void* cuda_stream) {
   if (!h || !g_host || !g_dev) return DS_ERR_INVALID_ARG;

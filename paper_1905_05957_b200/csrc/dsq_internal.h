@@ -150,6 +150,17 @@ void topk_plan(uint64_t d, uint32_t rows, uint64_t k, bool with_list, TopkPlan* 
 cudaError_t launch_topk(int src_kind, const SrcParams& src, const TopkPlan& plan, void* workspace, const TopkIO& io,
                         uint32_t rows, uint64_t k, cudaStream_t st);
 
+// The selection over ONE slice of a vector that lives on several GPUs, stage by stage (see
+// ds_server_topk_slice_* in dsq.h): the scratch is carved from the start of `workspace`.
+uint64_t topk_slice_workspace_bytes(uint64_t d_slice, uint64_t k);
+cudaError_t launch_topk_slice_begin(int src_kind, const SrcParams& src, void* workspace, float* v_out, uint64_t k,
+                                    uint32_t* hist_out, cudaStream_t st);
+cudaError_t launch_topk_slice_digit(int level, void* workspace, const float* v, uint64_t d_slice, int vec, uint64_t k,
+                                    uint32_t* hist_sum, uint32_t* hist_next, cudaStream_t st);
+cudaError_t launch_topk_slice_emit(void* workspace, float* v_io, uint64_t d_slice, uint64_t k, uint32_t ties_to_keep,
+                                   uint32_t count, uint32_t idx_base, uint32_t* out_idx, float* out_val, float* x, float gamma,
+                                   cudaStream_t st);
+
 cudaError_t launch_chunked(int op, int src_kind, const SrcParams& src, const ChunkParams& p, uint32_t rows,
                            uint32_t chunk, cudaStream_t st);
 

@@ -1038,7 +1038,7 @@ __device__ __forceinline__ void cta_scan_counts(uint32_t row, uint2* seg_cnt, co
     const uint32_t r = state[row].r;
     state[row].total_gt = tot.x;
     state[row].total_tie = tot.y;
-    if (tot.x + min(tot.y, r) != k) atomicOr(dev_status, DS_DEV_TOPK_INCONSISTENT);
+    if (k != 0xFFFFFFFFu && tot.x + min(tot.y, r) != k) atomicOr(dev_status, DS_DEV_TOPK_INCONSISTENT);
   }
 }
 
@@ -1047,6 +1047,33 @@ __global__ void __launch_bounds__(1024) k_topk_scan(uint2* seg_cnt, uint64_t nse
                                                     uint32_t* dev_status) {
   pdl_prologue();
   cta_scan_counts<false>(blockIdx.x, seg_cnt, nullptr, nseg, state, k, dev_status);
+}
+
+// ================================================================ a slice of a vector that lives on several GPUs
+// The selection over a vector whose slices sit on different GPUs is the pipeline without a list, cut
+// where a histogram is complete: the caller adds the slices' histograms up (an all-reduce of 16 KB) and
+// hands the sum back, every slice then picks the same digit.  See ds_server_topk_slice_* in dsq.h.
+
+// The prefix over the segment counts of ONE slice; how many entries the slice holds above tau and equal
+// to it, and the tie quota r of the whole vector, go to out[0..2].  No check against k: that is the
+// whole vector's business.
+__global__ void __launch_bounds__(1024) k_topk_slice_scan(uint2* seg_cnt, uint64_t nseg, TopkState* state, uint32_t* out) {
+  pdl_prologue();
+  __shared__ uint32_t s_ignore;
+  cta_scan_counts<false>(0, seg_cnt, nullptr, nseg, state, 0xFFFFFFFFu, &s_ignore);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    out[0] = state[0].total_gt;
+    out[1] = state[0].total_tie;
+    out[2] = state[0].r;
+    out[3] = state[0].tau;
+  }
+}
+
+// The slice's share of the tie quota, decided by the caller from all slices' tie counts.
+__global__ void k_topk_slice_quota(TopkState* state, uint32_t ties_to_keep) {
+  pdl_prologue();
+  if (threadIdx.x == 0 && blockIdx.x == 0) state[0].r = ties_to_keep;
 }
 
 // ---------------------------------------------------------------- classify + prefix
@@ -1106,7 +1133,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
                                                         const uint32_t* bm_gt, const uint32_t* bm_eq, uint64_t bm_stride,
                                                         const uint2* seg_pre, uint64_t nseg, uint8_t* payload,
                                                         uint64_t payload_stride, uint64_t off_idx, uint64_t off_val,
-                                                        uint32_t k, float* x, float gamma) {
+                                                        uint32_t k, float* x, float gamma, uint32_t idx_base) {
   pdl_prologue();
   __shared__ uint32_t s_warp[kThreads / 32];
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5, row = blockIdx.y;
@@ -1166,14 +1193,14 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
         // no tie in this word: the prefetched values are its first two entries
         if (b0[i] < 32u) {
           const uint64_t j = (widx + i) * 32u + b0[i];
-          if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v0[i]; }  // pos < k whenever the counts are consistent
+          if (pos < k) { out_idx[pos] = (uint32_t)j + idx_base; out_val[pos] = v0[i]; }  // pos < k whenever the counts are consistent
           vrow[j] = 0.f;                                                      // delta = v - Q[v] at a kept entry
           if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v0[i]));
           ++pos;
         }
         if (b1[i] < 32u) {
           const uint64_t j = (widx + i) * 32u + b1[i];
-          if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = v1[i]; }
+          if (pos < k) { out_idx[pos] = (uint32_t)j + idx_base; out_val[pos] = v1[i]; }
           vrow[j] = 0.f;
           if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, v1[i]));
           ++pos;
@@ -1186,7 +1213,7 @@ __global__ void __launch_bounds__(kThreads) k_topk_emit(float* v_io, uint64_t d,
         sel &= sel - 1u;
         const uint64_t j = (widx + i) * 32u + b;
         const float val = vrow[j];
-        if (pos < k) { out_idx[pos] = (uint32_t)j; out_val[pos] = val; }
+        if (pos < k) { out_idx[pos] = (uint32_t)j + idx_base; out_val[pos] = val; }
         vrow[j] = 0.f;
         if (x) x[j] = __fsub_rn(x[j], __fmul_rn(gamma, val));
         ++pos;
@@ -1302,7 +1329,93 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
   }
   launch_pdl(k_topk_scan, rows, 1024, st, seg, pl.nseg, state, k32, io.dev_status);
   launch_pdl(k_topk_emit, gs, kThreads, st, io.v_inout, d, state, bm_gt, bm_eq, pl.bm_stride, seg, pl.nseg,
-                                       reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x, io.gamma);
+                                       reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x, io.gamma, 0u);
+  count_launches(2);
+  return cudaGetLastError();
+}
+
+
+// ---------------------------------------------------------------- stages of the selection over a slice
+namespace {
+struct SlicePtrs {
+  uint32_t* hist;
+  TopkState* state;
+  uint32_t *bm_gt, *bm_eq;
+  uint2* seg;
+  TopkPlan pl;
+  uint64_t padded;
+};
+SlicePtrs slice_ptrs(uint64_t d_slice, uint64_t k, void* workspace) {
+  SlicePtrs p;
+  topk_plan(d_slice, 1, k, false, &p.pl);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  p.hist = reinterpret_cast<uint32_t*>(ws + p.pl.off_hist);
+  p.state = reinterpret_cast<TopkState*>(ws + p.pl.off_state);
+  p.bm_gt = reinterpret_cast<uint32_t*>(ws + p.pl.off_bm_gt);
+  p.bm_eq = reinterpret_cast<uint32_t*>(ws + p.pl.off_bm_eq);
+  p.seg = reinterpret_cast<uint2*>(ws + p.pl.off_seg);
+  p.padded = p.pl.nseg * (uint64_t)kSegElems;
+  return p;
+}
+dim3 stride_grid(const TopkPlan& pl) {
+  uint64_t ctas = 148ull * 4ull;
+  if (ctas > pl.ntile) ctas = pl.ntile;
+  return dim3((unsigned)ctas, 1, 1);
+}
+}  // namespace
+
+uint64_t topk_slice_workspace_bytes(uint64_t d_slice, uint64_t k) {
+  TopkPlan pl;
+  topk_plan(d_slice, 1, k, false, &pl);
+  return pl.bytes;
+}
+
+cudaError_t launch_topk_slice_begin(int srck, const SrcParams& src, void* workspace, float* v_out, uint64_t k, uint32_t* hist_out,
+                                    cudaStream_t st) {
+  const SlicePtrs p = slice_ptrs(src.d, k, workspace);
+  cudaError_t e = cudaMemsetAsync(hist_out, 0, kBins1 * 4, st);
+  if (e != cudaSuccess) return e;
+  uint64_t span = 16 * kTile;
+  while (span > kTile && ((p.padded + span - 1) / span) < 148ull * 16ull) span /= 2;
+  dim3 g1b((unsigned)((p.padded + span - 1) / span), 1, 1);
+#define DSQ_P1(S) launch_pdl(k_topk_pass1_basic<S>, g1b, kThreads, st, src, v_out, hist_out, span)
+  DSQ_SWITCH_SRC(srck, DSQ_P1)
+#undef DSQ_P1
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topk_slice_digit(int level, void* workspace, const float* v, uint64_t d_slice, int vec, uint64_t k,
+                                    uint32_t* hist_sum, uint32_t* hist_next, cudaStream_t st) {
+  const SlicePtrs p = slice_ptrs(d_slice, k, workspace);
+  const uint32_t k32 = (uint32_t)k;
+  dim3 gs((unsigned)p.pl.nseg, 1, 1);
+  cudaError_t e = cudaMemsetAsync(hist_next, 0, kBins1 * 4, st);
+  if (e != cudaSuccess) return e;
+  launch_pdl(k_topk_pick_basic, 1, 1024, st, hist_sum, p.state, (uint32_t)level, k32);   // clears hist_sum
+  if (level == 1) {
+    launch_pdl(k_topk_mark_basic, stride_grid(p.pl), kThreads, st, v, d_slice, vec, p.state, p.bm_gt, p.bm_eq, p.pl.bm_stride, p.padded);
+    launch_pdl(k_topk_refine<2>, gs, kThreads, st, v, d_slice, p.state, p.bm_eq, p.pl.bm_stride, hist_next);
+    count_launches(3);
+  } else if (level == 2) {
+    launch_pdl(k_topk_refine<3>, gs, kThreads, st, v, d_slice, p.state, p.bm_eq, p.pl.bm_stride, hist_next);
+    count_launches(2);
+  } else {
+    launch_pdl(k_topk_finalize, gs, kThreads, st, v, d_slice, p.state, p.bm_gt, p.bm_eq, p.pl.bm_stride, p.seg, p.pl.nseg);
+    launch_pdl(k_topk_slice_scan, 1, 1024, st, p.seg, p.pl.nseg, p.state, hist_next);
+    count_launches(3);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_topk_slice_emit(void* workspace, float* v_io, uint64_t d_slice, uint64_t k, uint32_t ties_to_keep, uint32_t count,
+                                   uint32_t idx_base, uint32_t* out_idx, float* out_val, float* x, float gamma, cudaStream_t st) {
+  const SlicePtrs p = slice_ptrs(d_slice, k, workspace);
+  dim3 gs((unsigned)p.pl.nseg, 1, 1);
+  const uint64_t off_val = (uint64_t)(reinterpret_cast<uint8_t*>(out_val) - reinterpret_cast<uint8_t*>(out_idx));
+  launch_pdl(k_topk_slice_quota, 1, 32, st, p.state, ties_to_keep);
+  launch_pdl(k_topk_emit, gs, kThreads, st, v_io, d_slice, p.state, p.bm_gt, p.bm_eq, p.pl.bm_stride, p.seg, p.pl.nseg,
+             reinterpret_cast<uint8_t*>(out_idx), (uint64_t)0, (uint64_t)0, off_val, count, x, gamma, idx_base);
   count_launches(2);
   return cudaGetLastError();
 }

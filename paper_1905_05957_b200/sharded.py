@@ -12,6 +12,10 @@ allows):
      compressed hop)                              exchange_server_payload
   5. update of x on the other slices              ds_apply_update_slice
 
+A top-k server (its threshold is a property of the whole vector) replaces 3-5 by the staged calls
+ds_server_topk_slice_begin / _digit / _emit with three all-reduces of a 4096-bin histogram and one
+all-gather of four words in between, then an all-gather of the slices' (index, value) lists.
+
 Every step of the arithmetic runs in the library's kernels; this module only says which bytes
 move where.  The moves go through a `transport` with two methods, so that the same plan runs over
 torch.distributed point-to-point operations (NCCL between GPUs, gloo in the CPU test) and over plain
@@ -167,6 +171,18 @@ class DistTransport:
     def all_gather(self, mine: torch.Tensor, recv_sizes: list[int]) -> list[torch.Tensor]:
         return self._exchange([mine] * self.world, recv_sizes)
 
+    def all_reduce_sum(self, t: torch.Tensor):
+        """In-place sum over the ranks (the 4096-bin histograms of a top-k over slices)."""
+        self.bytes_sent += int(t.numel() * t.element_size())
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM, group=self.group)
+
+    def all_gather_small(self, t: torch.Tensor) -> list[torch.Tensor]:
+        """Every rank's copy of a few words."""
+        out = [torch.empty_like(t) for _ in range(self.world)]
+        self.bytes_sent += int(t.numel() * t.element_size()) * (self.world - 1)
+        self.dist.all_gather(out, t, group=self.group)
+        return out
+
 
 class ShardedDoubleSqueeze:
     """One rank of the one-worker-per-GPU deployment (see the module text).  `ds` is this rank's
@@ -203,9 +219,94 @@ class ShardedDoubleSqueeze:
             if q != self.rank and hi > lo:
                 self.ds.apply_update_slice(lo, hi)
 
+    # -- a top-k server: its threshold belongs to the whole vector, so the pass is cut into stages between
+    # -- which the slices' histograms are added up over the ranks ------------------------------------------
+    @property
+    def server_is_topk(self) -> bool:
+        return self.ds.server_q.op == "topk"
+
+    def _hists(self):
+        if not hasattr(self, "_hist"):
+            dev = self.ds.server_payload.device
+            self._hist = [torch.zeros(4096, dtype=torch.int32, device=dev) for _ in range(2)]
+        return self._hist
+
+    def topk_begin(self, t: int) -> torch.Tensor:
+        """Stage 1: v on the own slice and its first-digit histogram (to be summed over the ranks)."""
+        h = self._hists()[0]
+        if self.hi > self.lo:
+            self.ds.server_topk_slice_begin(t, self.lo, self.hi, h)
+        else:
+            h.zero_()
+        return h
+
+    def topk_digit(self, level: int) -> torch.Tensor:
+        """Stage 2, level 1..3: consumes the summed histogram of the previous stage, returns this slice's next one
+        (after level 3: above, ties, r, tau in its first four words)."""
+        a, b = self._hists()
+        src, dst = (a, b) if level % 2 == 1 else (b, a)
+        if self.hi > self.lo:
+            self.ds.server_topk_slice_digit(level, self.lo, self.hi, src, dst)
+        else:
+            dst.zero_()          # an empty slice holds nothing; r and tau come from the others
+        return dst
+
+    @staticmethod
+    def topk_shares(totals: list[tuple[int, int]], r: int) -> list[tuple[int, int, int]]:
+        """From every slice's (entries above tau, entries equal to tau) and the vector's tie quota r: per slice
+        (ties to keep, entries kept, first output slot).  Ties go to lower indices, i.e. to earlier slices, first."""
+        out, ties_before, slot = [], 0, 0
+        for above, ties in totals:
+            keep = max(0, min(ties, r - ties_before))
+            out.append((keep, above + keep, slot))
+            ties_before += ties
+            slot += above + keep
+        return out
+
+    def topk_emit(self, share: tuple[int, int, int]):
+        keep, count, first = share
+        if self.hi > self.lo:
+            self.ds.server_topk_slice_emit(self.lo, self.hi, keep, count, first, fuse_apply=True)
+
+    def topk_parts(self, share: tuple[int, int, int]) -> tuple[torch.Tensor, torch.Tensor]:
+        """The own slice's part of the server payload: (indices, values) as byte tensors."""
+        _, count, first = share
+        v = self.ds.server_views()
+        return v["idx"][first:first + count].view(torch.uint8), v["val"][first:first + count].view(torch.uint8)
+
+    def topk_place(self, q: int, share: tuple[int, int, int], idx_bytes: torch.Tensor, val_bytes: torch.Tensor):
+        """Rank q's part into the local payload, and its update of x."""
+        _, count, first = share
+        if q == self.rank or count == 0:
+            return
+        v = self.ds.server_views()
+        v["idx"][first:first + count].view(torch.uint8).copy_(idx_bytes)
+        v["val"][first:first + count].view(torch.uint8).copy_(val_bytes)
+        self.ds.apply_update_sparse_range(first, count)
+
+    def server_topk(self, t: int, transport):
+        """The whole top-k server pass of this rank over a transport with collectives."""
+        h = self.topk_begin(t)
+        for level in (1, 2, 3):
+            transport.all_reduce_sum(h)
+            h = self.topk_digit(level)
+        words = [w.cpu() for w in transport.all_gather_small(h[:4].clone())]
+        r = max(int(w[2]) for w in words)                       # the same on every rank that holds a slice
+        shares = self.topk_shares([(int(w[0]), int(w[1])) for w in words], r)
+        self.topk_emit(shares[self.rank])
+        idx_b, val_b = self.topk_parts(shares[self.rank])
+        sizes = [4 * c for _, c, _ in shares]
+        got_idx = transport.all_gather(idx_b, sizes)
+        got_val = transport.all_gather(val_b, sizes)
+        for q in range(self.world):
+            self.topk_place(q, shares[q], got_idx[q], got_val[q])
+
     def step(self, g_row: torch.Tensor, t: int, transport):
         self.worker_pass(g_row, t)
         self.exchange_worker_payloads(transport)
+        if self.server_is_topk:
+            self.server_topk(t, transport)
+            return
         self.server_pass(t)
         self.exchange_server_payload(transport)
         self.apply_other_slices()
@@ -221,6 +322,23 @@ def step_in_process(ranks: list[ShardedDoubleSqueeze], g: torch.Tensor, t: int):
     sends = [r.plan.worker_send(r.ds.worker_payload) for r in ranks]
     for r in ranks:
         r.plan.worker_place(r.ds.worker_payload, [sends[i][r.rank] for i in range(world)])
+    if ranks[0].server_is_topk:
+        hs = [r.topk_begin(t) for r in ranks]
+        for level in (1, 2, 3):
+            total = torch.stack(hs).sum(dim=0, dtype=torch.int32)      # what the all-reduce would leave on every rank
+            for h in hs:
+                h.copy_(total)
+            hs = [r.topk_digit(level) for r in ranks]
+        words = [h[:4].cpu() for h in hs]
+        rr = max(int(w[2]) for w in words)
+        shares = ShardedDoubleSqueeze.topk_shares([(int(w[0]), int(w[1])) for w in words], rr)
+        for r in ranks:
+            r.topk_emit(shares[r.rank])
+        parts = [r.topk_parts(shares[r.rank]) for r in ranks]
+        for r in ranks:
+            for q in range(world):
+                r.topk_place(q, shares[q], parts[q][0], parts[q][1])
+        return
     for r in ranks:
         r.server_pass(t)
     slices = [r.plan.server_send(r.ds.server_payload) for r in ranks]

@@ -60,6 +60,48 @@ def test_sharded_step_equals_whole_vector_step(wq, sq, world, d):
     assert np.array_equal(whole.x.cpu().numpy().view(np.uint32), st.x.view(np.uint32))
 
 
+TOPK_PAIRS = [(SIGN, 1), (Q("qsgd", chunk=2048, levels=255), 2), (Q("clip", bits=16), 3), (Q("identity"), 4),
+              (Q("rsparse", chunk=1024, keep_one_in=8), 5)]
+
+
+@pytest.mark.parametrize("wq,kdiv", TOPK_PAIRS)
+@pytest.mark.parametrize("world,d", [(4, 5 * 8192 + 1234), (3, 8192 * 3), (5, 200_000), (2, 100)])
+def test_sharded_top_k_server_equals_whole_vector_step(wq, kdiv, world, d):
+    """A top-k server whose vector is spread over the ranks: the staged calls with the histograms summed over the ranks
+    in between must select exactly what the whole-vector pass selects (and that is the oracle's selection)."""
+    gamma, seed, T = 0.1, 78, 3
+    k = max(1, d // (20 * kdiv))
+    sq = Q("topk", k=k)
+    gen = torch.Generator().manual_seed(world * 1000 + d + kdiv)
+    gs = [torch.randn(world, d, generator=gen).cuda() for _ in range(T)]
+    if kdiv == 4:   # identity workers: integer-valued gradients, so that many entries tie at the threshold across slices
+        gs = [torch.randint(-3, 4, (world, d), generator=gen).float().cuda() for _ in range(T)]
+    whole = DoubleSqueeze(world, d, gamma, wq, sq, seed)
+    st = oracle.State.zeros(world, d)
+    ranks = [ShardedDoubleSqueeze(DoubleSqueeze(world, d, gamma, wq, sq, seed, delta_w_rows=1), r, world) for r in range(world)]
+    bounds = slice_bounds(d, world)
+    for t, g in enumerate(gs):
+        whole.step(g, t)
+        step_in_process(ranks, g, t)
+        torch.cuda.synchronize()
+        oracle.step(st, g.cpu().numpy(), to_oracle_q(wq), to_oracle_q(sq), gamma, seed, t)
+        compare_state(whole, st, g.cpu().numpy(), tag=f"whole, step {t}: ")
+        for r in ranks:
+            lo, hi = bounds[r.rank]
+            assert torch.equal(_bits(r.ds.x), _bits(whole.x)), f"x on rank {r.rank}, step {t}"
+            assert torch.equal(_bits(r.ds.delta_w[0]), _bits(whole.delta_w[r.rank]))
+            assert torch.equal(_bits(r.ds.delta_s[lo:hi]), _bits(whole.delta_s[lo:hi]))
+            for name, view in r.ds.server_views().items():
+                assert torch.equal(_bits(view), _bits(whole.server_views()[name])), f"server payload {name} on rank {r.rank}"
+            assert r.ds.device_status() == 0
+
+
+def test_tie_quota_is_dealt_to_earlier_slices_first():
+    shares = ShardedDoubleSqueeze.topk_shares([(5, 2), (0, 3), (7, 0), (1, 4)], r=4)
+    assert shares == [(2, 7, 0), (2, 2, 7), (0, 7, 9), (0, 1, 16)]
+    assert ShardedDoubleSqueeze.topk_shares([(0, 0), (3, 1)], r=1) == [(0, 0, 0), (1, 4, 0)]
+
+
 def test_slices_reject_what_they_cannot_do():
     ds = DoubleSqueeze(2, 40_000, 0.1, SIGN, SIGN)
     g = torch.randn(2, 40_000, device="cuda")

@@ -199,3 +199,40 @@ def test_whole_iteration_over_gloo_runs_its_phases_in_order_and_moves_the_planne
     # the compressed hops move a small fraction of what the dense vector would: 9/32 and 1/32 of 4 bytes per entry here
     dense = 4 * D
     assert got[0][2][0] < 0.25 * dense
+
+
+# ------------------------------------------------------------------ collectives of the top-k server over slices
+
+def _collectives_main(rank: int, world: int, port: int, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_1905_05957_b200.sharded import ShardedDoubleSqueeze
+    tr = DistTransport()
+    hist = (torch.arange(4096, dtype=torch.int32) % 7) * (rank + 1)        # this slice's histogram
+    tr.all_reduce_sum(hist)
+    words = tr.all_gather_small(torch.tensor([10 * rank + 1, rank, 5, 1234], dtype=torch.int32))
+    shares = ShardedDoubleSqueeze.topk_shares([(int(w[0]), int(w[1])) for w in words], max(int(w[2]) for w in words))
+    dist.barrier()
+    out.put((rank, hist.tolist()[:16], [w.tolist() for w in words], shares, tr.bytes_sent))
+    dist.destroy_process_group()
+
+
+def test_histogram_sum_and_totals_gather_over_gloo():
+    world, port = 3, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_collectives_main, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = [out.get(timeout=180) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    want_hist = [(i % 7) * (1 + 2 + 3) for i in range(16)]
+    want_words = [[10 * r + 1, r, 5, 1234] for r in range(world)]
+    # ties 0, 1, 2 per slice and a quota of 5: every tie is kept; the slots follow the kept counts
+    want_shares = [(0, 1, 0), (1, 12, 1), (2, 23, 13)]
+    for rank, hist, words, shares, sent in got:
+        assert hist == want_hist and words == want_words and shares == want_shares
+        assert sent == 4096 * 4 + 16 * (world - 1)
