@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the DoubleSqueeze step (worker pass + server pass with fused model update).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..8] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..12] [--impl ours|reference]
 
 One "step" is one whole iteration of Algorithm 1 over one batch of synthetic gradients
 (ds_worker_compress + ds_server_aggregate_compress with the fused update).  Prints ONE JSON line.
@@ -49,10 +49,13 @@ HEADLINE = 5                 # the largest one that fits one GPU
 # (a multi-pass capture must stay small) is scaled by the entries one launch processes: the
 # traffic of a streaming kernel grows in proportion.
 NCU_CAPTURES = {
-    "sign1": ("k_chunked<SIGN1, WORKER, 4, 256>", 748169472 + 332183040, 8 * 11_689_512, "5be2583994dd727b"),
-    "qsgd": ("k_chunked<QSGD, WORKER, 2, 256>", 1073773000 + 629989632, 8 * 16_777_216, "5be2583994dd727b"),
-    "clip": ("k_clip<WORKER, 16>", 748325376 + 508748800, 8 * 11_689_512, "8936b8b285292618"),
-    "rsparse": ("k_rsparse<WORKER>", 748242176 + 331810048, 8 * 11_689_512, "8936b8b285292618"),
+    "sign1": ("k_chunked<SIGN1, WORKER, 4, 256>", 748182784 + 332558080, 8 * 11_689_512, "776947eec84228a6"),
+    "qsgd": ("k_chunked<QSGD, WORKER, 2, 256>", 1073776000 + 630281472, 8 * 16_777_216, "776947eec84228a6"),
+    # the first kernel of the top-k worker pass alone (v read once, written once); the selection that follows it
+    # moves a few percent of that
+    "topk": ("k_topk_pass1<WORKER>", 537250304 + 221670400, 16 * 4_194_304, "473ea00871451d04"),
+    "clip": ("k_clip<WORKER, 16>", 748329216 + 508803584, 8 * 11_689_512, "8f64db8f3c6b7019"),
+    "rsparse": ("k_rsparse<WORKER>", 748263680 + 332954624, 8 * 11_689_512, "8f64db8f3c6b7019"),
 }
 KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "sign1": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
