@@ -33,6 +33,8 @@ enum Src : int {
   SRC_SRV_RSPARSE = 6,   // payload = the survivors of every chunk and the chunk's draw
   SRC_WORKER_PLAIN = 7,  // v = g[row]: a worker that keeps no error (no compensation)
   SRC_SRV_TERNARY = 8,   // payload = sign words, non-zero words and one factor per worker
+  SRC_STORED = 9,        // v = delta[row]: an earlier kernel of the same pass formed v and left it where the error lives
+                         // (operators with one factor per vector only; not part of DSQ_SWITCH_SRC)
 };
 
 __host__ __device__ constexpr bool is_worker_src(int src) { return src == SRC_WORKER || src == SRC_WORKER_PLAIN; }
@@ -150,6 +152,20 @@ __device__ __forceinline__ void src_load_tile(const SrcParams& p, uint32_t row, 
     const uint64_t off = (uint64_t)row * p.d;
 #pragma unroll
     for (int j = 0; j < V; ++j) v[j] = load_row4(p.g + off, e[j], cnt[j], p.vec);
+  } else if constexpr (SRC == SRC_STORED) {
+    // written by the previous kernel of the chain: ordinary loads
+    const float* vr = p.delta + (uint64_t)row * p.d;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (p.vec && cnt[j] == 4) {
+        v[j] = *reinterpret_cast<const float4*>(vr + e[j]);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)k < cnt[j]) comp(v[j], k) = vr[e[j] + k];
+      }
+    }
   } else {
     const uint32_t lane = threadIdx.x & 31u;
     float4 acc[V], ds[V];

@@ -6,9 +6,11 @@
 //     magnitude(v) / magnitude(ternary vector) multiplies the result.
 //
 // The factor needs a sum over all d entries before the first residual can be written, so a pass is a
-// chain of kernels.  v (Eq. 2 on a worker, Eq. 4 on the server) is recomputed from its source in each
-// of them rather than stored: that costs the same bytes as a round trip through memory and leaves
-// the error buffer untouched until the final kernel overwrites it.
+// chain of kernels.  Where an error is kept, the first kernel forms v (Eq. 2 on a worker, Eq. 4 on the
+// server) and leaves it in the error buffer, which the last kernel overwrites with the residual; the
+// kernels in between read v from there (source SRC_STORED: 4 bytes per entry instead of the 8 of a
+// worker's g and delta, and no second or third decoding of the n payloads on the server).  Without
+// an error buffer (no compensation) v is recomputed from its source in every kernel.
 //
 //   1-bit:    reduce (tile sums of |v| or v*v) -> finalize (factor) -> sign (words, residual, update)
 //   ternary:  reduce (tile sums of |v|, tile maxima) -> finalize (||v||_1, m) -> draw (sign and
@@ -59,6 +61,13 @@ __device__ __forceinline__ void load_tile(const SrcParams& src, uint32_t row, ui
       cnt[j] = 4;
       v[j] = add4_rn(a[j], b[j]);
     }
+  } else if constexpr (FULL && SRC == SRC_STORED) {
+    const float4* vp = reinterpret_cast<const float4*>(src.delta + (uint64_t)row * d + base) + tid;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      cnt[j] = 4;
+      v[j] = vp[j * kThreads];
+    }
   } else {
     uint64_t e[4];
 #pragma unroll
@@ -87,12 +96,28 @@ __device__ __forceinline__ uint32_t cta_reduce_u32(uint32_t x, uint32_t* s_w) {
 // ---------------------------------------------------------------- tile sums (and maxima)
 // MODE 0: sum |v|;  1: sum v*v;  2: sum |v| and max |v|.
 template <int SRC, int MODE, bool FULL>
-__device__ __forceinline__ void reduce_body(const SrcParams& src, const WholeScratch& ws, float* s_red, uint32_t* s_w) {
+__device__ __forceinline__ void reduce_body(const SrcParams& src, const WholeScratch& ws, float* v_store, float* s_red,
+                                            uint32_t* s_w) {
   const uint32_t row = blockIdx.y;
   const uint64_t tile = blockIdx.x;
   float4 v[4];
   uint32_t cnt[4];
   load_tile<SRC, FULL>(src, row, tile * kWTile, v, cnt);
+  if (v_store) {
+    // v for the kernels that follow
+    float* vr = v_store + (uint64_t)row * src.d;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint64_t e = tile * kWTile + (uint64_t)(j * kThreads + threadIdx.x) * 4u;
+      if (FULL || (src.vec && cnt[j] == 4)) {
+        *reinterpret_cast<float4*>(vr + e) = v[j];
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((uint32_t)k < cnt[j]) vr[e + k] = compc(v[j], k);
+      }
+    }
+  }
   float part[4];
   uint32_t mx = 0;
 #pragma unroll
@@ -118,12 +143,15 @@ __device__ __forceinline__ void reduce_body(const SrcParams& src, const WholeScr
 
 template <int SRC, int MODE>
 __global__ void __launch_bounds__(kThreads, is_worker_src(SRC) ? 0 : kServerCtasPerSm) k_whole_reduce(const SrcParams src,
-                                                                                                       const WholeScratch ws) {
+                                                                                                       const WholeScratch ws,
+                                                                                                       float* v_store) {
+  // v_store: NULL, or [rows, d] where v is left for the kernels that follow (it may be the buffer v's
+  // error term was just read from: a thread writes only the entries it has read)
   pdl_prologue();
   __shared__ float s_red[64];
   __shared__ uint32_t s_w[kThreads / 32];
-  if (src.vec && ((uint64_t)blockIdx.x + 1) * kWTile <= src.d) reduce_body<SRC, MODE, true>(src, ws, s_red, s_w);
-  else reduce_body<SRC, MODE, false>(src, ws, s_red, s_w);
+  if (src.vec && ((uint64_t)blockIdx.x + 1) * kWTile <= src.d) reduce_body<SRC, MODE, true>(src, ws, v_store, s_red, s_w);
+  else reduce_body<SRC, MODE, false>(src, ws, v_store, s_red, s_w);
 }
 
 // ---------------------------------------------------------------- combining the tile results
@@ -370,38 +398,47 @@ cudaError_t launch_whole(int op, int srck, const SrcParams& src, const WholePara
   ws.part_aux = reinterpret_cast<uint32_t*>(w + part_bytes);
   ws.fin = reinterpret_cast<WholeFin*>(w + 2 * part_bytes);
   const dim3 grid((unsigned)ws.ntile, rows, 1);
+  // v can be left in the error buffer if the pass has one, reads its error term from it and writes rows d apart
+  const bool stored = srck != SRC_WORKER_PLAIN && p.delta_out != nullptr && src.delta == p.delta_out &&
+                      (rows == 1 || p.delta_row_stride == src.d);
+  float* v_store = stored ? p.delta_out : nullptr;
+  // the source of the kernels after the first
+  const int srck2 = stored ? (int)SRC_STORED : srck;
+#define DSQ_SWITCH_SRC2(X)                                   \
+  if (srck2 == SRC_STORED) { X(SRC_STORED); } else { DSQ_SWITCH_SRC(srck2, X) }
   if (op == DS_Q_SIGN1) {
     if (p.l2) {
-#define DSQ_W(S) launch_pdl(k_whole_reduce<S, 1>, grid, kThreads, st, src, ws)
+#define DSQ_W(S) launch_pdl(k_whole_reduce<S, 1>, grid, kThreads, st, src, ws, v_store)
       DSQ_SWITCH_SRC(srck, DSQ_W)
 #undef DSQ_W
     } else {
-#define DSQ_W(S) launch_pdl(k_whole_reduce<S, 0>, grid, kThreads, st, src, ws)
+#define DSQ_W(S) launch_pdl(k_whole_reduce<S, 0>, grid, kThreads, st, src, ws, v_store)
       DSQ_SWITCH_SRC(srck, DSQ_W)
 #undef DSQ_W
     }
     launch_pdl(k_whole_finalize<0>, rows, 1024, st, ws, src.d, p.l2, p.out_scale, p.word_stride);
 #define DSQ_W(S) launch_pdl(k_whole_sign<S>, grid, kThreads, st, src, p, ws)
-    DSQ_SWITCH_SRC(srck, DSQ_W)
+    DSQ_SWITCH_SRC2(DSQ_W)
 #undef DSQ_W
     count_launches(3);
     return cudaGetLastError();
   }
   if (op == DS_Q_TERNARY) {
-#define DSQ_W(S) launch_pdl(k_whole_reduce<S, 2>, grid, kThreads, st, src, ws)
+#define DSQ_W(S) launch_pdl(k_whole_reduce<S, 2>, grid, kThreads, st, src, ws, v_store)
     DSQ_SWITCH_SRC(srck, DSQ_W)
 #undef DSQ_W
     launch_pdl(k_whole_finalize<1>, rows, 1024, st, ws, src.d, 0u, p.out_scale, p.word_stride);
 #define DSQ_W(S) launch_pdl(k_whole_ternary_draw<S>, grid, kThreads, st, src, p, ws)
-    DSQ_SWITCH_SRC(srck, DSQ_W)
+    DSQ_SWITCH_SRC2(DSQ_W)
 #undef DSQ_W
     launch_pdl(k_whole_finalize<2>, rows, 1024, st, ws, src.d, 0u, p.out_scale, p.word_stride);
 #define DSQ_W(S) launch_pdl(k_whole_ternary_apply<S>, grid, kThreads, st, src, p, ws)
-    DSQ_SWITCH_SRC(srck, DSQ_W)
+    DSQ_SWITCH_SRC2(DSQ_W)
 #undef DSQ_W
     count_launches(5);
     return cudaGetLastError();
   }
+#undef DSQ_SWITCH_SRC2
   return cudaErrorInvalidValue;
 }
 
