@@ -108,7 +108,7 @@ struct TopkState {
   uint32_t tau;        // full 31-bit key of the k-th largest entry
   uint32_t r;          // how many entries with key == tau are kept (lowest indices first)
   uint32_t total_gt, total_tie;
-  uint32_t need_mark;  // 1: the tile regions pass1 wrote (if any) do not bracket the threshold
+  uint32_t reserved0;
   uint32_t need_full;  // 1: the candidates pass1 listed (if any) did not contain the k-th entry
   uint32_t zeroed_above;  // entries with a key above this were zeroed in the residual when they were listed
 };

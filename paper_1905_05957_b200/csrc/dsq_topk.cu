@@ -17,14 +17,15 @@
 //   lhist 1    copies the entries inside the band (the candidates) out of the regions into one
 //              dense (key, index) list and counts the top 12 key bits on the way; accepts the
 //              prediction only if the k-th entry is a candidate (above < k <= above + candidates)
-//   hist, pick only after a miss (or without history): entries zeroed by pass1 are restored from
-//              the regions, then a full 4096-bin histogram of v gives the exact bin tb
-//   mark, compact  only after a miss: re-read v, rebuild regions and dense list for the exact bin
+//   hist       only after a miss (or without history): entries zeroed by pass1 are restored from
+//              the regions, then a full 4096-bin histogram of v is counted
+//   mark       only after a miss: the exact bin tb from that histogram; re-read v, rebuild the
+//              regions and the dense list for that bin
 //   lhist 2,3  the next 12, then the last 7 key bits from the dense list: tau and r
 //   classify   every candidate with key >= tau adds one to its tile's counters in tile_info
 //              (.z: above tau, .w: equal to tau)
-//   scan       exclusive prefix over the tiles of (above the band + above tau, ties); checks that
-//              exactly k entries will be emitted
+//              and the last CTA of a vector takes the exclusive prefix over the tiles of (above the
+//              band + above tau, ties) and checks that exactly k entries will be emitted
 //   emit       a warp per tile walks the region in index order; the prefix gives the tile's first
 //              output slot, ballots place the kept entries: write (index, value), zero the kept
 //              candidates in delta (delta = v - Q[v], Eq. 3), and on a fused server pass update x
@@ -258,16 +259,23 @@ __global__ void __launch_bounds__(kThreads, is_worker_src(SRC) || SRC == SRC_SRV
 }
 
 // ---------------------------------------------------------------- pick
-// Called by all 1024 threads of a CTA.  h: 4096 counters.  Finds the bin where the count from the
-// top reaches `want` and how many entries are still to take inside it: s_out[0] = bin,
+// Called by all NT threads of a CTA (NT = 1024 or 256).  h: 4096 counters.  Finds the bin where the
+// count from the top reaches `want` and how many entries are still to take inside it: s_out[0] = bin,
 // s_out[1] = remainder, s_out[2] = total count (valid after the final barrier; s_out[0..1] only if
-// 1 <= want <= total).
+// 1 <= want <= total).  s_warp: 32 words.
+template <int NT = 1024>
 __device__ __forceinline__ void cta_pick(const uint32_t* h, uint32_t want, uint32_t* s_warp, uint32_t* s_out) {
+  constexpr uint32_t BPT = kBins1 / NT;  // bins per thread
   const uint32_t tid = threadIdx.x, lane = tid & 31u, wrp = tid >> 5;
-  // thread t owns bins 4*(1023 - t) .. +3, so that a forward scan over threads walks bins downwards
-  const uint32_t b0 = 4u * (1023u - tid);
-  const uint32_t c3 = h[b0 + 3], c2 = h[b0 + 2], c1 = h[b0 + 1], c0 = h[b0];
-  const uint32_t mine = c0 + c1 + c2 + c3;
+  // thread t owns bins BPT*(NT-1 - t) .. +BPT-1, so that a forward scan over threads walks bins downwards
+  const uint32_t b0 = BPT * ((uint32_t)NT - 1u - tid);
+  uint32_t c[BPT];
+  uint32_t mine = 0;
+#pragma unroll
+  for (uint32_t i = 0; i < BPT; ++i) {
+    c[i] = h[b0 + i];
+    mine += c[i];
+  }
   uint32_t incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -277,7 +285,7 @@ __device__ __forceinline__ void cta_pick(const uint32_t* h, uint32_t want, uint3
   if (lane == 31) s_warp[wrp] = incl;
   __syncthreads();
   if (wrp == 0) {
-    const uint32_t w = s_warp[lane];
+    const uint32_t w = lane < (uint32_t)NT / 32u ? s_warp[lane] : 0u;
     uint32_t wi = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -287,39 +295,19 @@ __device__ __forceinline__ void cta_pick(const uint32_t* h, uint32_t want, uint3
     s_warp[lane] = wi - w;  // exclusive prefix of the warp totals
   }
   __syncthreads();
-  const uint32_t above = s_warp[wrp] + incl - mine;  // entries in bins above this thread's four
-  if (tid == 1023) s_out[2] = above + mine;
+  const uint32_t above = s_warp[wrp] + incl - mine;  // entries in bins above this thread's own
+  if (tid == (uint32_t)NT - 1u) s_out[2] = above + mine;
   if (want > above && want <= above + mine) {
-    uint32_t cum = above, tb = b0 + 3;
-    const uint32_t cs[4] = {c3, c2, c1, c0};
+    uint32_t cum = above, tb = b0 + BPT - 1u;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if (want <= cum + cs[i]) { tb = b0 + 3 - i; break; }
-      cum += cs[i];
+    for (int i = (int)BPT - 1; i >= 0; --i) {
+      if (want <= cum + c[i]) { tb = b0 + (uint32_t)i; break; }
+      cum += c[i];
     }
     s_out[0] = tb;
     s_out[1] = want - cum;
   }
   __syncthreads();
-}
-
-// Level-1 pick after a miss, one CTA per vector, on the full histogram written by k_topk_hist.
-__global__ void __launch_bounds__(1024) k_topk_pick1(uint32_t* hist, TopkState* state, uint32_t k) {
-  pdl_prologue();
-  __shared__ uint32_t s_warp[32], s_out[3];
-  const uint32_t tid = threadIdx.x, row = blockIdx.x;
-  uint32_t* h = hist + (uint64_t)row * kBins1;
-  TopkState* st = state + row;
-  if (!st->need_full) return;
-  if (tid == 0) { s_out[0] = 0; s_out[1] = 0; s_out[2] = 0; }
-  __syncthreads();
-  cta_pick(h, k, s_warp, s_out);
-  for (uint32_t b = tid; b < kBins1; b += 1024) h[b] = 0;
-  if (tid != 0) return;
-  st->tb1 = s_out[0];
-  st->k_rem = s_out[1];
-  st->need_mark = 1;
-  st->zeroed_above = (s_out[0] << 19) | 0x7FFFFu;  // mark zeroes the bins above the threshold bin
 }
 
 // ---------------------------------------------------------------- full histogram (after a miss)
@@ -372,46 +360,6 @@ __global__ void __launch_bounds__(kThreads) k_topk_hist(float* v_io, uint64_t d,
   for (uint32_t b = tid; b < kBins1; b += kThreads) {
     const uint32_t c = s_hist[b];
     if (c) atomicAdd(&h[b], c);
-  }
-}
-
-// ---------------------------------------------------------------- mark (after a miss)
-// Rebuilds the tile regions for the exact threshold bin: entries in bins above it are kept (and
-// zeroed), entries inside it are the candidates.  A small grid strides over the tiles.
-__global__ void __launch_bounds__(kThreads) k_topk_mark(float* v_io, uint64_t d, int vec, int keep_error, const TopkState* state,
-                                                        uint2* list, uint64_t cap, uint4* tile_info, uint64_t ntile) {
-  pdl_prologue();
-  __shared__ uint4 s_tot[kThreads / 32];
-  const uint32_t tid = threadIdx.x, row = blockIdx.y;
-  if (!state[row].need_mark) return;
-  const uint32_t lo = state[row].tb1 << 19, hi = lo | 0x7FFFFu;
-  float* vrow = v_io + (uint64_t)row * d;
-  for (uint64_t tile = blockIdx.x; tile < ntile; tile += gridDim.x) {
-    const uint64_t base = tile * kTile;
-    const bool full = vec && base + kTile <= d;
-    float4 v[4];
-    uint32_t cnt[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint64_t e = base + (uint64_t)(j * kThreads + tid) * 4u;
-      cnt[j] = e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u;
-      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (cnt[j]) {
-        if (vec && cnt[j] == 4) {
-          v[j] = *reinterpret_cast<const float4*>(vrow + e);
-        } else {
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            if ((uint32_t)k < cnt[j]) comp(v[j], k) = vrow[e + k];
-        }
-      }
-    }
-    uint2* region = list + (uint64_t)row * cap + base;
-    uint4* info = tile_info + (uint64_t)row * ntile + tile;
-    float* zero_in = keep_error ? vrow : nullptr;
-    if (full) mark_tile<true>(v, cnt, base, lo, hi, zero_in, region, info, s_tot);
-    else mark_tile<false>(v, cnt, base, lo, hi, zero_in, region, info, s_tot);
-    __syncthreads();  // s_tot is written again for the next tile
   }
 }
 
@@ -529,16 +477,75 @@ __device__ __forceinline__ uint32_t gather_tiles(const uint2* lrow, const uint4*
   return kept;
 }
 
-// After a miss: the candidates of the regions that mark rebuilt, made dense.
-__global__ void __launch_bounds__(kThreads) k_topk_compact(const uint2* list, uint64_t cap, const uint4* tile_info,
-                                                           uint64_t ntile, uint2* dense, uint32_t* dense_count,
-                                                           const TopkState* state) {
+// ---------------------------------------------------------------- pick + mark + compact (after a miss)
+// The rest of the full route in one kernel, for the vectors whose prediction missed.  Every CTA takes
+// the level-1 pick for itself from the full histogram k_topk_hist left (4096 counters), rebuilds the
+// regions of its run of tiles for that exact bin -- entries in bins above it are kept (and zeroed in
+// the residual), entries inside it are the candidates -- and copies its candidates into the dense
+// list.  The CTA of a vector that finishes last (a ticket counter, no waiting) records the pick for
+// the kernels that follow and clears the histogram.
+__global__ void __launch_bounds__(kThreads) k_topk_mark(float* v_io, uint64_t d, int vec, int keep_error, TopkState* state,
+                                                        uint2* list, uint64_t cap, uint4* tile_info, uint64_t ntile,
+                                                        uint32_t* hist, uint32_t k, uint2* dense, uint32_t* dense_count,
+                                                        uint32_t* done) {
   pdl_prologue();
-  __shared__ uint32_t s_n[kThreads], s_off[kThreads], s_warp[34];
-  const uint32_t row = blockIdx.y;
-  if (!state[row].need_mark) return;
+  __shared__ uint4 s_tot[kThreads / 32];
+  __shared__ uint32_t s_n[kThreads], s_off[kThreads], s_warp[34], s_out[3];
+  __shared__ uint32_t s_last;
+  const uint32_t tid = threadIdx.x, row = blockIdx.y;
+  TopkState* st = state + row;
+  if (!st->need_full) return;
+  uint32_t* h = hist + (uint64_t)row * kBins1;
+  if (tid == 0) { s_out[0] = 0; s_out[1] = 0; s_out[2] = 0; }
+  __syncthreads();
+  cta_pick<kThreads>(h, k, s_warp, s_out);
+  const uint32_t tb1 = s_out[0], k_rem = s_out[1];
+  const uint32_t lo = tb1 << 19, hi = lo | 0x7FFFFu;
+  float* vrow = v_io + (uint64_t)row * d;
+  // the run of tiles gather_tiles will take for this CTA
+  const uint64_t per = (ntile + gridDim.x - 1) / gridDim.x;
+  const uint64_t c0 = (uint64_t)blockIdx.x * per, c1 = min(ntile, c0 + per);
+  for (uint64_t tile = c0; tile < c1; ++tile) {
+    const uint64_t base = tile * kTile;
+    const bool full = vec && base + kTile <= d;
+    float4 v[4];
+    uint32_t cnt[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint64_t e = base + (uint64_t)(j * kThreads + tid) * 4u;
+      cnt[j] = e < d ? (uint32_t)min((uint64_t)4, d - e) : 0u;
+      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (cnt[j]) {
+        if (vec && cnt[j] == 4) {
+          v[j] = *reinterpret_cast<const float4*>(vrow + e);
+        } else {
+#pragma unroll
+          for (int k2 = 0; k2 < 4; ++k2)
+            if ((uint32_t)k2 < cnt[j]) comp(v[j], k2) = vrow[e + k2];
+        }
+      }
+    }
+    uint2* region = list + (uint64_t)row * cap + base;
+    uint4* info = tile_info + (uint64_t)row * ntile + tile;
+    float* zero_in = keep_error ? vrow : nullptr;
+    if (full) mark_tile<true>(v, cnt, base, lo, hi, zero_in, region, info, s_tot);
+    else mark_tile<false>(v, cnt, base, lo, hi, zero_in, region, info, s_tot);
+    __syncthreads();  // s_tot is written again for the next tile; the tile's region and counts are visible to the CTA
+  }
   gather_tiles<false>(list + (uint64_t)row * cap, tile_info + (uint64_t)row * ntile, ntile, dense + (uint64_t)row * cap, cap,
-                      &dense_count[row], (state[row].tb1 << 19) | 0x7FFFFu, nullptr, s_n, s_off, s_warp);
+                      &dense_count[row], hi, nullptr, s_n, s_off, s_warp);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&done[row], 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  // every CTA of the vector has read the histogram: clear it for the next digit
+  for (uint32_t b = tid; b < kBins1; b += kThreads) h[b] = 0;
+  if (tid != 0) return;
+  done[row] = 0;
+  st->tb1 = tb1;
+  st->k_rem = k_rem;
+  st->zeroed_above = hi;  // mark zeroed the bins above the threshold bin
 }
 
 // ---------------------------------------------------------------- list histogram + pick
@@ -630,11 +637,9 @@ __global__ void __launch_bounds__(1024) k_topk_lhist(const uint2* list, uint64_t
       st->tb1 = s_out[0];
       st->k_rem = s_out[1];
       st->need_full = 0;
-      st->need_mark = 0;
       st->zeroed_above = band_hi;
     } else {
-      st->need_full = 1;  // hist, pick, mark and compact rebuild the regions and the list for the exact bin
-      st->need_mark = 1;
+      st->need_full = 1;  // hist and mark rebuild the regions and the list for the exact bin
       dense_count[row] = 0;
     }
   } else if (LEVEL == 2) {
@@ -1296,9 +1301,8 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     launch_pdl(k_topk_lhist<1>, gl1, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred, io.dev_status);
     launch_pdl(k_topk_hist, gm, kThreads, st, io.v_inout, d, src.vec, io.keep_error, state, pred, list, cap, tile_info, hist);
-    launch_pdl(k_topk_pick1, rows, 1024, st, hist, state, k32);
-    launch_pdl(k_topk_mark, gm, kThreads, st, io.v_inout, d, src.vec, io.keep_error, state, list, cap, tile_info, pl.ntile);
-    launch_pdl(k_topk_compact, gm, kThreads, st, list, cap, tile_info, pl.ntile, dense, list_count, state);
+    launch_pdl(k_topk_mark, gm, kThreads, st, io.v_inout, d, src.vec, io.keep_error, state, list, cap, tile_info, pl.ntile, hist, k32,
+               dense, list_count, done);
     launch_pdl(k_topk_lhist<2>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
                                          k32, pred, io.dev_status);
     launch_pdl(k_topk_lhist<3>, gl, 1024, st, list, cap, tile_info, pl.ntile, dense, list_count, kept_count, state, hist, done,
@@ -1309,7 +1313,7 @@ cudaError_t launch_topk(int srck, const SrcParams& src, const TopkPlan& pl, void
     launch_pdl(k_topk_emit_list, ge, kThreads, st, io.v_inout, d, state, list, cap, tile_info, seg, pl.ntile,
                                               reinterpret_cast<uint8_t*>(io.idx), io.payload_stride, 0, off_val, k32, io.x,
                                               io.gamma, io.keep_error, io.span_off);
-    count_launches(10);
+    count_launches(8);
     return cudaGetLastError();
   } else {
 #define DSQ_P1(S) launch_pdl(k_topk_pass1_basic<S>, g1b, kThreads, st, src, io.v_inout, hist, span)
