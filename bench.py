@@ -49,13 +49,13 @@ HEADLINE = 5                 # the largest one that fits one GPU
 # (a multi-pass capture must stay small) is scaled by the entries one launch processes: the
 # traffic of a streaming kernel grows in proportion.
 NCU_CAPTURES = {
-    "sign1": ("k_chunked<SIGN1, WORKER, 4, 256>", 748182784 + 332558080, 8 * 11_689_512, "776947eec84228a6"),
-    "qsgd": ("k_chunked<QSGD, WORKER, 2, 256>", 1073776000 + 630281472, 8 * 16_777_216, "776947eec84228a6"),
+    "sign1": ("k_chunked<SIGN1, WORKER, 4, 256>", 748182272 + 331582464, 8 * 11_689_512, "3e80faecea9d3b0a"),
+    "qsgd": ("k_chunked<QSGD, WORKER, 2, 256>", 1073773000 + 630182144, 8 * 16_777_216, "3e80faecea9d3b0a"),
     # the first kernel of the top-k worker pass alone (v read once, written once); the selection that follows it
     # moves a few percent of that
-    "topk": ("k_topk_pass1<WORKER>", 537250304 + 221670400, 16 * 4_194_304, "473ea00871451d04"),
-    "clip": ("k_clip<WORKER, 16>", 748329216 + 508803584, 8 * 11_689_512, "8f64db8f3c6b7019"),
-    "rsparse": ("k_rsparse<WORKER>", 748263680 + 332954624, 8 * 11_689_512, "8f64db8f3c6b7019"),
+    "topk": ("k_topk_pass1<WORKER>", 537251328 + 221441280, 16 * 4_194_304, "8493784d4c9f8058"),
+    "clip": ("k_clip<WORKER, 16>", 748323328 + 508980736, 8 * 11_689_512, "ccfe82e0a4de6e6b"),
+    "rsparse": ("k_rsparse<WORKER>", 748263680 + 333547008, 8 * 11_689_512, "ccfe82e0a4de6e6b"),
 }
 KERNEL_SOURCES = {  # files whose change invalidates the captured counters
     "sign1": ("dsq_chunked.cuh", "dsq_common.cuh", "dsq_internal.h"),
