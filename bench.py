@@ -592,7 +592,7 @@ def main():
     ap.add_argument("--min-seconds", type=float, default=0.5, help="GPU time to collect per workload (blocks are repeated)")
     ap.add_argument("--max-blocks", type=int, default=40)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--cpu-steps", type=int, default=5, help="oracle steps timed for cpu_baseline (about 2.3 s each on the headline sample)")
     ap.add_argument("--dump-steps", action="store_true", help="add the per-step times to the JSON line")
     ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this d (profiling captures)")
     args = ap.parse_args()
