@@ -276,7 +276,7 @@ def test_many_workers_and_one_worker():
     run_lockstep(7, 20_000, TOPK(200), TOPK(200), randn_steps(7, 20_000, 2))
 
 
-# ------------------------------------------------------------------ the five workloads, scaled down
+# ------------------------------------------------------------------ the workloads, scaled down
 
 @pytest.mark.parametrize("wid", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12])
 def test_workload_recipes_scaled(wid):
